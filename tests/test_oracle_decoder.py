@@ -1,0 +1,141 @@
+"""Pins for the oracle's decoder: closed forms, and an independent dense float64 decoder."""
+import ctypes as C
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import spd_inputs as si
+from oracle import spd_oracle as so
+from tests.ref_decoder import dense_forward, f64
+
+
+def _bits(vals):
+    return so.bf16_bits(torch.tensor(vals, dtype=torch.float32).to(torch.bfloat16))
+
+
+def test_round_bf16_matches_library_rounding():
+    rng = np.random.default_rng(0)
+    xs = np.concatenate([rng.standard_normal(2000).astype(np.float32) * 3,
+                         np.array([1.00390625, 1.01171875, -1.00390625, 0.0, 3.0e38, 1e-40], np.float32)])
+    want = torch.from_numpy(xs).to(torch.bfloat16).to(torch.float32).numpy()
+    got = np.array([so.lib().orc_round_bf16(float(x)) for x in xs], np.float32)
+    assert np.array_equal(got, want)
+    # exact ties go to the even mantissa: 1 + 2^-8 -> 1, 1 + 3*2^-8 -> 1 + 2^-6
+    assert got[2000] == 1.0 and got[2001] == 1.015625
+
+
+def test_rmsnorm_closed_forms():
+    d = 8
+    y = np.zeros(d)
+    g = _bits([0.5, 1, 2, 1, 1, 1, 1, 1])
+    x = np.full(d, -3.0)
+    so.lib().orc_rmsnorm(x.ctypes.data, g.ctypes.data, d, 0.0, y.ctypes.data)
+    assert np.allclose(y, -np.array([0.5, 1, 2, 1, 1, 1, 1, 1]), atol=1e-15)      # constant vector -> sign * gain
+    x = np.array([3.0, 4.0, 0, 0, 0, 0, 0, 0])
+    so.lib().orc_rmsnorm(x.ctypes.data, g.ctypes.data, d, 0.0, y.ctypes.data)
+    assert np.allclose(y[:2], [0.5 * 3 / math.sqrt(25 / 8), 4 / math.sqrt(25 / 8)], atol=1e-15)
+    so.lib().orc_rmsnorm(x.ctypes.data, g.ctypes.data, d, 1.0, y.ctypes.data)
+    assert np.allclose(y[1], 4 / math.sqrt(25 / 8 + 1.0), atol=1e-15)               # eps sits inside the root
+
+
+def test_rope_closed_forms():
+    hd = 8
+    x0 = np.arange(1.0, hd + 1)
+    x = x0.copy()
+    so.lib().orc_rope(x.ctypes.data, hd, 0, 10000.0)
+    assert np.array_equal(x, x0)                                                    # position 0 is the identity
+    x = x0.copy()
+    so.lib().orc_rope(x.ctypes.data, hd, 3, 10000.0)
+    assert np.allclose(x[0::2] ** 2 + x[1::2] ** 2, x0[0::2] ** 2 + x0[1::2] ** 2)  # a rotation per pair
+    # pair 0 turns by pos radians, pair i by pos * theta^(-2i/hd); counter-clockwise
+    assert np.allclose(x[:2], [1 * math.cos(3) - 2 * math.sin(3), 1 * math.sin(3) + 2 * math.cos(3)])
+    a = 3 * 10000.0 ** (-2 * 2 / 8)
+    assert np.allclose(x[4:6], [5 * math.cos(a) - 6 * math.sin(a), 5 * math.sin(a) + 6 * math.cos(a)])
+    # relative property: <rope(q,p), rope(k,s)> depends on p - s only
+    q, k = np.random.default_rng(1).standard_normal((2, hd))
+    def dot(p, s):
+        a_, b_ = q.copy(), k.copy()
+        so.lib().orc_rope(a_.ctypes.data, hd, p, 10000.0)
+        so.lib().orc_rope(b_.ctypes.data, hd, s, 10000.0)
+        return float(a_ @ b_)
+    assert abs(dot(7, 4) - dot(13, 10)) < 1e-12 and abs(dot(7, 4) - dot(8, 4)) > 1e-6
+
+
+def test_attention_closed_forms():
+    hd, T, stride = 4, 3, 8
+    K = np.zeros((T, stride), np.float32)
+    V = np.zeros((T, stride), np.float32)
+    V[:, :hd] = [[1, 2, 3, 4], [5, 6, 7, 8], [-1, 0, 1, 2]]
+    q = np.array([0.3, -0.2, 0.1, 0.9])
+    o = np.zeros(hd)
+    so.lib().orc_attention_head(q.ctypes.data, K.ctypes.data, V.ctypes.data, 1, hd, stride, o.ctypes.data)
+    assert np.array_equal(o, V[0, :hd])                                             # one position: output = v
+    so.lib().orc_attention_head(q.ctypes.data, K.ctypes.data, V.ctypes.data, 3, hd, stride, o.ctypes.data)
+    assert np.allclose(o, V[:, :hd].mean(0))                                        # equal scores: plain mean
+    K[1, :hd] = q * 2
+    so.lib().orc_attention_head(q.ctypes.data, K.ctypes.data, V.ctypes.data, 3, hd, stride, o.ctypes.data)
+    s = float(q @ (q * 2)) / math.sqrt(hd)                                          # scale is 1/sqrt(hd)
+    w = np.array([1.0, math.exp(s), 1.0])
+    assert np.allclose(o, (w[:, None] * V[:, :hd]).sum(0) / w.sum())
+
+
+@pytest.mark.parametrize("kv_dtype,tol", [("f32", 2e-6), ("bf16", 2e-3)])
+def test_prefill_logits_match_independent_dense_decoder(tiny_inputs, kv_dtype, tol):
+    wl, weights, tables, prefix = tiny_inputs
+    cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, kv_dtype)
+    o = so.Oracle(cfg, weights, tables)
+    o.prefill(prefix)
+    X = f64(weights["tok_emb"])[torch.tensor(prefix)]
+    logits, trace = dense_forward(weights, wl.shape, X, kv_dtype)
+    assert np.abs(o.logits() - logits[-1].numpy()).max() < tol
+    tr = o.trace()
+    for l in range(wl.shape.n_layers):
+        assert np.abs(tr[l, 0] - trace[2 * l][-1].numpy()).max() < tol
+        assert np.abs(tr[l, 1] - trace[2 * l + 1][-1].numpy()).max() < tol
+
+
+def test_cached_superposed_steps_match_dense_pass_over_all_input_rows(tiny_inputs):
+    """Eq. 3 + the shared cache: step logits equal a cache-free dense pass whose input rows are the
+    prefix embeddings followed by the superposed embeddings sum_i gamma_i E[token_i]."""
+    wl, weights, tables, prefix = tiny_inputs
+    cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "f32")
+    o = so.Oracle(cfg, weights, tables)
+    E = f64(weights["tok_emb"])
+    rows = [E[t] for t in prefix]
+    ids, g = o.prefill(prefix)
+    for _ in range(4):
+        assert abs(g.sum() - 1) < 1e-12
+        rows.append(sum(float(g[i]) * E[int(ids[i])] for i in range(3)))
+        ids, par, g = o.step()
+        logits, _ = dense_forward(weights, wl.shape, torch.stack(rows), "f32")
+        assert np.abs(o.logits() - logits[-1].numpy()).max() < 2e-6
+
+
+def test_dense_prefill_equals_token_by_token_decoding(tiny_inputs):
+    wl, weights, tables, prefix = tiny_inputs
+    for kv in ("f32", "bf16"):
+        cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, kv)
+        a = so.Oracle(cfg, weights, tables)
+        b = so.Oracle(cfg, weights, tables)
+        a.prefill(prefix)
+        for t in prefix:
+            b.feed_token(t)
+        assert a.T() == b.T() == len(prefix)
+        assert np.abs(a.logits() - b.logits()).max() < 1e-12
+        ka, va = a.kv_cache()
+        kb, vb = b.kv_cache()
+        assert np.array_equal(ka, kb) and np.array_equal(va, vb)
+
+
+def test_bf16_cache_holds_bf16_values(tiny_inputs):
+    wl, weights, tables, prefix = tiny_inputs
+    cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "bf16")
+    o = so.Oracle(cfg, weights, tables)
+    o.prefill(prefix)
+    k, v = o.kv_cache()
+    for a in (k[:, :16], v[:, :16]):
+        t = torch.from_numpy(np.ascontiguousarray(a))
+        assert torch.equal(t.to(torch.bfloat16).to(torch.float32), t) and t.abs().max() > 0
+    assert np.all(k[:, 16:] == 0)
