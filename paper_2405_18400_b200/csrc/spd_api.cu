@@ -1,0 +1,491 @@
+// Host side of the C ABI declared in include/spd.h: argument checks, workspace layout, launches.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "spd.h"
+#include "spd_params.h"
+
+extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size_t dyn_smem, cudaStream_t stream);
+extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm);
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e, const char *what) {
+  std::snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
+  cudaGetLastError();
+  return SPD_ECUDA;
+}
+#define SPD_CUDA(call)                                 \
+  do {                                                 \
+    cudaError_t e_ = (call);                           \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+  } while (0)
+
+constexpr size_t kPartBytes = 20480;  // per-block scratch after the ring: row partials / attention merge / tail
+constexpr size_t kSmemLimit = 232448; // 227 KB opt-in maximum per block on sm_100
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
+      trace, total;
+};
+
+bool valid_config(const spd_config *c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->d_ffn < 8 || c->vocab < 1 || c->max_pos < 2) return false;
+  if (c->d_model % 8 || c->d_ffn % 8 || c->d_model % c->n_heads) return false;
+  const int hd = c->d_model / c->n_heads;
+  if (hd % 32 || hd > 256) return false;
+  if (c->vocab > 65535) return false;
+  if (c->d_model > spd::kMaxVec * spd::kConsumerThreads * 8 || c->d_ffn > spd::kMaxVec * spd::kConsumerThreads * 8) return false;
+  if (c->k < 1 || c->k > SPD_MAX_K) return false;
+  if (c->n_min < 2 || c->n_max > SPD_MAX_N) return false;
+  if (!(c->tau > 0.f) || !(c->delta > 0.f) || c->delta > 1.f || !(c->alpha >= 0.f) || c->alpha > 1.f) return false;
+  if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
+  if (c->eos_id != -1) return false;
+  if (c->kv_dtype != 0 && c->kv_dtype != 1) return false;
+  return true;
+}
+
+Layout make_layout(const spd_config &c, int grid) {
+  Layout L{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = off;
+    off = align_up(off + bytes, 256);
+    return at;
+  };
+  const size_t kvb = (size_t)c.n_layers * c.max_pos * c.d_model * (c.kv_dtype ? 2 : 4);
+  const int hd = c.d_model / c.n_heads;
+  L.kcache = take(kvb);
+  L.vcache = take(kvb);
+  L.rope = take((size_t)c.max_pos * (hd / 2) * sizeof(float2));
+  L.layers = take((size_t)c.n_layers * sizeof(spd::LayerW));
+  L.h = take((size_t)c.d_model * 4);
+  L.q = take((size_t)c.d_model * 4);
+  L.u = take((size_t)c.d_ffn * 4);
+  L.logits = take((size_t)c.vocab * 4);
+  L.opart = take((size_t)c.n_heads * spd::kMaxSplit * hd * 4);
+  L.oml = take((size_t)c.n_heads * spd::kMaxSplit * sizeof(float2));
+  L.pk_val = take((size_t)grid * c.k * 4);
+  L.pk_id = take((size_t)grid * c.k * 4);
+  L.pk_ms = take((size_t)grid * sizeof(float2));
+  L.state = take(sizeof(spd::State));
+  L.hist_tok = take((size_t)c.max_pos * c.k * 4);
+  L.hist_par = take((size_t)c.max_pos * c.k * 4);
+  L.prefix = take((size_t)c.max_pos * 4);
+  L.trace = take((size_t)c.n_layers * 2 * c.d_model * 4);
+  L.total = off;
+  return L;
+}
+
+constexpr int kLayoutGrid = 1024;  // workspace is sized for up to this many blocks
+
+}  // namespace
+
+struct spd_ctx {
+  spd_config cfg;
+  spd::KParams kp;
+  Layout lay;
+  uint8_t *ws;
+  cudaStream_t stream;
+  int device;
+  int grid;
+  size_t dyn_smem;
+  bool prefilled;
+  int32_t m;       // prefix length
+  int32_t n_gen;   // tokens generated per draft
+  int64_t launches;
+};
+
+namespace {
+
+int pick_ring(const spd_config &c, int32_t stage_bytes, int32_t n_stages, int32_t *out_stage, int32_t *out_n) {
+  const size_t maxrow = (size_t)2 * (c.d_model > c.d_ffn ? c.d_model : c.d_ffn);
+  size_t sb = stage_bytes > 0 ? (size_t)stage_bytes : 32768;
+  if (stage_bytes <= 0 && sb < maxrow) sb = align_up(maxrow, 1024);
+  if (sb % 128 || sb < maxrow) return SPD_EINVAL;
+  const size_t avail = kSmemLimit - kPartBytes - 2048;  // static shared memory and alignment slack
+  int ns = n_stages > 0 ? n_stages : (int)(avail / sb);
+  if (ns > spd::kMaxStages) ns = spd::kMaxStages;
+  if (ns < 2 || (size_t)ns * sb > avail) return SPD_EINVAL;
+  *out_stage = (int32_t)sb;
+  *out_n = ns;
+  return SPD_OK;
+}
+
+int check_device_error(spd_ctx *ctx) {
+  int32_t err[2] = {0, 0};
+  SPD_CUDA(cudaMemcpyAsync(err, ctx->ws + ctx->lay.state + offsetof(spd::State, err), sizeof err, cudaMemcpyDeviceToHost,
+                           ctx->stream));
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));
+  return err[0];
+}
+
+int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0) {
+  spd::KParams &kp = ctx->kp;
+  kp.mode = mode;
+  kp.n_iters = n_iters;
+  kp.pos0 = pos0;
+  kp.step0 = step0;
+  // barrier counters, abort flag and error word start from zero at every launch
+  SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, offsetof(spd::State, win_len), ctx->stream));
+  SPD_CUDA(spd_internal_launch(&kp, ctx->grid, ctx->dyn_smem, ctx->stream));
+  ctx->launches += 1;
+  return SPD_OK;
+}
+
+int set_device(const spd_ctx *ctx) {
+  int dev = -1;
+  SPD_CUDA(cudaGetDevice(&dev));
+  if (dev != ctx->device) SPD_CUDA(cudaSetDevice(ctx->device));
+  return SPD_OK;
+}
+
+int read_state(spd_ctx *ctx, size_t field_off, void *dst, size_t bytes) {
+  SPD_CUDA(cudaMemcpyAsync(dst, ctx->ws + ctx->lay.state + field_off, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+  return SPD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *spd_strerror(int status) {
+  switch (status) {
+    case SPD_OK: return "ok";
+    case SPD_EINVAL: return "invalid argument";
+    case SPD_ESTATE: return "call out of order (prefill first)";
+    case SPD_ERANGE: return "value out of range";
+    case SPD_ENOMEM: return "buffer too small";
+    case SPD_ECUDA: return "CUDA runtime error";
+    case SPD_ETABLE: return "n-gram table probe exceeded its bound";
+    case SPD_ETIMEOUT: return "bounded device wait expired";
+    default: return "unknown status";
+  }
+}
+
+const char *spd_last_cuda_error(void) { return g_cuda_err; }
+
+int spd_workspace_bytes(const spd_config *cfg, size_t *bytes) {
+  if (!valid_config(cfg) || !bytes) return SPD_EINVAL;
+  *bytes = make_layout(*cfg, kLayoutGrid).total;
+  return SPD_OK;
+}
+
+int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_table *tables, int32_t n_tables, void *workspace,
+               size_t workspace_bytes, spd_ctx **out) {
+  if (!valid_config(cfg) || !w || !workspace || !out) return SPD_EINVAL;
+  if (n_tables < 0 || n_tables > spd::kMaxTables || (n_tables > 0 && !tables)) return SPD_EINVAL;
+  if ((uintptr_t)workspace % 256) return SPD_EINVAL;
+  if (!w->tok_emb || !w->final_norm || !w->lm_head || !w->attn_norm || !w->wqkv || !w->wo || !w->ffn_norm || !w->wgate_up ||
+      !w->wdown)
+    return SPD_EINVAL;
+  auto misaligned = [](const void *p) { return p == nullptr || ((uintptr_t)p % 16) != 0; };
+  if (misaligned(w->tok_emb) || misaligned(w->final_norm) || misaligned(w->lm_head)) return SPD_EINVAL;
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (misaligned(w->attn_norm[l]) || misaligned(w->wqkv[l]) || misaligned(w->wo[l]) || misaligned(w->ffn_norm[l]) ||
+        misaligned(w->wgate_up[l]) || misaligned(w->wdown[l]))
+      return SPD_EINVAL;
+  for (int t = 0; t < n_tables; ++t) {
+    const spd_ngram_table &tb = tables[t];
+    if (tb.n < 2 || tb.n > SPD_MAX_N || misaligned(tb.ngram) || misaligned(tb.ctx)) return SPD_EINVAL;
+    if (!tb.ngram_slots || (tb.ngram_slots & (tb.ngram_slots - 1)) || !tb.ctx_slots || (tb.ctx_slots & (tb.ctx_slots - 1)))
+      return SPD_EINVAL;
+    for (int s = 0; s < t; ++s)
+      if (tables[s].n >= tb.n) return SPD_EINVAL;  // ascending orders, one table per order
+  }
+  const Layout lay = make_layout(*cfg, kLayoutGrid);
+  if (workspace_bytes < lay.total) return SPD_ENOMEM;
+
+  spd_ctx *ctx = new (std::nothrow) spd_ctx();
+  if (!ctx) return SPD_ENOMEM;
+  ctx->cfg = *cfg;
+  ctx->lay = lay;
+  ctx->ws = static_cast<uint8_t *>(workspace);
+  ctx->stream = static_cast<cudaStream_t>(cfg->stream);
+  ctx->prefilled = false;
+  ctx->m = ctx->n_gen = 0;
+  ctx->launches = 0;
+  auto fail = [&](int rc) {
+    delete ctx;
+    return rc;
+  };
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDevice"));
+  cudaDeviceProp prop;
+  e = cudaGetDeviceProperties(&prop, ctx->device);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDeviceProperties"));
+  if (!prop.cooperativeLaunch) return fail(SPD_EINVAL);
+  ctx->grid = prop.multiProcessorCount < kLayoutGrid ? prop.multiProcessorCount : kLayoutGrid;
+
+  spd::KParams &kp = ctx->kp;
+  std::memset(&kp, 0, sizeof kp);
+  int rc = pick_ring(*cfg, 0, 0, &kp.stage_bytes, &kp.n_stages);
+  if (rc) return fail(rc);
+  ctx->dyn_smem = (size_t)kp.stage_bytes * kp.n_stages + kPartBytes;
+  int per_sm = 0;
+  e = spd_internal_prepare(ctx->dyn_smem, &per_sm);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "kernel attributes"));
+  if (per_sm < 1) return fail(SPD_EINVAL);
+
+  const int hd = cfg->d_model / cfg->n_heads;
+  kp.L = cfg->n_layers; kp.d = cfg->d_model; kp.H = cfg->n_heads; kp.hd = hd; kp.f = cfg->d_ffn; kp.V = cfg->vocab;
+  kp.max_pos = cfg->max_pos; kp.eps = cfg->rms_eps; kp.kv_bf16 = cfg->kv_dtype;
+  kp.tok_emb = static_cast<const __nv_bfloat16 *>(w->tok_emb);
+  kp.final_norm = static_cast<const __nv_bfloat16 *>(w->final_norm);
+  kp.lm_head = static_cast<const __nv_bfloat16 *>(w->lm_head);
+  kp.k = cfg->k; kp.n_min = cfg->n_min; kp.n_max = cfg->n_max; kp.n_tables = n_tables;
+  for (int i = 0; i < 8; ++i) kp.lambda[i] = cfg->lambda[i];
+  kp.alpha = cfg->alpha;
+  kp.inv_tau = 1.0f / cfg->tau;
+  kp.log_delta = std::log(cfg->delta);
+  for (int t = 0; t < n_tables; ++t) {
+    kp.tab[t].n = tables[t].n;
+    kp.tab[t].ngram = static_cast<const SpdSlot *>(tables[t].ngram);
+    kp.tab[t].ctx = static_cast<const SpdSlot *>(tables[t].ctx);
+    kp.tab[t].ngram_mask = tables[t].ngram_slots - 1;
+    kp.tab[t].ctx_mask = tables[t].ctx_slots - 1;
+  }
+  uint8_t *ws = ctx->ws;
+  kp.kcache = ws + lay.kcache; kp.vcache = ws + lay.vcache;
+  kp.rope = reinterpret_cast<const float2 *>(ws + lay.rope);
+  kp.layers = reinterpret_cast<const spd::LayerW *>(ws + lay.layers);
+  kp.h = reinterpret_cast<float *>(ws + lay.h); kp.q = reinterpret_cast<float *>(ws + lay.q);
+  kp.u = reinterpret_cast<float *>(ws + lay.u); kp.logits = reinterpret_cast<float *>(ws + lay.logits);
+  kp.opart = reinterpret_cast<float *>(ws + lay.opart); kp.oml = reinterpret_cast<float2 *>(ws + lay.oml);
+  kp.pk_val = reinterpret_cast<float *>(ws + lay.pk_val); kp.pk_id = reinterpret_cast<int32_t *>(ws + lay.pk_id);
+  kp.pk_ms = reinterpret_cast<float2 *>(ws + lay.pk_ms);
+  kp.st = reinterpret_cast<spd::State *>(ws + lay.state);
+  kp.hist_tok = reinterpret_cast<int32_t *>(ws + lay.hist_tok); kp.hist_par = reinterpret_cast<int32_t *>(ws + lay.hist_par);
+  kp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
+  kp.trace = reinterpret_cast<float *>(ws + lay.trace);
+
+  // rotary table: cos / sin of pos * theta^(-2i/hd), evaluated in double and rounded once
+  std::vector<float2> rope((size_t)cfg->max_pos * (hd / 2));
+  for (int pos = 0; pos < cfg->max_pos; ++pos)
+    for (int i = 0; i < hd / 2; ++i) {
+      const double ang = (double)pos * std::pow((double)cfg->rope_theta, -2.0 * i / hd);
+      rope[(size_t)pos * (hd / 2) + i] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+    }
+  std::vector<spd::LayerW> layers(cfg->n_layers);
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    layers[l].attn_norm = static_cast<const __nv_bfloat16 *>(w->attn_norm[l]);
+    layers[l].wqkv = static_cast<const __nv_bfloat16 *>(w->wqkv[l]);
+    layers[l].wo = static_cast<const __nv_bfloat16 *>(w->wo[l]);
+    layers[l].ffn_norm = static_cast<const __nv_bfloat16 *>(w->ffn_norm[l]);
+    layers[l].wgate_up = static_cast<const __nv_bfloat16 *>(w->wgate_up[l]);
+    layers[l].wdown = static_cast<const __nv_bfloat16 *>(w->wdown[l]);
+  }
+  cudaStream_t s = ctx->stream;
+  e = cudaMemcpyAsync(ws + lay.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + lay.layers, layers.data(), layers.size() * sizeof(spd::LayerW), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.state, 0, sizeof(spd::State), s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.trace, 0, (size_t)cfg->n_layers * 2 * cfg->d_model * 4, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "workspace initialisation"));
+  *out = ctx;
+  return SPD_OK;
+}
+
+int spd_destroy(spd_ctx *ctx) {
+  delete ctx;
+  return SPD_OK;
+}
+
+int spd_set_ring(spd_ctx *ctx, int32_t stage_bytes, int32_t n_stages) {
+  if (!ctx) return SPD_EINVAL;
+  int32_t sb, ns;
+  int rc = pick_ring(ctx->cfg, stage_bytes, n_stages, &sb, &ns);
+  if (rc) return rc;
+  if ((rc = set_device(ctx))) return rc;
+  const size_t dyn = (size_t)sb * ns + kPartBytes;
+  int per_sm = 0;
+  SPD_CUDA(spd_internal_prepare(dyn > ctx->dyn_smem ? dyn : ctx->dyn_smem, &per_sm));
+  if (per_sm < 1) return SPD_EINVAL;
+  ctx->kp.stage_bytes = sb;
+  ctx->kp.n_stages = ns;
+  ctx->dyn_smem = dyn;
+  return SPD_OK;
+}
+
+int spd_prefill(spd_ctx *ctx, const int32_t *prefix_ids, int32_t m, int32_t *out_ids, float *out_gamma) {
+  if (!ctx || !prefix_ids) return SPD_EINVAL;
+  const spd_config &c = ctx->cfg;
+  if (m < 1 || m >= c.max_pos) return SPD_ERANGE;
+  for (int i = 0; i < m; ++i)
+    if (prefix_ids[i] < 0 || prefix_ids[i] >= c.vocab) return SPD_ERANGE;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  // fresh draft state: every history window holds the end of the prefix
+  spd::State st;
+  std::memset(&st, 0, sizeof st);
+  st.win_len = m < spd::kWin ? m : spd::kWin;
+  for (int i = 0; i < c.k; ++i)
+    for (int j = 0; j < st.win_len; ++j) st.win[i][spd::kWin - st.win_len + j] = prefix_ids[m - st.win_len + j];
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.state, &st, sizeof st, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix, prefix_ids, (size_t)m * 4, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));  // st and the caller's ids may go out of scope
+  ctx->prefilled = false;
+  if ((rc = launch(ctx, spd::kModePrefill, m, 0, 0))) return rc;
+  int32_t ids[SPD_MAX_K];
+  float gamma[SPD_MAX_K];
+  if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;
+  if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
+  if ((rc = check_device_error(ctx))) return rc;
+  ctx->prefilled = true;
+  ctx->m = m;
+  ctx->n_gen = 1;
+  for (int i = 0; i < c.k; ++i) {
+    if (out_ids) out_ids[i] = ids[i];
+    if (out_gamma) out_gamma[i] = gamma[i];
+  }
+  return SPD_OK;
+}
+
+int spd_generate_async(spd_ctx *ctx, int32_t n_steps) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return SPD_ESTATE;
+  if (n_steps < 1) return SPD_ERANGE;
+  const int pos0 = ctx->m + ctx->n_gen - 1;  // position of the first superposed input of this launch
+  if (pos0 + n_steps > ctx->cfg.max_pos || ctx->n_gen + n_steps > ctx->cfg.max_pos) return SPD_ERANGE;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  if ((rc = launch(ctx, spd::kModeDecode, n_steps, pos0, ctx->n_gen))) return rc;
+  ctx->n_gen += n_steps;
+  return SPD_OK;
+}
+
+int spd_sync(spd_ctx *ctx) {
+  if (!ctx) return SPD_EINVAL;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  rc = check_device_error(ctx);
+  if (rc) ctx->prefilled = false;
+  return rc;
+}
+
+int spd_step(spd_ctx *ctx, int32_t *out_ids, int32_t *out_parent, float *out_gamma) {
+  int rc = spd_generate_async(ctx, 1);
+  if (rc) return rc;
+  const int k = ctx->cfg.k;
+  int32_t ids[SPD_MAX_K], par[SPD_MAX_K];
+  float gamma[SPD_MAX_K];
+  const size_t row = (size_t)(ctx->n_gen - 1) * k * 4;
+  SPD_CUDA(cudaMemcpyAsync(ids, ctx->ws + ctx->lay.hist_tok + row, (size_t)k * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  SPD_CUDA(cudaMemcpyAsync(par, ctx->ws + ctx->lay.hist_par + row, (size_t)k * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
+  if ((rc = spd_sync(ctx))) return rc;
+  for (int i = 0; i < k; ++i) {
+    if (out_ids) out_ids[i] = ids[i];
+    if (out_parent) out_parent[i] = par[i];
+    if (out_gamma) out_gamma[i] = gamma[i];
+  }
+  return SPD_OK;
+}
+
+int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *out_len, float *out_logp, float *out_gamma) {
+  int rc = spd_generate_async(ctx, n_steps);
+  if (rc) return rc;
+  const int k = ctx->cfg.k, len = ctx->n_gen;
+  std::vector<int32_t> tok((size_t)len * k), par((size_t)len * k);
+  float logp[SPD_MAX_K], gamma[SPD_MAX_K];
+  SPD_CUDA(cudaMemcpyAsync(tok.data(), ctx->ws + ctx->lay.hist_tok, tok.size() * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  SPD_CUDA(cudaMemcpyAsync(par.data(), ctx->ws + ctx->lay.hist_par, par.size() * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  if ((rc = read_state(ctx, offsetof(spd::State, logP), logp, sizeof logp))) return rc;
+  if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
+  if ((rc = spd_sync(ctx))) return rc;
+  if (out_tokens) {
+    // follow each surviving draft's parent links back to the first timestep
+    for (int r = 0; r < k; ++r) {
+      int cur = r;
+      for (int s = len - 1; s >= 0; --s) {
+        out_tokens[(size_t)r * len + s] = tok[(size_t)s * k + cur];
+        cur = par[(size_t)s * k + cur];
+      }
+    }
+  }
+  if (out_len) *out_len = len;
+  for (int i = 0; i < k; ++i) {
+    if (out_logp) out_logp[i] = logp[i];
+    if (out_gamma) out_gamma[i] = gamma[i];
+  }
+  return SPD_OK;
+}
+
+int64_t spd_launch_count(const spd_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes) {
+  if (!ctx || !host_buf) return SPD_EINVAL;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  const spd_config &c = ctx->cfg;
+  const int k = c.k;
+  const uint8_t *st = ctx->ws + ctx->lay.state;
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));
+  auto copy = [&](const void *src, size_t n) -> int {
+    if (bytes < n) return SPD_ENOMEM;
+    SPD_CUDA(cudaMemcpy(host_buf, src, n, cudaMemcpyDeviceToHost));
+    return SPD_OK;
+  };
+  auto copy_rows = [&](const void *src, int rows, size_t row_bytes, size_t row_stride) -> int {
+    if (bytes < (size_t)rows * row_bytes) return SPD_ENOMEM;
+    SPD_CUDA(cudaMemcpy2D(host_buf, row_bytes, src, row_stride, row_bytes, rows, cudaMemcpyDeviceToHost));
+    return SPD_OK;
+  };
+  switch (what) {
+    case SPD_DBG_LOGITS: return copy(ctx->ws + ctx->lay.logits, (size_t)c.vocab * 4);
+    case SPD_DBG_CAND_TOK: return copy(st + offsetof(spd::State, cand_tok), (size_t)k * 4);
+    case SPD_DBG_CAND_LP: return copy(st + offsetof(spd::State, cand_lp), (size_t)k * 4);
+    case SPD_DBG_LOGP_IN: return copy(st + offsetof(spd::State, logP_in), (size_t)k * 4);
+    case SPD_DBG_SCORE: return copy(st + offsetof(spd::State, score), (size_t)k * k * 4);
+    case SPD_DBG_PNG: return copy(st + offsetof(spd::State, png), (size_t)k * k * 4);
+    case SPD_DBG_CNT: return copy(st + offsetof(spd::State, cnt), (size_t)k * k * spd::kMaxTables * 4);
+    case SPD_DBG_TOT: return copy(st + offsetof(spd::State, tot), (size_t)k * spd::kMaxTables * 4);
+    case SPD_DBG_SEL: return copy(st + offsetof(spd::State, sel), (size_t)k * 4);
+    case SPD_DBG_LOGP: return copy(st + offsetof(spd::State, logP), (size_t)k * 4);
+    case SPD_DBG_HIST_IN: return copy_rows(st + offsetof(spd::State, win_in), k, spd::kWin * 4, spd::kWin * 4);
+    case SPD_DBG_TRACE: return copy(ctx->ws + ctx->lay.trace, (size_t)c.n_layers * 2 * c.d_model * 4);
+    case SPD_DBG_HIDDEN: return copy(ctx->ws + ctx->lay.h, (size_t)c.d_model * 4);
+    default: return SPD_EINVAL;
+  }
+}
+
+int spd_debug_score(spd_ctx *ctx, const int32_t *hist, int32_t hist_len, const float *logp, const int32_t *cand_tok,
+                    const float *cand_lp) {
+  if (!ctx || !hist || !logp || !cand_tok || !cand_lp) return SPD_EINVAL;
+  if (hist_len < 0 || hist_len > spd::kWin) return SPD_ERANGE;
+  const spd_config &c = ctx->cfg;
+  for (int i = 0; i < c.k; ++i) {
+    if (cand_tok[i] < 0 || cand_tok[i] >= c.vocab) return SPD_ERANGE;
+    for (int j = 0; j < hist_len; ++j)
+      if (hist[i * hist_len + j] < 0 || hist[i * hist_len + j] >= c.vocab) return SPD_ERANGE;
+  }
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  spd::State st;
+  std::memset(&st, 0, sizeof st);
+  st.win_len = hist_len;
+  for (int i = 0; i < c.k; ++i) {
+    for (int j = 0; j < hist_len; ++j) st.win[i][spd::kWin - hist_len + j] = hist[i * hist_len + j];
+    st.logP[i] = logp[i];
+    st.cand_tok[i] = cand_tok[i];
+    st.cand_lp[i] = cand_lp[i];
+  }
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.state, &st, sizeof st, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));
+  ctx->prefilled = false;  // the draft state no longer belongs to a decoding run
+  // launch() zeroes the head of the state only; the fields set above lie behind it
+  if ((rc = launch(ctx, spd::kModeScoreOnly, 0, 0, 0))) return rc;
+  return spd_sync(ctx);
+}
+
+}  // extern "C"

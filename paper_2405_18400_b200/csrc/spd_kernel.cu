@@ -1,0 +1,960 @@
+// Persistent decode kernel for Superposed Decoding on sm_100a.
+//
+// One cooperative launch runs n_iters timesteps.  Every block keeps one producer warp and sixteen
+// consumer warps.  The producer thread walks the static list of weight chunks that its block owns
+// (contiguous row ranges of every matrix, in the order the decoder uses them) and streams them
+// into a shared-memory ring with bulk asynchronous copies that signal mbarriers; because weights do
+// not depend on activations it runs ahead across phase boundaries and across timesteps, so HBM
+// stays busy while the consumers exchange activation vectors through L2 at grid barriers.  The
+// consumers split the columns of each row among all threads (the activation slice of a thread stays
+// in registers for a whole phase), reduce with shuffles, and finish rows in per-phase epilogues
+// (rotary embedding + cache append, residual add, SwiGLU, logits + block-level top-k).  Block 0 then
+// runs the method's tail: KeepTopK over the whole vocabulary, the k*k expansion with n-gram hash
+// probes (Eq. 5), the interpolation (Eq. 6/7), the selection of the k best options (Eq. 2) and the
+// new weights gamma (Eq. 4), and forms the next superposed input (Eq. 3).
+//
+// Every wait (mbarrier, grid barrier, table probe) is bounded; a wait that gives up records an
+// error, raises an abort flag that turns all later waits into no-ops, and the kernel runs to its end.
+#include <cuda_runtime.h>
+#include <math_constants.h>
+
+#include "spd_params.h"
+
+namespace spd {
+
+constexpr unsigned long long kWaitNs = 1500ull * 1000ull * 1000ull;  // 1.5 s per wait
+constexpr int kErrTable = -6, kErrTimeout = -7;
+
+// ---------------------------------------------------------------- small PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bulk asynchronous copy global -> shared of `bytes` (multiple of 16, both addresses 16-byte aligned);
+// completion is counted on `bar` in bytes.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ unsigned int ld_acquire(const unsigned int *p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned int ld_relaxed(const unsigned int *p) {
+  unsigned int v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 lds128(const void *p) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_u32(p)));
+  return v;
+}
+
+// ---------------------------------------------------------------- block context
+struct Blk {
+  const KParams *p;
+  uint8_t *ring;
+  float *part;       // [2][kTile][kConsumerWarps]
+  uint64_t *full, *empty;
+  float *red;        // [64] reduction scratch
+  volatile int *dead;
+  volatile int *quit;  // block-uniform copy of *dead, refreshed inside every grid barrier
+  unsigned int bar_target;
+  unsigned int tail_target;
+  // consumer ring cursor
+  uint32_t c_stage, c_phase;
+};
+
+__device__ __forceinline__ void give_up(Blk &b, int code, int info) {
+  State *st = b.p->st;
+  if (atomicCAS(&st->err, 0, code) == 0) st->err_info = info;
+  atomicExch(&st->abort_flag, 1u);
+  *b.dead = 1;
+}
+
+// Bounded wait on an mbarrier phase.  Returns at once when the block is already giving up.
+__device__ __forceinline__ void wait_mbar(Blk &b, uint64_t *bar, uint32_t parity, int info) {
+  if (mbar_try_wait(bar, parity)) return;
+  if (*b.dead) return;
+  unsigned long long t0 = globaltimer();
+  uint32_t n = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++n & 31u) == 0) {
+      if (*b.dead) return;
+      if (ld_relaxed(&b.p->st->abort_flag)) { *b.dead = 1; return; }
+      if (globaltimer() - t0 > kWaitNs) { give_up(b, kErrTimeout, info); return; }
+    }
+  }
+}
+
+// Grid-wide barrier for the consumer threads of all blocks (all blocks are co-resident: cooperative launch).
+// Returns true, to every consumer thread of the block alike, once the block is giving up.
+__device__ __forceinline__ bool grid_barrier(Blk &b) {
+  named_sync(1, kConsumerThreads);
+  if (threadIdx.x == 0) {
+    b.bar_target += gridDim.x;
+    if (!*b.dead) {
+      unsigned int *bar = &b.p->st->bar;
+      __threadfence();
+      atomicAdd(bar, 1u);
+      unsigned long long t0 = globaltimer();
+      uint32_t n = 0;
+      while ((int)(ld_acquire(bar) - b.bar_target) < 0) {
+        if ((++n & 63u) == 0) {
+          if (ld_relaxed(&b.p->st->abort_flag)) { *b.dead = 1; break; }
+          if (globaltimer() - t0 > kWaitNs) { give_up(b, kErrTimeout, 100); break; }
+        }
+      }
+    }
+    *b.quit = *b.dead;
+  }
+  named_sync(1, kConsumerThreads);
+  return *b.quit != 0;
+}
+
+__device__ __forceinline__ void cta_rows(int R, int gran, int &r0, int &r1) {
+  long long U = R / gran;
+  r0 = (int)(U * blockIdx.x / gridDim.x) * gran;
+  r1 = (int)(U * (blockIdx.x + 1) / gridDim.x) * gran;
+}
+
+__device__ __forceinline__ int rows_per_chunk(const KParams &p, int C) {
+  int rpc = p.stage_bytes / (C * 2);
+  return rpc > kMaxRowsPerChunk ? kMaxRowsPerChunk : rpc;
+}
+
+// ---------------------------------------------------------------- producer
+struct Producer {
+  uint32_t stage, phase;
+  uint32_t issued;  // chunks issued so far (saturating at n_stages for the drain)
+};
+
+__device__ __forceinline__ void produce_matrix(Blk &b, Producer &pr, const __nv_bfloat16 *W, int R, int C, int gran) {
+  const KParams &p = *b.p;
+  int r0, r1;
+  cta_rows(R, gran, r0, r1);
+  const int rpc = rows_per_chunk(p, C);
+  const uint32_t rowbytes = (uint32_t)C * 2u;
+  for (int t0 = r0; t0 < r1; t0 += kTile) {
+    const int t1 = min(t0 + kTile, r1);
+    for (int r = t0; r < t1; r += rpc) {
+      const int n = min(rpc, t1 - r);
+      wait_mbar(b, &b.empty[pr.stage], pr.phase ^ 1u, 200);
+      if (*b.dead) return;
+      const uint32_t bytes = (uint32_t)n * rowbytes;
+      mbar_expect_tx(&b.full[pr.stage], bytes);
+      bulk_load(b.ring + (size_t)pr.stage * p.stage_bytes, (const uint8_t *)W + (size_t)r * rowbytes, bytes,
+                &b.full[pr.stage]);
+      if (pr.issued < (uint32_t)p.n_stages) ++pr.issued;
+      if (++pr.stage == (uint32_t)p.n_stages) { pr.stage = 0; pr.phase ^= 1u; }
+    }
+  }
+}
+
+__device__ void producer_main(Blk &b) {
+  const KParams &p = *b.p;
+  Producer pr{0u, 0u, 0u};
+  for (int it = 0; it < p.n_iters && !*b.dead; ++it) {
+    for (int l = 0; l < p.L && !*b.dead; ++l) {
+      const LayerW lw = p.layers[l];
+      produce_matrix(b, pr, lw.wqkv, 3 * p.d, p.d, 2);
+      produce_matrix(b, pr, lw.wo, p.d, p.d, 1);
+      produce_matrix(b, pr, lw.wgate_up, 2 * p.f, p.d, 2);
+      produce_matrix(b, pr, lw.wdown, p.d, p.f, 1);
+    }
+    if (p.mode == kModeDecode || it == p.n_iters - 1) produce_matrix(b, pr, p.lm_head, p.V, p.d, 1);
+  }
+  if (*b.dead) {
+    // Giving up: nothing more is issued; wait (bounded) until every copy already issued has landed,
+    // so that no copy writes into shared memory after the block has gone.
+    uint32_t s = pr.stage, ph = pr.phase;
+    for (uint32_t i = 0; i < pr.issued; ++i) {
+      if (s == 0) { s = (uint32_t)p.n_stages; ph ^= 1u; }
+      --s;
+      unsigned long long t0 = globaltimer();
+      while (!mbar_try_wait(&b.full[s], ph) && globaltimer() - t0 < kWaitNs) {}
+    }
+  }
+}
+
+// ---------------------------------------------------------------- consumer: row dot products
+__device__ __forceinline__ float dot8(const uint4 w, const float (&x)[8], float acc) {
+  acc = fmaf(__uint_as_float(w.x << 16), x[0], acc);
+  acc = fmaf(__uint_as_float(w.x & 0xffff0000u), x[1], acc);
+  acc = fmaf(__uint_as_float(w.y << 16), x[2], acc);
+  acc = fmaf(__uint_as_float(w.y & 0xffff0000u), x[3], acc);
+  acc = fmaf(__uint_as_float(w.z << 16), x[4], acc);
+  acc = fmaf(__uint_as_float(w.z & 0xffff0000u), x[5], acc);
+  acc = fmaf(__uint_as_float(w.w << 16), x[6], acc);
+  acc = fmaf(__uint_as_float(w.w & 0xffff0000u), x[7], acc);
+  return acc;
+}
+
+// Sums NR per-lane accumulators over the warp with a folding butterfly.  Afterwards lane
+// r * (32 / NR) holds the total of accumulator r.
+template <int NR>
+__device__ __forceinline__ float warp_fold(float (&a)[NR], int lane) {
+  if constexpr (NR == 8) {
+    float b4[4];
+    const bool up = lane & 16;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float send = up ? a[i] : a[i + 4];
+      const float keep = up ? a[i + 4] : a[i];
+      b4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+    float b2[2];
+    const bool up2 = lane & 8;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float send = up2 ? b4[i] : b4[i + 2];
+      const float keep = up2 ? b4[i + 2] : b4[i];
+      b2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+    const bool up3 = lane & 4;
+    float v = (up3 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up3 ? b2[0] : b2[1], 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
+  } else if constexpr (NR == 4) {
+    float b2[2];
+    const bool up = lane & 16;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float send = up ? a[i] : a[i + 2];
+      const float keep = up ? a[i + 2] : a[i];
+      b2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+    const bool up2 = lane & 8;
+    float v = (up2 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up2 ? b2[0] : b2[1], 8);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
+  } else if constexpr (NR == 2) {
+    const bool up = lane & 16;
+    float v = (up ? a[1] : a[0]) + __shfl_xor_sync(0xffffffffu, up ? a[0] : a[1], 16);
+    v += __shfl_xor_sync(0xffffffffu, v, 8);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
+  } else {
+    float v = a[0];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+  }
+}
+
+// One chunk of n (<= NR) rows in a ring stage: every thread multiplies its column vectors, the warp
+// folds, and the warp's partial of row j goes to part[(trow + j) * warps + warp].
+template <int NR>
+__device__ __forceinline__ void consume_chunk(const uint8_t *stage, int n, int rowbytes, int nv,
+                                              const float (&xr)[kMaxVec][8], float *part_rows, int warp, int lane) {
+  float acc[NR];
+#pragma unroll
+  for (int r = 0; r < NR; ++r) acc[r] = 0.f;
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) {
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {
+        if (r < n) {
+          const uint4 w = lds128(stage + (size_t)r * rowbytes + (size_t)v * 16);
+          acc[r] = dot8(w, xr[i], acc[r]);
+        }
+      }
+    }
+  }
+  const float v = warp_fold<NR>(acc, lane);
+  constexpr int kStride = 32 / NR;
+  const int j = lane / kStride;
+  if ((lane % kStride) == 0 && j < n) part_rows[j * kConsumerWarps + warp] = v;
+}
+
+enum Epi { kEpiQKV = 0, kEpiAddH = 1, kEpiSwiGLU = 2, kEpiLogits = 3 };
+
+struct EpiArgs {
+  int layer, pos, which;  // which: 0 = after attention, 1 = after FFN (trace slot)
+};
+
+__device__ __forceinline__ float part_sum(const float *row) {
+  const float4 *q = reinterpret_cast<const float4 *>(row);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < kConsumerWarps / 4; ++i) {
+    const float4 a = q[i];
+    s += a.x;
+    s += a.y;
+    s += a.z;
+    s += a.w;
+  }
+  return s;
+}
+
+__device__ __forceinline__ void store_kv(const KParams &p, void *cache, size_t idx, float v) {
+  if (p.kv_bf16) reinterpret_cast<__nv_bfloat16 *>(cache)[idx] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float *>(cache)[idx] = v;
+}
+
+// Finishes rows [t0, t1) of the current matrix from the warps' partial sums.
+__device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, const float *part, int t0, int t1) {
+  const KParams &p = *b.p;
+  const int tid = threadIdx.x;
+  const int rows = t1 - t0;
+  if (kind == kEpiQKV) {
+    // rows come in pairs (2i, 2i+1) of one head: rotate q and k, append k and v to the cache
+    if (tid * 2 < rows) {
+      const int r = t0 + tid * 2;
+      float a = part_sum(part + (size_t)(tid * 2) * kConsumerWarps);
+      float c = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps);
+      const int sec = r / p.d, col = r - sec * p.d;
+      if (sec < 2) {
+        const float2 cs = p.rope[(size_t)ea.pos * (p.hd / 2) + (col % p.hd) / 2];
+        const float ra = a * cs.x - c * cs.y, rc = a * cs.y + c * cs.x;
+        a = ra;
+        c = rc;
+      }
+      const size_t kv = ((size_t)ea.layer * p.max_pos + ea.pos) * p.d + col;
+      if (sec == 0) {
+        p.q[col] = a;
+        p.q[col + 1] = c;
+      } else if (sec == 1) {
+        store_kv(p, p.kcache, kv, a);
+        store_kv(p, p.kcache, kv + 1, c);
+      } else {
+        store_kv(p, p.vcache, kv, a);
+        store_kv(p, p.vcache, kv + 1, c);
+      }
+    }
+  } else if (kind == kEpiAddH) {
+    if (tid < rows) {
+      const int r = t0 + tid;
+      const float y = __ldcg(p.h + r) + part_sum(part + (size_t)tid * kConsumerWarps);
+      p.h[r] = y;
+      if (p.trace) p.trace[((size_t)ea.layer * 2 + ea.which) * p.d + r] = y;
+    }
+  } else if (kind == kEpiSwiGLU) {
+    if (tid * 2 < rows) {
+      const float g = part_sum(part + (size_t)(tid * 2) * kConsumerWarps);
+      const float up = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps);
+      p.u[(t0 >> 1) + tid] = g / (1.f + __expf(-g)) * up;
+    }
+  } else {
+    if (tid < rows) p.logits[t0 + tid] = part_sum(part + (size_t)tid * kConsumerWarps);
+  }
+}
+
+// Streams this block's rows of one matrix through the ring against the register-resident x.
+__device__ __forceinline__ void consume_matrix(Blk &b, int R, int C, int gran, const float (&xr)[kMaxVec][8], int kind,
+                                               const EpiArgs &ea) {
+  const KParams &p = *b.p;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int r0, r1;
+  cta_rows(R, gran, r0, r1);
+  const int rpc = rows_per_chunk(p, C);
+  const int rowbytes = C * 2, nv = C / 8;
+  int buf = 0;
+  for (int t0 = r0; t0 < r1; t0 += kTile) {
+    const int t1 = min(t0 + kTile, r1);
+    float *part = b.part + (size_t)buf * kTile * kConsumerWarps;
+    for (int r = t0; r < t1; r += rpc) {
+      const int n = min(rpc, t1 - r);
+      wait_mbar(b, &b.full[b.c_stage], b.c_phase, 300);
+      const uint8_t *stage = b.ring + (size_t)b.c_stage * p.stage_bytes;
+      float *prow = part + (size_t)(r - t0) * kConsumerWarps;
+      if (n > 4) consume_chunk<8>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      else if (n > 2) consume_chunk<4>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      else if (n > 1) consume_chunk<2>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      else consume_chunk<1>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&b.empty[b.c_stage]);
+      if (++b.c_stage == (uint32_t)p.n_stages) { b.c_stage = 0; b.c_phase ^= 1u; }
+    }
+    named_sync(1, kConsumerThreads);
+    epilogue(b, kind, ea, part, t0, t1);
+    buf ^= 1;
+  }
+}
+
+// ---------------------------------------------------------------- consumer: activation prologues
+__device__ __forceinline__ float block_sum(Blk &b, float v) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  named_sync(1, kConsumerThreads);  // red[] free again
+  if (lane == 0) b.red[warp] = v;
+  named_sync(1, kConsumerThreads);
+  float s = 0.f;
+#pragma unroll
+  for (int w = 0; w < kConsumerWarps; ++w) s += b.red[w];
+  return s;
+}
+
+__device__ __forceinline__ void load8(const float *src, float (&x)[8]) {
+  const float4 a = __ldcg(reinterpret_cast<const float4 *>(src));
+  const float4 c = __ldcg(reinterpret_cast<const float4 *>(src) + 1);
+  x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+  x[4] = c.x; x[5] = c.y; x[6] = c.z; x[7] = c.w;
+}
+
+// x = RMSNorm(h) * gain, each thread keeping its own column vectors
+__device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const __nv_bfloat16 *gain, int C,
+                                              float (&xr)[kMaxVec][8]) {
+  const int nv = C / 8;
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) {
+      load8(h + (size_t)v * 8, xr[i]);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
+    }
+  }
+  ss = block_sum(b, ss);
+  const float rs = rsqrtf(ss / (float)C + b.p->eps);
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) {
+      const uint4 g = *reinterpret_cast<const uint4 *>(gain + (size_t)v * 8);
+      const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        xr[i][2 * e] = xr[i][2 * e] * rs * __uint_as_float(gw[e] << 16);
+        xr[i][2 * e + 1] = xr[i][2 * e + 1] * rs * __uint_as_float(gw[e] & 0xffff0000u);
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void prologue_plain(const float *src, int C, float (&xr)[kMaxVec][8]) {
+  const int nv = C / 8;
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) load8(src + (size_t)v * 8, xr[i]);
+  }
+}
+
+__device__ __forceinline__ int attn_splits(const KParams &p, int T) {
+  int ms = (int)gridDim.x / p.H;
+  ms = ms < 1 ? 1 : (ms > kMaxSplit ? kMaxSplit : ms);
+  int ns = (T + 63) / 64;
+  return ns < 1 ? 1 : (ns > ms ? ms : ns);
+}
+
+// x = attention output: merges the per-split partial sums of each head
+__device__ __forceinline__ void prologue_attn(const KParams &p, int T, float (&xr)[kMaxVec][8]) {
+  const int nv = p.d / 8, ns = attn_splits(p, T);
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) {
+      const int col = v * 8, head = col / p.hd, c = col - head * p.hd;
+      float M = -CUDART_INF_F;
+      for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&p.oml[head * ns + s]).x);
+      float den = 0.f, acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      for (int s = 0; s < ns; ++s) {
+        const float2 ml = __ldcg(&p.oml[head * ns + s]);
+        const float w = __expf(ml.x - M);
+        den = fmaf(ml.y, w, den);
+        float o[8];
+        load8(p.opart + (size_t)(head * ns + s) * p.hd + c, o);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(o[e], w, acc[e]);
+      }
+      const float inv = 1.f / den;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xr[i][e] = acc[e] * inv;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- attention over the shared cache
+__device__ __forceinline__ float load_kv(const KParams &p, const void *cache, size_t idx) {
+  if (p.kv_bf16) {
+    const unsigned short raw = __ldcg(reinterpret_cast<const unsigned short *>(cache) + idx);
+    return __uint_as_float((uint32_t)raw << 16);
+  }
+  return __ldcg(reinterpret_cast<const float *>(cache) + idx);
+}
+
+__device__ void attention_phase(Blk &b, int layer, int pos) {
+  const KParams &p = *b.p;
+  const int T = pos + 1, ns = attn_splits(p, T), items = p.H * ns;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int epl = p.hd / 32;  // elements per lane, <= 8
+  const float scale = 1.f / sqrtf((float)p.hd);
+  float *s_acc = b.part;                           // [warps][hd]
+  float *s_m = b.part + kConsumerWarps * 256;      // [warps]
+  float *s_l = s_m + kConsumerWarps;               // [warps]
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int head = item / ns, sp = item - head * ns;
+    const int t0 = (int)((long long)T * sp / ns), t1 = (int)((long long)T * (sp + 1) / ns);
+    float q[8], acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      q[e] = e < epl ? __ldcg(p.q + head * p.hd + lane * epl + e) : 0.f;
+      acc[e] = 0.f;
+    }
+    float m = -CUDART_INF_F, l = 0.f;
+    for (int t = t0 + warp; t < t1; t += kConsumerWarps) {
+      const size_t base = ((size_t)layer * p.max_pos + t) * p.d + head * p.hd + lane * epl;
+      float dot = 0.f, vv[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        if (e < epl) {
+          dot = fmaf(q[e], load_kv(p, p.kcache, base + e), dot);
+          vv[e] = load_kv(p, p.vcache, base + e);
+        } else {
+          vv[e] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      const float s = dot * scale;
+      const float mn = fmaxf(m, s);
+      const float c = __expf(m - mn), pw = __expf(s - mn);
+      l = l * c + pw;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = acc[e] * c + pw * vv[e];
+      m = mn;
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      if (e < epl) s_acc[warp * 256 + lane * epl + e] = acc[e];
+    if (lane == 0) {
+      s_m[warp] = m;
+      s_l[warp] = l;
+    }
+    named_sync(1, kConsumerThreads);
+    if ((int)threadIdx.x < p.hd) {
+      float M = -CUDART_INF_F;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, s_m[w]);
+      float L = 0.f, A = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) {
+        const float wgt = s_m[w] == -CUDART_INF_F ? 0.f : __expf(s_m[w] - M);
+        L = fmaf(s_l[w], wgt, L);
+        A = fmaf(s_acc[w * 256 + threadIdx.x], wgt, A);
+      }
+      p.opart[(size_t)item * p.hd + threadIdx.x] = A;
+      if (threadIdx.x == 0) p.oml[item] = make_float2(M, L);
+    }
+    named_sync(1, kConsumerThreads);
+  }
+}
+
+// ---------------------------------------------------------------- LM head: block-level top-k and softmax statistics
+// Ranking order everywhere: larger value first, then smaller index.
+__device__ __forceinline__ bool ranks_before(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+
+__device__ __forceinline__ void warp_best(float &v, int &i) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+    if (oi >= 0 && (i < 0 || ranks_before(ov, oi, v, i))) { v = ov; i = oi; }
+  }
+}
+
+// Warp 0 of each block: the k best logits among rows [r0, r1) and (max, sum exp) of z / tau over them.
+__device__ void block_topk(const KParams &p, int r0, int r1) {
+  const int lane = threadIdx.x & 31;
+  float pv = 0.f;
+  int pi = -1;
+  float mx = -CUDART_INF_F;
+  for (int j = 0; j < p.k; ++j) {
+    float bv = 0.f;
+    int bi = -1;
+    for (int r = r0 + lane; r < r1; r += 32) {
+      const float z = p.logits[r];
+      if (j > 0 && !ranks_before(pv, pi, z, r)) continue;  // already taken (or is the previous winner)
+      if (bi < 0 || ranks_before(z, r, bv, bi)) { bv = z; bi = r; }
+    }
+    warp_best(bv, bi);
+    if (lane == 0) {
+      p.pk_val[(size_t)blockIdx.x * p.k + j] = bi >= 0 ? bv : -CUDART_INF_F;
+      p.pk_id[(size_t)blockIdx.x * p.k + j] = bi;
+    }
+    pv = bv;
+    pi = bi;
+    if (j == 0) mx = bi >= 0 ? bv * p.inv_tau : -CUDART_INF_F;
+    if (bi < 0) {  // fewer rows than k: the rest stay empty
+      for (int jj = j + 1; jj < p.k; ++jj)
+        if (lane == 0) {
+          p.pk_val[(size_t)blockIdx.x * p.k + jj] = -CUDART_INF_F;
+          p.pk_id[(size_t)blockIdx.x * p.k + jj] = -1;
+        }
+      break;
+    }
+  }
+  float s = 0.f;
+  for (int r = r0 + lane; r < r1; r += 32) s += __expf(p.logits[r] * p.inv_tau - mx);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) p.pk_ms[blockIdx.x] = make_float2(mx, s);
+}
+
+// ---------------------------------------------------------------- the method's tail (block 0)
+__device__ __forceinline__ int probe(Blk &b, const SpdSlot *tab, uint64_t mask, uint32_t w0, uint32_t w1, uint32_t w2) {
+  uint64_t idx = spd_key_hash(w0, w1, w2) & mask;
+  const uint64_t limit = mask + 1 < 16384 ? mask + 1 : 16384;
+  for (uint64_t i = 0; i < limit; ++i) {
+    const uint4 s = __ldg(reinterpret_cast<const uint4 *>(tab + idx));
+    if (s.w == 0u) return 0;
+    if (s.x == w0 && s.y == w1 && s.z == w2) return (int)s.w;
+    idx = (idx + 1) & mask;
+  }
+  if (mask + 1 > limit) give_up(b, kErrTable, 400);
+  return 0;
+}
+
+// KeepTopK over the whole vocabulary from the blocks' partial lists (Algorithm 1), with
+// log-probabilities under temperature tau.  Warp 0.
+__device__ void tail_keep_topk(const KParams &p) {
+  const int lane = threadIdx.x & 31;
+  State *st = p.st;
+  const int ncand = (int)gridDim.x * p.k;
+  float M = -CUDART_INF_F;
+  for (int g = lane; g < (int)gridDim.x; g += 32) M = fmaxf(M, __ldcg(&p.pk_ms[g]).x);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  float S = 0.f;
+  for (int g = lane; g < (int)gridDim.x; g += 32) {
+    const float2 ms = __ldcg(&p.pk_ms[g]);
+    if (ms.x > -CUDART_INF_F) S = fmaf(ms.y, __expf(ms.x - M), S);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
+  const float lse = M + __logf(S);
+  float pv = 0.f;
+  int pi = -1;
+  for (int j = 0; j < p.k; ++j) {
+    float bv = 0.f;
+    int bi = -1;
+    for (int c = lane; c < ncand; c += 32) {
+      const int id = __ldcg(&p.pk_id[c]);
+      if (id < 0) continue;
+      const float z = __ldcg(&p.pk_val[c]);
+      if (j > 0 && !ranks_before(pv, pi, z, id)) continue;
+      if (bi < 0 || ranks_before(z, id, bv, bi)) { bv = z; bi = id; }
+    }
+    warp_best(bv, bi);
+    if (lane == 0) {
+      st->cand_tok[j] = bi;
+      st->cand_lp[j] = bv * p.inv_tau - lse;
+    }
+    pv = bv;
+    pi = bi;
+  }
+  __syncwarp();
+}
+
+// Scores the k*k options, keeps the k best, updates the draft state.  `first` = first timestep: draft i
+// simply takes kept token i (Eq. 1).  All consumer threads of block 0.
+__device__ void tail_score_select(Blk &b, bool first, int step) {
+  const KParams &p = *b.p;
+  State *st = p.st;
+  const int tid = threadIdx.x, k = p.k, nt = p.n_tables;
+  int *s_cnt = reinterpret_cast<int *>(b.part);           // [k*k][8]
+  int *s_tot = s_cnt + kMaxK * kMaxK * kMaxTables;         // [k][8]
+  float *s_png = reinterpret_cast<float *>(s_tot + kMaxK * kMaxTables);  // [k*k]
+  float *s_score = s_png + kMaxK * kMaxK;                  // [k*k]
+  named_sync(1, kConsumerThreads);
+  if (first) {
+    if (tid < k) {
+      const int tok = st->cand_tok[tid];
+      st->logP_in[tid] = 0.f;
+      int w[kWin];
+#pragma unroll
+      for (int j = 0; j < kWin; ++j) w[j] = st->win[tid][j];
+#pragma unroll
+      for (int j = 0; j < kWin; ++j) st->win_in[tid][j] = w[j];
+#pragma unroll
+      for (int j = 0; j + 1 < kWin; ++j) st->win[tid][j] = w[j + 1];
+      st->win[tid][kWin - 1] = tok;
+      st->logP[tid] = st->cand_lp[tid];
+      st->sel[tid] = tid;
+      p.hist_tok[(size_t)step * k + tid] = tok;
+      p.hist_par[(size_t)step * k + tid] = tid;
+    }
+  } else {
+    // Eq. 5 lookups: one thread per (draft, token, table) count and per (draft, table) context total
+    const int n_cnt = k * k * nt, n_all = n_cnt + k * nt;
+    const int wl = st->win_len;
+    for (int qi = tid; qi < n_all; qi += kConsumerThreads) {
+      int i, j, ti;
+      if (qi < n_cnt) {
+        i = qi / (k * nt);
+        j = (qi / nt) % k;
+        ti = qi % nt;
+      } else {
+        const int r = qi - n_cnt;
+        i = r / nt;
+        j = -1;
+        ti = r % nt;
+      }
+      const TableDev &tb = p.tab[ti];
+      int res = -1;
+      if (tb.n >= p.n_min && tb.n <= p.n_max && wl >= tb.n - 1) {
+        int32_t key[6];
+#pragma unroll
+        for (int e = 0; e < 6; ++e) key[e] = 0;
+        for (int e = 0; e < tb.n - 1; ++e) key[e] = st->win[i][kWin - (tb.n - 1) + e];
+        int len = tb.n - 1;
+        if (j >= 0) key[len++] = st->cand_tok[j];
+        uint32_t w0, w1, w2;
+        spd_pack_key(key, len, w0, w1, w2);
+        res = j >= 0 ? probe(b, tb.ngram, tb.ngram_mask, w0, w1, w2) : probe(b, tb.ctx, tb.ctx_mask, w0, w1, w2);
+      }
+      if (j >= 0) s_cnt[(i * k + j) * kMaxTables + ti] = res;
+      else s_tot[i * kMaxTables + ti] = res;
+    }
+    named_sync(1, kConsumerThreads);
+    if (tid < k * k) {
+      const int i = tid / k;
+      float png = 0.f;
+      for (int ti = 0; ti < nt; ++ti) {
+        const int c = s_cnt[tid * kMaxTables + ti], t = s_tot[i * kMaxTables + ti];
+        st->cnt[tid][ti] = c;
+        if (tid % k == 0) st->tot[i][ti] = t;
+        if (t > 0) png = fmaf(p.lambda[p.tab[ti].n - 2], (float)c / (float)t, png);
+      }
+      s_png[tid] = png;
+      st->png[tid] = png;
+    }
+    named_sync(1, kConsumerThreads);
+    if (tid < k * k) {
+      const int i = tid / k, j = tid - i * k;
+      bool overlap = false;
+      for (int jj = 0; jj < k; ++jj) overlap |= s_png[i * k + jj] > 0.f;
+      const float base = st->logP[i] + (1.f - p.alpha) * st->cand_lp[j];
+      float sc;
+      if (!overlap) sc = base + p.log_delta;                                   // Eq. 7
+      else if (s_png[tid] > 0.f) sc = base + p.alpha * logf(s_png[tid]);       // Eq. 6
+      else sc = -CUDART_INF_F;                                                 // token absent from the n-gram distribution
+      s_score[tid] = sc;
+      st->score[tid] = sc;
+    }
+    named_sync(1, kConsumerThreads);
+    if (tid < 32) {
+      // the k best options, best first (Eq. 2); then the state moves to the new drafts
+      const int lane = tid;
+      float pv = 0.f;
+      int pi = -1;
+      int my_sel = -1;
+      float my_score = 0.f;
+      for (int r = 0; r < k; ++r) {
+        float bv = 0.f;
+        int bi = -1;
+        for (int c = lane; c < k * k; c += 32) {
+          const float z = s_score[c];
+          if (r > 0 && !ranks_before(pv, pi, z, c)) continue;
+          if (bi < 0 || ranks_before(z, c, bv, bi)) { bv = z; bi = c; }
+        }
+        warp_best(bv, bi);
+        if (lane == r) { my_sel = bi; my_score = bv; }
+        pv = bv;
+        pi = bi;
+      }
+      int w[kWin];
+      float old_lp = 0.f;
+      if (lane < k) {
+        old_lp = st->logP[lane];
+        const int par = my_sel / k;
+#pragma unroll
+        for (int j = 0; j < kWin; ++j) w[j] = st->win[par][j];
+      }
+      int own[kWin];
+      if (lane < k) {
+#pragma unroll
+        for (int j = 0; j < kWin; ++j) own[j] = st->win[lane][j];
+      }
+      __syncwarp();
+      if (lane < k) {
+        const int par = my_sel / k, tok = st->cand_tok[my_sel - par * k];
+        st->logP_in[lane] = old_lp;
+#pragma unroll
+        for (int j = 0; j < kWin; ++j) st->win_in[lane][j] = own[j];
+#pragma unroll
+        for (int j = 0; j + 1 < kWin; ++j) st->win[lane][j] = w[j + 1];
+        st->win[lane][kWin - 1] = tok;
+        st->logP[lane] = my_score;
+        st->sel[lane] = my_sel;
+        p.hist_tok[(size_t)step * k + lane] = tok;
+        p.hist_par[(size_t)step * k + lane] = par;
+      }
+    }
+  }
+  named_sync(1, kConsumerThreads);
+  if (tid < 32) {
+    // gamma_i = p_i / sum_j p_j (Eq. 4), from log-probabilities
+    const int lane = tid;
+    const float lp = lane < k ? st->logP[lane] : -CUDART_INF_F;
+    float mx = lp;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const float e = lane < k ? expf(lp - mx) : 0.f;
+    float den = e;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    if (lane < k) st->gamma[lane] = e / den;
+    if (lane == 0) {
+      st->win_len = min(st->win_len + 1, kWin);
+      st->n_gen += 1;
+    }
+  }
+  named_sync(1, kConsumerThreads);
+}
+
+// Next LM input (block 0): the token embedding in prefill, the superposed embedding of Eq. 3 in decode.
+__device__ void embed_input(const KParams &p, int it) {
+  const State *st = p.st;
+  if (p.mode == kModePrefill) {
+    const int tok = p.prefix[it];
+    for (int c = threadIdx.x; c < p.d; c += kConsumerThreads) p.h[c] = __bfloat162float(p.tok_emb[(size_t)tok * p.d + c]);
+  } else {
+    for (int c = threadIdx.x; c < p.d; c += kConsumerThreads) {
+      float acc = 0.f;
+      for (int i = 0; i < p.k; ++i)
+        acc = fmaf(st->gamma[i], __bfloat162float(p.tok_emb[(size_t)st->win[i][kWin - 1] * p.d + c]), acc);
+      p.h[c] = acc;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- consumer main loop
+__device__ void consumer_main(Blk &b) {
+  const KParams &p = *b.p;
+  float xr[kMaxVec][8];
+  for (int it = 0; it < p.n_iters; ++it) {
+    const int pos = p.pos0 + it;
+    if (blockIdx.x == 0) embed_input(p, it);
+    if (grid_barrier(b)) return;
+    for (int l = 0; l < p.L; ++l) {
+      const LayerW lw = p.layers[l];
+      EpiArgs ea{l, pos, 0};
+      prologue_norm(b, p.h, lw.attn_norm, p.d, xr);
+      consume_matrix(b, 3 * p.d, p.d, 2, xr, kEpiQKV, ea);
+      if (grid_barrier(b)) return;
+      attention_phase(b, l, pos);
+      if (grid_barrier(b)) return;
+      prologue_attn(p, pos + 1, xr);
+      consume_matrix(b, p.d, p.d, 1, xr, kEpiAddH, ea);
+      if (grid_barrier(b)) return;
+      prologue_norm(b, p.h, lw.ffn_norm, p.d, xr);
+      consume_matrix(b, 2 * p.f, p.d, 2, xr, kEpiSwiGLU, ea);
+      if (grid_barrier(b)) return;
+      prologue_plain(p.u, p.f, xr);
+      ea.which = 1;
+      consume_matrix(b, p.d, p.f, 1, xr, kEpiAddH, ea);
+      if (grid_barrier(b)) return;
+    }
+    const bool last = it == p.n_iters - 1;
+    if (p.mode == kModeDecode || last) {
+      EpiArgs ea{0, pos, 0};
+      prologue_norm(b, p.h, p.final_norm, p.d, xr);
+      consume_matrix(b, p.V, p.d, 1, xr, kEpiLogits, ea);
+      named_sync(1, kConsumerThreads);
+      int r0, r1;
+      cta_rows(p.V, 1, r0, r1);
+      if (threadIdx.x < 32) block_topk(p, r0, r1);
+      if (grid_barrier(b)) return;
+      if (blockIdx.x == 0) {
+        if (threadIdx.x < 32) tail_keep_topk(p);
+        const bool first = p.mode == kModePrefill;
+        tail_score_select(b, first, first ? 0 : p.step0 + it);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages];
+  __shared__ float s_red[64];
+  __shared__ int s_dead, s_quit;
+  Blk b;
+  b.p = &p;
+  b.ring = smem;
+  b.part = reinterpret_cast<float *>(smem + (size_t)p.n_stages * p.stage_bytes);
+  b.full = s_full;
+  b.empty = s_empty;
+  b.red = s_red;
+  b.dead = &s_dead;
+  b.quit = &s_quit;
+  b.bar_target = 0;
+  b.tail_target = 0;
+  b.c_stage = 0;
+  b.c_phase = 0;
+  if (threadIdx.x == 0) {
+    s_dead = 0;
+    s_quit = 0;
+    for (int s = 0; s < p.n_stages; ++s) {
+      mbar_init(&s_full[s], 1);
+      mbar_init(&s_empty[s], kConsumerWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (p.mode == kModeScoreOnly) {
+    if (blockIdx.x == 0 && threadIdx.x < kConsumerThreads) tail_score_select(b, false, p.step0);
+    return;
+  }
+  if (threadIdx.x >= kConsumerThreads) {
+    if (threadIdx.x == kConsumerThreads) producer_main(b);
+  } else {
+    consumer_main(b);
+  }
+  __syncthreads();
+}
+
+}  // namespace spd
+
+// Host-side launcher used by the API file.
+extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size_t dyn_smem, cudaStream_t stream) {
+  void *args[] = {const_cast<spd::KParams *>(p)};
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&spd::spd_decode_kernel), dim3(grid), dim3(spd::kThreads),
+                                     args, dyn_smem, stream);
+}
+
+extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm) {
+  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_decode_kernel),
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void *>(&spd::spd_decode_kernel),
+                                                       spd::kThreads, dyn_smem);
+}

@@ -1,0 +1,85 @@
+// Structures shared by the host API and the decode kernel (device side of the library only).
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "spd_hash.h"
+
+namespace spd {
+
+constexpr int kMaxK = 16;
+constexpr int kMaxTables = 8;
+constexpr int kWin = 8;             // tokens of history kept per draft (n_max - 1 <= 5 are used)
+constexpr int kConsumerWarps = 16;  // warps that multiply; one more warp streams weights
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;
+constexpr int kTile = 128;          // rows between two epilogues
+constexpr int kMaxRowsPerChunk = 8;
+constexpr int kMaxStages = 16;
+constexpr int kMaxVec = 4;          // 16-byte column vectors per thread: columns <= 4 * 512 * 8
+constexpr int kMaxSplit = 8;        // attention splits per head
+
+enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2 };
+
+struct LayerW {
+  const __nv_bfloat16 *attn_norm, *wqkv, *wo, *ffn_norm, *wgate_up, *wdown;
+};
+
+struct TableDev {
+  const SpdSlot *ngram, *ctx;
+  uint64_t ngram_mask, ctx_mask;
+  int32_t n, pad;
+};
+
+// Draft state and the last step's intermediates, in device memory.
+struct State {
+  unsigned int bar;         // grid barrier counter (zeroed by the host before every launch)
+  unsigned int tail_bar;    // arrivals of the LM-head phase
+  unsigned int abort_flag;  // set by any thread that gave up a wait
+  int32_t err, err_info;
+  int32_t win_len;          // valid tokens in each history window
+  int32_t n_gen;            // tokens generated per draft so far
+  int32_t win[kMaxK][kWin]; // right-aligned: win[i][kWin-1] is draft i's last token
+  float logP[kMaxK], gamma[kMaxK];
+  // intermediates of the last step
+  int32_t cand_tok[kMaxK];
+  float cand_lp[kMaxK];
+  float logP_in[kMaxK];
+  int32_t win_in[kMaxK][kWin];
+  float score[kMaxK * kMaxK], png[kMaxK * kMaxK];
+  int32_t cnt[kMaxK * kMaxK][kMaxTables];
+  int32_t tot[kMaxK][kMaxTables];
+  int32_t sel[kMaxK];
+};
+
+struct KParams {
+  // model
+  int32_t L, d, H, hd, f, V, max_pos;
+  float eps;
+  int32_t kv_bf16;
+  const LayerW *layers;
+  const __nv_bfloat16 *tok_emb, *final_norm, *lm_head;
+  // method
+  int32_t k, n_min, n_max, n_tables;
+  float lambda[8];
+  float alpha, inv_tau, log_delta;
+  TableDev tab[kMaxTables];
+  // workspace
+  void *kcache, *vcache;     // [L][max_pos][d] float or bf16
+  const float2 *rope;        // [max_pos][hd/2] (cos, sin)
+  float *h, *q, *u, *logits; // [d], [d], [f], [V]
+  float *opart;              // [H * kMaxSplit][hd] unnormalised attention partials
+  float2 *oml;               // [H * kMaxSplit] (running max, running sum)
+  float *pk_val;             // [grid][k] per-block top logits
+  int32_t *pk_id;            // [grid][k]
+  float2 *pk_ms;             // [grid] (max of z/tau, sum of exp(z/tau - max))
+  State *st;
+  int32_t *hist_tok, *hist_par;  // [max_pos][k]
+  const int32_t *prefix;     // [max_pos]
+  float *trace;              // [L][2][d] or null
+  // launch
+  int32_t mode, n_iters, pos0, step0;
+  int32_t stage_bytes, n_stages;
+};
+
+}  // namespace spd

@@ -1,0 +1,104 @@
+"""Helpers shared by the GPU parity tests: build the CUDA context and the oracle on the same seeded
+inputs, and compare one timestep with the margin rule."""
+import math
+
+import numpy as np
+
+import spd_inputs as si
+from oracle import spd_oracle as so
+
+LOGIT_TOL = 2e-2      # max-abs logit tolerance (bf16 weights, fp32 accumulation)
+GAMMA_TOL = 1e-4
+
+
+def make_pair(shape, weights, tables, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype="bf16", device="cuda:0"):
+    import paper_2405_18400_b200 as P
+
+    packed = P.pack_weights(weights, device)
+    dtabs = P.build_ngram_tables(tables, device)
+    ctx = P.SpdContext(shape, packed, dtabs, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype)
+    cfg = so.make_config(shape, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype)
+    orc = so.Oracle(cfg, weights, sorted(tables, key=lambda t: int(t["n"])))
+    return ctx, orc
+
+
+def make_tiny_pair(tiny_inputs, k=None, kv_dtype="bf16", max_pos=None, tables=None, alpha=None, delta=None):
+    wl, weights, tabs, prefix = tiny_inputs
+    return make_pair(wl.shape, weights, tabs if tables is None else tables, wl.k if k is None else k, wl.orders,
+                     wl.lambdas(), wl.alpha if alpha is None else alpha, wl.tau, wl.delta if delta is None else delta,
+                     wl.max_pos if max_pos is None else max_pos, kv_dtype)
+
+
+def top_gap(values, k):
+    """Smallest gap between neighbours among the k+1 largest float32 values (inf if fewer exist)."""
+    v = np.sort(np.asarray(values, dtype=np.float32)[np.isfinite(values)])[::-1][: k + 1].astype(np.float64)
+    return float(np.min(-np.diff(v))) if v.size > 1 else math.inf
+
+
+def compare_first_step(ctx, orc, prefix, stats=None):
+    ids, g = ctx.spd_prefill(prefix)
+    ids_o, g_o = orc.prefill(prefix)
+    z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
+    eps_z = float(np.abs(z - z_o).max())
+    assert eps_z <= LOGIT_TOL, eps_z
+    k = ctx.k
+    assert top_gap(z_o, k) > 2 * eps_z, "fixture has a near-tie among the top logits"
+    assert ids.tolist() == ids_o.tolist()
+    assert np.abs(ctx.spd_debug_read("CAND_LP") - orc.cand_lp()).max() <= 2 * eps_z / orc.cfg.tau + 1e-4
+    assert np.abs(g - g_o).max() <= max(GAMMA_TOL, 4 * eps_z / orc.cfg.tau)
+    if stats is not None:
+        stats.append({"eps_z": eps_z, "dgamma": float(np.abs(g - g_o).max())})
+    return ids, g
+
+
+def compare_step(ctx, orc, stats=None):
+    """One later timestep on both sides.  Exact ids / parents / counts when the oracle's margins exceed
+    twice the measured float error; otherwise the device's choice must be one the oracle rates within
+    that error of its own, and the oracle follows it."""
+    k = ctx.k
+    tau, alpha = orc.cfg.tau, orc.cfg.alpha
+    hist_o = orc.drafts()
+    logP_o = orc.logP()
+    ids, par, g = ctx.spd_step()
+    orc.step_forward()
+    z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
+    eps_z = float(np.abs(z - z_o).max())
+    assert eps_z <= LOGIT_TOL, eps_z
+    assert top_gap(z_o, k) > 2 * eps_z, "fixture has a near-tie among the top logits"
+    cand = ctx.spd_debug_read("CAND_TOK")
+    assert cand.tolist() == orc.cand_tok().tolist()
+    cand_lp = ctx.spd_debug_read("CAND_LP").astype(np.float64)
+    assert np.abs(cand_lp - orc.cand_lp()).max() <= 2 * eps_z / tau + 1e-4
+    # the device scored the same drafts
+    win = ctx.spd_debug_read("HIST_IN")
+    w = min(8, hist_o.shape[1])
+    assert np.array_equal(win[:, 8 - w:], hist_o[:, -w:])
+    logP_in = ctx.spd_debug_read("LOGP_IN").astype(np.float64)
+    sel_o, nl_o, ng_o = orc.step_score()
+    nt = orc.tables.n
+    assert np.array_equal(ctx.spd_debug_read("CNT")[:, :nt], orc.counts())      # integer lookups: always exact
+    assert np.array_equal(ctx.spd_debug_read("TOT")[:, :nt], orc.totals())
+    sc, sc_o = ctx.spd_debug_read("SCORE").astype(np.float64), orc.scores()
+    assert np.array_equal(np.isfinite(sc), np.isfinite(sc_o))
+    fin = np.isfinite(sc_o)
+    eps_s = float(np.abs(sc[fin] - sc_o[fin]).max())
+    assert eps_s <= np.abs(logP_in - logP_o).max() + (1 - alpha) / tau * 2 * eps_z + 1e-4
+    sel = ctx.spd_debug_read("SEL")
+    tie_free = top_gap(sc_o, k) > 2 * eps_s
+    if tie_free:
+        assert sel.tolist() == sel_o.tolist()
+    else:
+        kth = np.sort(sc_o[fin])[::-1][k - 1]
+        assert all(sc_o[q] >= kth - 2 * eps_s for q in sel) and len(set(sel.tolist())) == k
+    assert par.tolist() == (sel // k).tolist() and ids.tolist() == cand[sel % k].tolist()
+    # stage check: the oracle's scoring stage on the device's own inputs reproduces choice and gamma
+    st = so.score_stage(orc.cfg, orc.tables, hist_o[:, -w:], logP_in, cand, cand_lp)
+    if top_gap(st["score"], k) > 1e-4:
+        assert st["sel"].tolist() == sel.tolist()
+        assert np.abs(st["gamma"] - g).max() <= GAMMA_TOL
+        assert np.abs(st["logP"] - ctx.spd_debug_read("LOGP")).max() <= 1e-4 * max(1.0, np.abs(st["logP"]).max())
+    orc.step_commit(sel, sc_o[sel])
+    dg = float(np.abs(orc.gamma() - g).max())
+    if stats is not None:
+        stats.append({"eps_z": eps_z, "eps_s": eps_s, "dgamma": dg, "tie_free": tie_free})
+    return ids, par, g

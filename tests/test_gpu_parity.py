@@ -1,0 +1,233 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element on seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import spd_inputs as si
+from oracle import spd_oracle as so
+from tests.gpu_common import (GAMMA_TOL, LOGIT_TOL, compare_first_step, compare_step, make_pair, make_tiny_pair)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "f32"])
+def test_tiny_workload_stepwise(tiny_inputs, kv_dtype):
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, orc = make_tiny_pair(tiny_inputs, kv_dtype=kv_dtype)
+    stats = []
+    compare_first_step(ctx, orc, prefix, stats)
+    tr, tr_o = ctx.spd_debug_read("TRACE").astype(np.float64), orc.trace()
+    assert np.abs(tr - tr_o).max() < 1e-3
+    for _ in range(wl.gen_tokens - 1):
+        compare_step(ctx, orc, stats)
+        assert np.abs(ctx.spd_debug_read("TRACE").astype(np.float64) - orc.trace()).max() < 1e-3
+    assert max(s["eps_z"] for s in stats) < 2e-4          # far inside the 2e-2 bound when quantisation points agree
+    if max(s["eps_z"] for s in stats) <= 2e-5:
+        assert max(s["dgamma"] for s in stats) <= GAMMA_TOL
+    toks, lp, g = ctx.spd_generate(1, wl.gen_tokens + 1)
+    ids_o, par_o, g_o = orc.step()
+    assert np.array_equal(toks, orc.drafts()[:, len(prefix):])
+    ctx.close()
+
+
+@pytest.mark.parametrize("k", [1, 2, 5, 16])
+def test_draft_counts(tiny_inputs, k):
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, orc = make_tiny_pair(tiny_inputs, k=k)
+    compare_first_step(ctx, orc, prefix)
+    for _ in range(4):
+        ids, par, g = compare_step(ctx, orc)
+        assert abs(float(g.sum()) - 1.0) < 1e-5 and np.all(np.diff(g) <= 0)
+    ctx.close()
+
+
+def test_one_launch_generate_equals_single_steps(tiny_inputs):
+    wl, weights, tables, prefix = tiny_inputs
+    a, orc = make_tiny_pair(tiny_inputs)
+    b, _ = make_tiny_pair(tiny_inputs)
+    a.spd_prefill(prefix)
+    b.spd_prefill(prefix)
+    hist = [[int(t)] for t in a.spd_debug_read("CAND_TOK")]
+    for _ in range(6):
+        ids, par, g = a.spd_step()
+        hist = [hist[int(par[r])] + [int(ids[r])] for r in range(a.k)]
+    toks, lp, g2 = b.spd_generate(6, 7)
+    assert toks.tolist() == hist
+    assert np.array_equal(g, g2) and np.array_equal(lp, a.spd_debug_read("LOGP"))       # bit-identical
+    assert np.array_equal(a.spd_debug_read("LOGITS"), b.spd_debug_read("LOGITS"))
+    assert a.spd_launch_count() == 7 and b.spd_launch_count() == 2
+    # and again from the start on the same context: prefill restarts it
+    b.spd_prefill(prefix)
+    toks2, lp2, g3 = b.spd_generate(6, 7)
+    assert np.array_equal(toks, toks2) and np.array_equal(lp, lp2)
+    a.close(); b.close()
+
+
+def test_long_context_uses_split_attention(tiny_inputs):
+    """A 200-token prefix makes the attention phase split each head's positions over several blocks."""
+    wl, weights, tables, _ = tiny_inputs
+    prefix = si.make_prefix("zipf", 200, wl.shape.vocab, 1.1, seed=7)
+    ctx, orc = make_tiny_pair(tiny_inputs, max_pos=256)
+    compare_first_step(ctx, orc, prefix)
+    for _ in range(3):
+        compare_step(ctx, orc)
+    ctx.close()
+
+
+def test_odd_shape_model():
+    """head_dim 96, d_ffn not a multiple of the thread count, vocabulary not divisible by the grid."""
+    shape = si.ModelShape("odd", 1, 192, 2, 200, 1000)
+    weights = si.make_weights(shape, seed=4)
+    tables = si.make_ngram_tables(shape.vocab, 1.1, 50_000, (2, 3), 5000, seed=8)
+    lam = [0.3, 0.2] + [0.0] * 6
+    ctx, orc = make_pair(shape, weights, tables, 4, (2, 3), lam, 0.4, 0.2, 0.05, 64, "f32")
+    prefix = si.make_prefix("uniform", 9, shape.vocab, seed=9)
+    compare_first_step(ctx, orc, prefix)
+    for _ in range(5):
+        compare_step(ctx, orc)
+    ctx.close()
+
+
+def _hit_case(tables, rng, k, vocab):
+    big = tables[-1]
+    n = int(big["n"])
+    keys = big["keys"].numpy()
+    rows = keys[rng.integers(0, keys.shape[0], size=k)]
+    hist = np.concatenate([rng.integers(0, vocab, size=(k, 8 - (n - 1))), rows[:, : n - 1]], axis=1).astype(np.int32)
+    cand = list(dict.fromkeys(int(rows[i % k, n - 1]) for i in range(max(1, k // 2))))
+    while len(cand) < k:
+        t = int(rng.integers(0, vocab))
+        if t not in cand:
+            cand.append(t)
+    return hist, np.array(cand, np.int32)
+
+
+@pytest.mark.parametrize("k", [2, 3, 5, 8, 16])
+def test_scoring_stage_with_ngram_hits(tiny_inputs, k):
+    """Random-weight models rarely hit the tables, so the hit path is driven directly: histories end
+    in stored contexts and kept tokens include stored continuations (Eq. 5-7, Eq. 2, Eq. 4)."""
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, orc = make_tiny_pair(tiny_inputs, k=k)
+    rng = np.random.default_rng(100 + k)
+    hits = 0
+    for trial in range(12):
+        hist, cand = _hit_case(tables, rng, k, wl.shape.vocab)
+        if trial % 3 == 0:
+            hist[k - 1] = rng.integers(0, wl.shape.vocab, size=8)
+        hist_len = 8 if trial % 4 else 2                       # short histories skip the longer orders
+        hist = np.ascontiguousarray(hist[:, 8 - hist_len:])
+        logP = (-rng.random(k) * 3).astype(np.float32)
+        cand_lp = np.sort((-rng.random(k) * 4).astype(np.float32))[::-1].copy()
+        ctx.spd_debug_score(hist, logP, cand, cand_lp)
+        want = so.score_stage(orc.cfg, orc.tables, hist, logP, cand, cand_lp)
+        assert np.array_equal(ctx.spd_debug_read("CNT")[:, :3], want["cnt"])
+        assert np.array_equal(ctx.spd_debug_read("TOT")[:, :3], want["tot"])
+        hits += int((want["cnt"] > 0).sum())
+        assert np.abs(ctx.spd_debug_read("PNG") - want["png"]).max() < 1e-6
+        sc = ctx.spd_debug_read("SCORE").astype(np.float64)
+        fin = np.isfinite(want["score"])
+        assert np.array_equal(np.isfinite(sc), fin)
+        assert np.abs(sc[fin] - want["score"][fin]).max() < 2e-5
+        srt = np.sort(want["score"][fin])[::-1][: k + 1]
+        if np.min(-np.diff(srt)) > 1e-4:
+            assert ctx.spd_debug_read("SEL").tolist() == want["sel"].tolist()
+            assert np.abs(ctx.spd_debug_read("LOGP") - want["logP"]).max() < 2e-5
+    assert hits > 10
+    ctx.close()
+
+
+def test_every_stored_ngram_is_found_and_absent_ones_miss(tiny_inputs):
+    wl, weights, tables, prefix = tiny_inputs
+    k = 16
+    ctx, orc = make_tiny_pair(tiny_inputs, k=k)
+    rng = np.random.default_rng(77)
+    for ti, t in enumerate(tables):
+        n = int(t["n"])
+        keys = t["keys"].numpy()
+        cnts = t["counts"].numpy()
+        for _ in range(6):
+            idx = rng.integers(0, keys.shape[0], size=k)
+            hist = np.ascontiguousarray(keys[idx, : n - 1]).astype(np.int32)
+            cand = np.array(sorted(set(keys[idx, n - 1].tolist())), np.int32)
+            while cand.size < k:
+                c = int(rng.integers(0, wl.shape.vocab))
+                if c not in cand:
+                    cand = np.append(cand, np.int32(c))
+            ctx.spd_debug_score(hist, np.zeros(k, np.float32), cand, np.zeros(k, np.float32))
+            cnt = ctx.spd_debug_read("CNT").reshape(k, k, 8)
+            want = so.score_stage(orc.cfg, orc.tables, hist, np.zeros(k), cand, np.zeros(k))
+            assert np.array_equal(cnt[:, :, :3].reshape(k * k, 3), want["cnt"])
+            for i in range(k):
+                j = int(np.where(cand == keys[idx[i], n - 1])[0][0])
+                assert cnt[i, j, ti] == cnts[idx[i]]
+    ctx.close()
+
+
+def test_self_generated_corpus_gives_hits_end_to_end(tiny_inputs):
+    """Tables counted over text the model itself produces (greedy continuations of random prefixes)
+    make the n-gram lookups hit during real decoding, so the interpolation path runs end to end."""
+    wl, weights, tables, prefix = tiny_inputs
+    empty = [{"n": n, "keys": np.zeros((0, n), np.int32), "counts": np.zeros(0, np.int64)} for n in wl.orders]
+    cfg1 = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "bf16")
+    stream = []
+    for s in range(6):
+        pf = prefix if s == 0 else si.make_prefix("uniform", 16, wl.shape.vocab, seed=50 + s)
+        o = so.Oracle(cfg1, weights, empty)
+        o.prefill(pf)
+        for _ in range(10):
+            o.step()
+        for row in o.drafts():
+            stream += row.tolist()
+    st = torch.tensor(stream, dtype=torch.int64)
+    own = [si.count_ngrams(st, n) for n in wl.orders]
+    ctx, orc = make_tiny_pair(tiny_inputs, tables=own)
+    compare_first_step(ctx, orc, prefix)
+    hits = 0
+    for _ in range(8):
+        compare_step(ctx, orc)
+        hits += int((ctx.spd_debug_read("CNT")[:, :3] > 0).sum())
+    assert hits > 0
+    ctx.close()
+
+
+def test_call_order_and_range_errors(tiny_inputs):
+    import paper_2405_18400_b200 as P
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, _ = make_tiny_pair(tiny_inputs, max_pos=24)
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_step()
+    assert e.value.status == -2
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_prefill([0, 5000])
+    assert e.value.status == -3
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_prefill(list(range(24)))
+    assert e.value.status == -3
+    ctx.spd_prefill(prefix)                    # 16 positions used, 8 left
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_generate(9, 10)
+    assert e.value.status == -3
+    toks, lp, g = ctx.spd_generate(8, 9)
+    assert toks.shape == (3, 9)
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_step()
+    assert e.value.status == -3
+    ctx.close()
+
+
+def test_ring_settings_do_not_change_results(tiny_inputs):
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, _ = make_tiny_pair(tiny_inputs)
+    ctx.spd_prefill(prefix)
+    base, lp0, _ = ctx.spd_generate(5, 6)
+    z0 = ctx.spd_debug_read("LOGITS")
+    for sb, ns in [(2048, 2), (4096, 16), (65536, 3)]:
+        ctx.spd_set_ring(sb, ns)
+        ctx.spd_prefill(prefix)
+        toks, lp, _ = ctx.spd_generate(5, 6)
+        assert np.array_equal(toks, base)
+        assert np.abs(ctx.spd_debug_read("LOGITS") - z0).max() < 1e-4
+    import paper_2405_18400_b200 as P
+    with pytest.raises(P.SpdError):
+        ctx.spd_set_ring(1024, 4)              # a 688-column row (1376 bytes) does not fit
+    ctx.close()
