@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the Superposed Decoding decode step on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b_k3] [--impl ours|reference]
+
+A "step" is one decode timestep: superposed embedding -> decoder over the shared KV cache -> LM
+head + KeepTopK -> k*k n-gram expansion -> selection and gamma.  The timed region is ONE
+spd_generate_async(K) launch after a prefill and W warm-up steps, timed with CUDA events on the
+launching stream; inputs (13 GB of weights) exceed L2, so nothing is flushed between steps.
+With N > 1 (torchrun) every rank serves its own prefix on its own GPU: replicas, no collective
+on the data path.  Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import spd_inputs as si
+
+METRIC = "k-draft tokens/s"
+UNIT = "tokens/s"
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def step_bytes(wl, k, T):
+    """Algorithmic bytes one decode step must move: every weight once, norm gains, k embedding rows,
+    the KV cache of T positions, one 32-byte sector per table probe."""
+    s = wl.shape
+    kvb = 2 if wl.kv_dtype == "bf16" else 4
+    return (s.step_weight_bytes + 2 * (2 * s.n_layers + 1) * s.d_model + k * s.d_model * 2
+            + s.n_layers * 2 * T * s.d_model * kvb + (k + k * k) * len(wl.orders) * 32)
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            p = [x.strip() for x in ln.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); mx.append(float(p[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def make_inputs(wl, device, rank):
+    t0 = time.time()
+    weights = si.make_weights(wl.shape, seed=0, device=device)
+    log("[bench] weights %.1fs" % (time.time() - t0))
+    t0 = time.time()
+    tables = si.make_ngram_tables(wl.shape.vocab, wl.zipf_s, wl.stream_len, wl.orders, wl.retain, seed=1, device=device)
+    log("[bench] n-gram tables %.1fs (%s entries)" % (time.time() - t0, [int(t["counts"].shape[0]) for t in tables]))
+    prefix = si.make_prefix(wl.prefix_kind, wl.prefix_len, wl.shape.vocab, wl.zipf_s, seed=2, tensor_id=rank)
+    return weights, tables, prefix
+
+
+def run_ours(args, wl):
+    import paper_2405_18400_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    P.load_library()
+    k, K, W = args.k or wl.k, args.steps, args.warmup
+    weights, tables, prefix = make_inputs(wl, dev, rank)
+    host_weights = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        t0 = time.time()
+        host_weights = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in weights.items()}
+        log("[bench] weights to host %.1fs" % (time.time() - t0))
+    t0 = time.time()
+    packed = P.pack_weights(weights, dev, consume=True)
+    del weights
+    dtabs = P.build_ngram_tables(tables, dev)
+    torch.cuda.empty_cache()
+    log("[bench] pack + table build %.1fs" % (time.time() - t0))
+    max_pos = max(wl.max_pos, wl.prefix_len + W + K + 2)
+    ctx = P.SpdContext(wl.shape, packed, dtabs, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, max_pos, wl.kv_dtype)
+    if args.stage_bytes or args.stages:
+        ctx.spd_set_ring(args.stage_bytes, args.stages)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident throughput: one launch of K steps
+    ctx.spd_prefill(prefix)
+    ctx.spd_generate_async(W)
+    ctx.spd_sync()
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = local
+    sampler = ClockSampler(gpu_id)
+    reps = max(1, args.reps)
+    ms_list = []
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = ctx.spd_launch_count()
+    for rep in range(reps):
+        if rep:
+            ctx.spd_prefill(prefix)
+            ctx.spd_generate_async(W)
+            ctx.spd_sync()
+            launches0 = ctx.spd_launch_count()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.spd_generate_async(K)
+        e1.record()
+        ctx.spd_sync()
+        barrier()
+        ms_list.append(e0.elapsed_time(e1))
+    launches = ctx.spd_launch_count() - launches0
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    ms = float(np.median(ms_list))
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    T_mid = wl.prefix_len + W + (K + 1) // 2
+    bytes_step = step_bytes(wl, k, T_mid)
+    peak, peak_kind = measured_peak_gbs()
+    achieved = bytes_step * K / (ms * 1e-3) / 1e9
+    value = world * k * K / (ms * 1e-3)
+
+    # ---- end to end through the C ABI with host buffers: prefill(host ids) + per-step calls returning to the host
+    gen = wl.gen_tokens
+    e2e_t = []
+    for _ in range(2):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ctx.spd_prefill(prefix)
+        for _ in range(gen - 1):
+            ctx.spd_step()
+        e2e_t.append(time.perf_counter() - t0)
+    e2e_s = min(e2e_t)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e = {"value": world * k * gen / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len / gen,
+           "d2h_bytes_per_step": 12.0 * k, "what": "spd_prefill(host ids) + %d spd_step calls returning ids, parents and gamma "
+           "to the host, per request of %d tokens per draft; prefill replays the decode kernels token by token" % (gen - 1, gen),
+           "ms_per_request": e2e_s * 1e3}
+
+    # ---- the same number of drafts from k separate single-draft passes through the same kernels
+    kpass = None
+    if rank == 0 and not args.no_kpass and k > 1:
+        c1 = P.SpdContext(wl.shape, packed, dtabs, 1, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, max_pos, wl.kv_dtype)
+        c1.spd_prefill(prefix)
+        c1.spd_generate_async(W)
+        c1.spd_sync()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        c1.spd_generate_async(K)
+        e1.record()
+        c1.spd_sync()
+        one = e0.elapsed_time(e1)
+        kpass = {"ms_per_step_single_draft": one / K, "ms_per_step_k_passes": k * one / K, "ms_per_step_spd": ms / K,
+                 "saving": k * one / ms, "note": "k sequential batch-1 passes (k=1 contexts, own KV cache) vs one superposed pass"}
+        c1.close()
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "%s: %s-shape decoder, prefix %d, k=%d, bs1, n-gram n=%s, %d entries/order" % (
+            wl.name, wl.shape.name, wl.prefix_len, k, "%d..%d" % (min(wl.orders), max(wl.orders)), wl.retain),
+            "l2": "inputs_exceed_l2", "kv_dtype": wl.kv_dtype, "parallelism": "replicas x%d" % world, "reps": reps},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_decode_kernel"},
+        "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+    }
+    if kpass:
+        out["k_pass"] = kpass
+    ctx.close()
+
+    if rank == 0 and host_weights is not None:
+        out["cpu_baseline"] = cpu_baseline(wl, k, host_weights, tables, prefix, args.cpu_steps)
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wl, k, host_weights, tables, prefix, n_steps):
+    """The oracle as it stands on the host cores: n_steps decode steps after an untimed prefill."""
+    from oracle import spd_oracle as so
+
+    cfg = so.make_config(wl.shape, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, wl.prefix_len + n_steps + 2,
+                         wl.kv_dtype)
+    orc = so.Oracle(cfg, host_weights, tables)
+    t0 = time.time()
+    orc.prefill(prefix)
+    log("[bench] oracle prefill %.1fs" % (time.time() - t0))
+    t0 = time.perf_counter()
+    for _ in range(n_steps):
+        orc.step()
+    dt = time.perf_counter() - t0
+    orc.close()
+    return {"value": k * n_steps / dt, "unit": UNIT, "cores": so.max_threads(), "kind": "oracle",
+            "ms_per_step": dt / n_steps * 1e3,
+            "sample": "%d decode steps of the same workload after an untimed %d-token prefill" % (n_steps, wl.prefix_len)}
+
+
+def run_reference(args, wl):
+    """The CPU oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import spd_oracle as so
+
+    k, K, W = args.k or wl.k, args.steps, args.warmup
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    weights, tables, prefix = make_inputs(wl, dev, 0)
+    host = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in weights.items()}
+    del weights
+    cfg = so.make_config(wl.shape, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, wl.prefix_len + W + K + 2, wl.kv_dtype)
+    orc = so.Oracle(cfg, host, tables)
+    orc.prefill(prefix)
+    t1 = time.perf_counter()
+    for _ in range(W):
+        orc.step()
+    per = (time.perf_counter() - t1) / max(1, W)
+    K_run = K if W == 0 else max(1, min(K, int(150.0 / max(per, 1e-9))))
+    t0 = time.perf_counter()
+    for _ in range(K_run):
+        orc.step()
+    dt = time.perf_counter() - t0
+    value = k * K_run / dt
+    cores = so.max_threads()
+    sample = "%d decode steps (of %d asked) after an untimed %d-token prefill and %d warm-up steps" % (K_run, K, wl.prefix_len, W)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": K_run, "warmup": W,
+           "ms_per_step": dt / K_run * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+           "data": "synthetic",
+           "config": {"workload": "%s: %s-shape decoder, prefix %d, k=%d, bs1, n-gram n=%d..%d, %d entries/order" % (
+               wl.name, wl.shape.name, wl.prefix_len, k, min(wl.orders), max(wl.orders), wl.retain)},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=9)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="7b_k3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--k", type=int, default=0, help="override the number of drafts")
+    ap.add_argument("--reps", type=int, default=5, help="timed launches (median reported)")
+    ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kpass", action="store_true")
+    ap.add_argument("--stage-bytes", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    args = ap.parse_args()
+    if args.warmup < 1:
+        args.warmup = 1
+    wl = si.get_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
