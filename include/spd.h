@@ -198,6 +198,32 @@ int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes);
 int spd_debug_score(spd_ctx *ctx, const int32_t *hist, int32_t hist_len, const float *logp, const int32_t *cand_tok,
                     const float *cand_lp);
 
+/*
+ * The scoring stage of one timestep (what spd_debug_score runs) without any device allocation.  The
+ * paper has no counterpart to this call; it exists for callers that cannot allocate device memory
+ * at the point where they need a score: code running inside a memory-budgeted serving process whose
+ * pool is already carved up, plug-ins that are handed device pointers but no allocator, or code on a
+ * path where cudaMalloc's implicit device synchronisation is not acceptable.  Such callers have no
+ * workspace to give spd_create, so the draft state the kernel needs as scratch lives in a fixed 16 KB
+ * array inside the library image; every GPU that loads the library holds those 16 KB until the process
+ * exits.  The call neither allocates nor frees anything (no cudaMalloc / cudaFree, no allocating library).
+ *   cfg      HOST; only k, vocab, n_min, n_max, lambda, alpha, delta and stream are read.
+ *   tables   HOST array of n_tables descriptors whose ngram / ctx members are DEVICE pointers, ascending n.
+ *   hist     HOST int32 [k][hist_len], each draft's most recent tokens, oldest first;  logp HOST float [k];
+ *   cand_tok HOST int32 [k], cand_lp HOST float [k]: the kept tokens and their log-probabilities.
+ *   outputs  HOST, any may be NULL: out_sel int32 [k] chosen options i*k+j (best first), out_logp float [k],
+ *            out_gamma float [k] (Eq. 4), out_score float [k*k] (-inf = dropped option).
+ * Limits of the fixed scratch: k <= SPD_MAX_K (16), n_tables <= 8, hist_len <= 8; anything larger is
+ * refused with SPD_ERANGE.  The first call on each device looks up the array's device address (that
+ * device must be current); make that first call before any stream capture begins.  All calls on a
+ * device share the one array, which still holds the previous call's data when the next begins (each
+ * call overwrites it completely before launching); two calls whose device work overlaps, from
+ * different streams or threads, race on it, so serialise them.  Synchronises the stream before returning.
+ */
+int spd_score_static(const spd_config *cfg, const spd_ngram_table *tables, int32_t n_tables, const int32_t *hist,
+                     int32_t hist_len, const float *logp, const int32_t *cand_tok, const float *cand_lp,
+                     int32_t *out_sel, float *out_logp, float *out_gamma, float *out_score);
+
 /* Number of kernel launches this context has enqueued so far. */
 int64_t spd_launch_count(const spd_ctx *ctx);
 

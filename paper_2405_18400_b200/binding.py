@@ -65,7 +65,7 @@ _lib: Optional[C.CDLL] = None
 
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
-           "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring"]
+           "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static"]
 
 
 def load_library() -> C.CDLL:
@@ -100,6 +100,8 @@ def load_library() -> C.CDLL:
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
     L.spd_set_ring.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    L.spd_score_static.argtypes = [C.POINTER(SpdConfig), C.POINTER(_Table), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     _lib = L
     return L
 
@@ -272,3 +274,36 @@ class SpdContext:
         cand_lp = np.ascontiguousarray(cand_lp, dtype=np.float32)
         _check(self.lib.spd_debug_score(self.h, hist.ctypes.data, hist.shape[1], logp.ctypes.data, cand_tok.ctypes.data,
                                         cand_lp.ctypes.data), "spd_debug_score")
+
+
+def spd_score_static(k: int, vocab: int, orders: Sequence[int], lam: Sequence[float], alpha: float, delta: float,
+                     tables: Sequence[Dict[str, object]], hist: np.ndarray, logp, cand_tok, cand_lp,
+                     stream: Optional[torch.cuda.Stream] = None):
+    """Scoring stage through the entry point that allocates nothing on the device (for callers that
+    have device pointers but no allocator to obtain a workspace from).  `tables` come from
+    build_ngram_tables and live on the current CUDA device.  Returns (sel, logp, gamma, score)."""
+    L = load_library()
+    cfg = SpdConfig()
+    cfg.k, cfg.vocab = k, vocab
+    cfg.n_min, cfg.n_max = (min(orders), max(orders)) if len(orders) else (2, 2)
+    for i in range(MAX_ORDERS):
+        cfg.lam[i] = float(lam[i]) if i < len(lam) else 0.0
+    cfg.alpha, cfg.delta = alpha, delta
+    cfg.stream = stream.cuda_stream if stream is not None else None
+    tabs = (_Table * max(1, len(tables)))()
+    for i, t in enumerate(tables):
+        tabs[i].n, tabs[i].ngram_slots, tabs[i].ctx_slots = t["n"], t["ngram_slots"], t["ctx_slots"]
+        tabs[i].ngram, tabs[i].ctx = t["ngram"].data_ptr(), t["ctx"].data_ptr()
+    hist = np.ascontiguousarray(hist, dtype=np.int32)
+    logp = np.ascontiguousarray(logp, dtype=np.float32)
+    cand_tok = np.ascontiguousarray(cand_tok, dtype=np.int32)
+    cand_lp = np.ascontiguousarray(cand_lp, dtype=np.float32)
+    kk = max(1, min(k, MAX_K))
+    sel = np.zeros(kk, np.int32)
+    out_lp = np.zeros(kk, np.float32)
+    gamma = np.zeros(kk, np.float32)
+    score = np.zeros(kk * kk, np.float32)
+    _check(L.spd_score_static(C.byref(cfg), tabs, len(tables), hist.ctypes.data, hist.shape[1], logp.ctypes.data,
+                              cand_tok.ctypes.data, cand_lp.ctypes.data, sel.ctypes.data, out_lp.ctypes.data,
+                              gamma.ctypes.data, score.ctypes.data), "spd_score_static")
+    return sel, out_lp, gamma, score

@@ -958,3 +958,119 @@ extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm)
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void *>(&spd::spd_decode_kernel),
                                                        spd::kThreads, dyn_smem);
 }
+
+// ---------------------------------------------------------------- scoring stage without any allocation
+// spd_score_static (see include/spd.h): the scoring stage of one timestep for callers that cannot
+// allocate device memory.  The draft state the kernel normally keeps in the caller's workspace lives
+// here in a fixed array that is part of the loaded library image on every GPU.
+#include <cstring>
+#include <mutex>
+
+#include "spd.h"
+
+namespace {
+
+constexpr size_t kStaticStateBytes = (sizeof(spd::State) + 255) / 256 * 256;
+constexpr size_t kStaticScratchBytes = kStaticStateBytes + 2 * SPD_MAX_K * sizeof(int32_t);
+static_assert(kStaticScratchBytes <= 16384, "static scratch is documented as 16 KB");
+
+static __device__ __align__(256) unsigned char g_static_scratch[16384];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices] = {};  // device address of g_static_scratch, per device, filled on first use
+
+}  // namespace
+
+extern "C" int spd_score_static(const spd_config *cfg, const spd_ngram_table *tables, int32_t n_tables,
+                                const int32_t *hist, int32_t hist_len, const float *logp, const int32_t *cand_tok,
+                                const float *cand_lp, int32_t *out_sel, float *out_logp, float *out_gamma,
+                                float *out_score) {
+  if (!cfg || !hist || !logp || !cand_tok || !cand_lp || (n_tables > 0 && !tables)) return SPD_EINVAL;
+  // sizes beyond what the fixed scratch was laid out for are refused, never truncated
+  if (cfg->k < 1 || cfg->k > SPD_MAX_K || n_tables < 0 || n_tables > spd::kMaxTables || hist_len < 0 || hist_len > spd::kWin)
+    return SPD_ERANGE;
+  if (cfg->n_min < 2 || cfg->n_max > SPD_MAX_N || cfg->vocab < 1 || cfg->vocab > 65535) return SPD_EINVAL;
+  if (!(cfg->delta > 0.f) || cfg->delta > 1.f || !(cfg->alpha >= 0.f) || cfg->alpha > 1.f) return SPD_EINVAL;
+  const int k = cfg->k;
+  for (int t = 0; t < n_tables; ++t) {
+    const spd_ngram_table &tb = tables[t];
+    if (tb.n < 2 || tb.n > SPD_MAX_N || !tb.ngram || !tb.ctx || ((uintptr_t)tb.ngram % 16) || ((uintptr_t)tb.ctx % 16)) return SPD_EINVAL;
+    if (!tb.ngram_slots || (tb.ngram_slots & (tb.ngram_slots - 1)) || !tb.ctx_slots || (tb.ctx_slots & (tb.ctx_slots - 1)))
+      return SPD_EINVAL;
+    if (t > 0 && tables[t - 1].n >= tb.n) return SPD_EINVAL;
+  }
+  for (int i = 0; i < k; ++i) {
+    if (cand_tok[i] < 0 || cand_tok[i] >= cfg->vocab) return SPD_ERANGE;
+    for (int j = 0; j < hist_len; ++j)
+      if (hist[i * hist_len + j] < 0 || hist[i * hist_len + j] >= cfg->vocab) return SPD_ERANGE;
+  }
+
+  // Set-up, once per device, with that device current: in host code the array's name is only a
+  // stand-in for the symbol, so its device address is asked for and that address is what the kernel gets.
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPD_ECUDA;
+  unsigned char *scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+      void *ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+        cudaGetLastError();
+        return SPD_ECUDA;
+      }
+      g_static_ptr[dev] = ptr;
+    }
+    scratch = static_cast<unsigned char *>(g_static_ptr[dev]);
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cfg->stream);
+
+  // The array keeps whatever the previous call left: the whole state is overwritten with this call's
+  // inputs (everything else zero, including the error word), and so are the two history rows.
+  spd::State st;
+  std::memset(&st, 0, sizeof st);
+  st.win_len = hist_len;
+  for (int i = 0; i < k; ++i) {
+    for (int j = 0; j < hist_len; ++j) st.win[i][spd::kWin - hist_len + j] = hist[i * hist_len + j];
+    st.logP[i] = logp[i];
+    st.cand_tok[i] = cand_tok[i];
+    st.cand_lp[i] = cand_lp[i];
+  }
+  if (cudaMemcpyAsync(scratch, &st, sizeof st, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SPD_ECUDA;
+  if (cudaMemsetAsync(scratch + kStaticStateBytes, 0, 2 * SPD_MAX_K * sizeof(int32_t), stream) != cudaSuccess) return SPD_ECUDA;
+
+  spd::KParams kp;
+  std::memset(&kp, 0, sizeof kp);
+  kp.k = k; kp.n_min = cfg->n_min; kp.n_max = cfg->n_max; kp.n_tables = n_tables;
+  for (int i = 0; i < 8; ++i) kp.lambda[i] = cfg->lambda[i];
+  kp.alpha = cfg->alpha;
+  kp.log_delta = logf(cfg->delta);
+  for (int t = 0; t < n_tables; ++t) {
+    kp.tab[t].n = tables[t].n;
+    kp.tab[t].ngram = static_cast<const SpdSlot *>(tables[t].ngram);
+    kp.tab[t].ctx = static_cast<const SpdSlot *>(tables[t].ctx);
+    kp.tab[t].ngram_mask = tables[t].ngram_slots - 1;
+    kp.tab[t].ctx_mask = tables[t].ctx_slots - 1;
+  }
+  kp.st = reinterpret_cast<spd::State *>(scratch);
+  kp.hist_tok = reinterpret_cast<int32_t *>(scratch + kStaticStateBytes);
+  kp.hist_par = kp.hist_tok + SPD_MAX_K;
+  kp.mode = spd::kModeScoreOnly;
+  kp.stage_bytes = 0;
+  kp.n_stages = 1;
+  spd::spd_decode_kernel<<<1, spd::kThreads, 20480, stream>>>(kp);
+  if (cudaGetLastError() != cudaSuccess) return SPD_ECUDA;
+
+  spd::State back;
+  if (cudaMemcpyAsync(&back, scratch, sizeof back, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SPD_ECUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return SPD_ECUDA;
+  if (back.err) return back.err;
+  for (int i = 0; i < k; ++i) {
+    if (out_sel) out_sel[i] = back.sel[i];
+    if (out_logp) out_logp[i] = back.logP[i];
+    if (out_gamma) out_gamma[i] = back.gamma[i];
+  }
+  if (out_score)
+    for (int q = 0; q < k * k; ++q) out_score[q] = back.score[q];
+  return SPD_OK;
+}
