@@ -198,14 +198,14 @@ def run_ours(args, wl):
     # ---- end to end through the C ABI with host buffers: prefill(host ids) + per-step calls returning to the host
     gen = wl.gen_tokens
     e2e_t = []
-    for _ in range(2):
+    for _ in range(0 if args.no_e2e else 2):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         ctx.spd_prefill(prefix)
         for _ in range(gen - 1):
             ctx.spd_step()
         e2e_t.append(time.perf_counter() - t0)
-    e2e_s = min(e2e_t)
+    e2e_s = min(e2e_t) if e2e_t else float("nan")
     if world > 1:
         import torch.distributed as dist
         t = torch.tensor([e2e_s], device=dev)
@@ -328,10 +328,21 @@ def main():
     ap.add_argument("--no-kpass", action="store_true")
     ap.add_argument("--stage-bytes", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="profiling only: keep this many layers of the shape")
+    ap.add_argument("--retain", type=int, default=0, help="profiling only: n-grams kept per order")
+    ap.add_argument("--stream-len", type=int, default=0, help="profiling only: tokens of the n-gram corpus")
+    ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.warmup < 1:
         args.warmup = 1
     wl = si.get_workload(args.workload)
+    if args.layers or args.retain or args.stream_len:
+        import dataclasses
+        sh = wl.shape
+        if args.layers:
+            sh = dataclasses.replace(sh, n_layers=args.layers, name="%s[%d layers]" % (sh.name, args.layers))
+        wl = dataclasses.replace(wl, shape=sh, retain=args.retain or wl.retain, stream_len=args.stream_len or wl.stream_len,
+                                 name=wl.name + "-reduced")
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -69,16 +69,19 @@ EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_
 
 
 def load_library() -> C.CDLL:
-    """Loads libspd.so, building it first when its sources are newer.  Raises if neither is possible."""
+    """Loads libspd.so, building it first when its sources are newer (the environment variable
+    SPD_LIBRARY names another build of the library to load instead).  Raises if neither is possible."""
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
-    try:
-        path = _build.build()
-    except Exception as exc:  # no compiler on this machine: the prebuilt library must be there
-        if not os.path.exists(path):
-            raise RuntimeError("libspd.so is missing and could not be built: %s" % exc) from exc
+    path = os.environ.get("SPD_LIBRARY", "")
+    if not path:
+        path = _build.LIB
+        try:
+            path = _build.build()
+        except Exception as exc:  # no compiler on this machine: the prebuilt library must be there
+            if not os.path.exists(path):
+                raise RuntimeError("libspd.so is missing and could not be built: %s" % exc) from exc
     L = C.CDLL(path)
     L.spd_workspace_bytes.argtypes = [C.POINTER(SpdConfig), C.POINTER(C.c_size_t)]
     L.spd_create.argtypes = [C.POINTER(SpdConfig), C.POINTER(_Weights), C.POINTER(_Table), C.c_int32, C.c_void_p,

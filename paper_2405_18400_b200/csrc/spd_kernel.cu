@@ -674,7 +674,8 @@ __device__ void tail_keep_topk(const KParams &p) {
     }
     warp_best(bv, bi);
     if (lane == 0) {
-      st->cand_tok[j] = bi;
+      // non-finite logits can leave a round without a winner: keep the token id valid
+      st->cand_tok[j] = bi < 0 ? 0 : bi;
       st->cand_lp[j] = bv * p.inv_tau - lse;
     }
     pv = bv;
