@@ -29,6 +29,11 @@ import torch
 
 import spd_inputs as si
 
+# dram bytes (read + write) / algorithmic bytes measured by ncu on the 4-layer case of the same kernel
+# (profiles/spd_decode_kernel_7b_k3.md); traffic grows in proportion to the layers streamed.  Set to None
+# whenever the kernel changes until the counters are taken again.
+TRAFFIC_RATIO = 1.006
+
 METRIC = "k-draft tokens/s"
 UNIT = "tokens/s"
 
@@ -205,16 +210,16 @@ def run_ours(args, wl):
         for _ in range(gen - 1):
             ctx.spd_step()
         e2e_t.append(time.perf_counter() - t0)
-    e2e_s = min(e2e_t) if e2e_t else float("nan")
-    if world > 1:
+    e2e_s = min(e2e_t) if e2e_t else None
+    if world > 1 and e2e_s:
         import torch.distributed as dist
         t = torch.tensor([e2e_s], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
-    e2e = {"value": world * k * gen / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len / gen,
+    e2e = {"value": world * k * gen / e2e_s if e2e_s else None, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len / gen,
            "d2h_bytes_per_step": 12.0 * k, "what": "spd_prefill(host ids) + %d spd_step calls returning ids, parents and gamma "
            "to the host, per request of %d tokens per draft; prefill replays the decode kernels token by token" % (gen - 1, gen),
-           "ms_per_request": e2e_s * 1e3}
+           "ms_per_request": e2e_s * 1e3 if e2e_s else None}
 
     # ---- the same number of drafts from k separate single-draft passes through the same kernels
     kpass = None
@@ -242,7 +247,7 @@ def run_ours(args, wl):
             wl.name, wl.shape.name, wl.prefix_len, k, "%d..%d" % (min(wl.orders), max(wl.orders)), wl.retain),
             "l2": "inputs_exceed_l2", "kv_dtype": wl.kv_dtype, "parallelism": "replicas x%d" % world, "reps": reps},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_decode_kernel"},
+                     "traffic": TRAFFIC_RATIO * bytes_step * K if TRAFFIC_RATIO else None, "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_decode_kernel"},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
     }
     if kpass:
