@@ -60,6 +60,21 @@ def step_bytes(wl, k, T):
             + s.n_layers * 2 * T * s.d_model * kvb + (k + k * k) * len(wl.orders) * 32)
 
 
+def max_over_ranks(x: float, dev, world: int) -> float:
+    """The slowest rank's value (every rank gets it); a plain pass-through for one rank."""
+    if world <= 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, k: int, steps: int, ms: float) -> float:
+    """Whole-job k-draft tokens per second: every rank advances k drafts by `steps` tokens in `ms`."""
+    return world * k * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -188,17 +203,12 @@ def run_ours(args, wl):
     launches = ctx.spd_launch_count() - launches0
     time.sleep(0.2)
     clocks = sampler.stop()
-    ms = float(np.median(ms_list))
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(float(np.median(ms_list)), dev, world)
     T_mid = wl.prefix_len + W + (K + 1) // 2
     bytes_step = step_bytes(wl, k, T_mid)
     peak, peak_kind = measured_peak_gbs()
     achieved = bytes_step * K / (ms * 1e-3) / 1e9
-    value = world * k * K / (ms * 1e-3)
+    value = job_throughput(world, k, K, ms)
 
     # ---- end to end through the C ABI with host buffers: prefill(host ids) + per-step calls returning to the host
     gen = wl.gen_tokens
@@ -211,11 +221,8 @@ def run_ours(args, wl):
             ctx.spd_step()
         e2e_t.append(time.perf_counter() - t0)
     e2e_s = min(e2e_t) if e2e_t else None
-    if world > 1 and e2e_s:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    if e2e_s:
+        e2e_s = max_over_ranks(e2e_s, dev, world)
     e2e = {"value": world * k * gen / e2e_s if e2e_s else None, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len / gen,
            "d2h_bytes_per_step": 12.0 * k, "what": "spd_prefill(host ids) + %d spd_step calls returning ids, parents and gamma "
            "to the host, per request of %d tokens per draft; prefill replays the decode kernels token by token" % (gen - 1, gen),
