@@ -181,11 +181,13 @@ int spd_ngram_build(int32_t n, int64_t n_entries, const int32_t *keys, const int
  *   SPD_DBG_HIST_IN   int32 [k][8]         last 8 tokens of each draft before the last step's selection (right-aligned)
  *   SPD_DBG_TRACE     float [n_layers][2][d_model]  residual after attention / after the FFN of the last LM pass
  *   SPD_DBG_HIDDEN    float [d_model]      residual stream after the last LM pass
+ *   SPD_DBG_KCACHE    float [n_layers][T][d_model]  cached keys of the T positions written so far (T = prefix
+ *                     length + tokens generated - 1), widened to float32;  SPD_DBG_VCACHE likewise for values
  * SPD_ENOMEM if `bytes` is smaller than the buffer.
  */
 enum {
   SPD_DBG_LOGITS = 0, SPD_DBG_CAND_TOK, SPD_DBG_CAND_LP, SPD_DBG_LOGP_IN, SPD_DBG_SCORE, SPD_DBG_PNG, SPD_DBG_CNT,
-  SPD_DBG_TOT, SPD_DBG_SEL, SPD_DBG_LOGP, SPD_DBG_HIST_IN, SPD_DBG_TRACE, SPD_DBG_HIDDEN
+  SPD_DBG_TOT, SPD_DBG_SEL, SPD_DBG_LOGP, SPD_DBG_HIST_IN, SPD_DBG_TRACE, SPD_DBG_HIDDEN, SPD_DBG_KCACHE, SPD_DBG_VCACHE
 };
 int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes);
 

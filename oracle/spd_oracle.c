@@ -74,6 +74,9 @@ typedef struct {
   double logP[ORC_MAX_K], gamma[ORC_MAX_K];
   double *logits;   /* [vocab], last LM pass */
   double *trace;    /* [L][2][d]: last processed position's residual after attention / after FFN */
+  const float *force_k, *force_v; /* [L][force_T][d] cache values to adopt where they are a valid rounding, or NULL */
+  int force_T;
+  int64_t force_flips, force_bad;
   /* last step's intermediates */
   int32_t cand_tok[ORC_MAX_K];
   double cand_lp[ORC_MAX_K];
@@ -167,6 +170,26 @@ static float quant_kv(const orc_config *c, double x) {
 }
 
 /*
+ * The cache value for the exact value x.  Rounding to the cache type is a decision that float
+ * rounding can tip either way when x lies within rounding error of the midpoint of two
+ * representable values.  When the tests supply another implementation's cache value `other`, it is adopted
+ * if it is x rounded to its other neighbour (|other - x| below the spacing of the cache type in x's
+ * binade); anything else is counted as a mismatch and not adopted.
+ */
+static float follow_kv(orc_ctx *o, double x, const float *other) {
+  float own = quant_kv(&o->c, x);
+  if (!other) return own;
+  if (*other == own) return own;
+  double spacing = x == 0.0 ? 0.0 : ldexp(1.0, ilogb(x) - (o->c.kv_dtype == 1 ? 7 : 23));
+  if (fabs((double)*other - x) < spacing) {
+    o->force_flips++;
+    return *other;
+  }
+  o->force_bad++;
+  return own;
+}
+
+/*
  * The decoder over m new positions pos0..pos0+m-1 whose input rows are X[m][d]; the positions
  * before pos0 are already in the cache.  Layer by layer over all new positions (the dense causal
  * pass); m = 1 is an ordinary cached decode step.  Leaves the final residual rows in X.
@@ -195,8 +218,11 @@ static void decoder_forward(orc_ctx *o, double *X, int m, int pos0) {
         orc_rope(Kn + (size_t)t * d + h * hd, hd, pos0 + t, c->rope_theta);
       }
       for (int j = 0; j < d; ++j) {
-        kc[(size_t)(pos0 + t) * d + j] = quant_kv(c, Kn[(size_t)t * d + j]);
-        vc[(size_t)(pos0 + t) * d + j] = quant_kv(c, Vn[(size_t)t * d + j]);
+        const int fp = pos0 + t;
+        const float *fk = (o->force_k && fp < o->force_T) ? o->force_k + ((size_t)l * o->force_T + fp) * d + j : NULL;
+        const float *fv = (o->force_v && fp < o->force_T) ? o->force_v + ((size_t)l * o->force_T + fp) * d + j : NULL;
+        kc[(size_t)fp * d + j] = follow_kv(o, Kn[(size_t)t * d + j], fk);
+        vc[(size_t)fp * d + j] = follow_kv(o, Vn[(size_t)t * d + j], fv);
       }
     }
 #pragma omp parallel for collapse(2) schedule(static)
@@ -483,6 +509,31 @@ void orc_step_commit(orc_ctx *o, const int32_t *sel, const double *new_logP) {
   free(nd);
   o->len += 1;
   orc_gamma(o->logP, k, o->gamma);
+}
+
+/*
+ * Gives the next LM passes another implementation's cache contents ([L][T][d] keys and values as float32)
+ * to follow wherever they are a valid rounding of this oracle's exact values; NULL switches it off.
+ * flips / bad (either may be NULL) report how many values were adopted / refused since the last call.
+ */
+void orc_follow_cache(orc_ctx *o, const float *k, const float *v, int T, int64_t *flips, int64_t *bad) {
+  if (flips) *flips = o->force_flips;
+  if (bad) *bad = o->force_bad;
+  o->force_k = k;
+  o->force_v = v;
+  o->force_T = T;
+  o->force_flips = o->force_bad = 0;
+}
+
+/*
+ * Replaces the draft log-probabilities (and with them gamma, Eq. 4).  The tests use it so that a
+ * stage-by-stage comparison feeds both implementations the same superposed input: at tau = 0.06 a logit
+ * difference of e moves a log-probability by e / tau, so rounding-level differences in one step's logits
+ * would otherwise change the next step's input.
+ */
+void orc_set_logP(orc_ctx *o, const double *logP) {
+  for (int i = 0; i < o->c.k; ++i) o->logP[i] = logP[i];
+  orc_gamma(o->logP, o->c.k, o->gamma);
 }
 
 /* One later timestep of Algorithm 1.  out_parent[r] = index of the draft that new draft r extends. */

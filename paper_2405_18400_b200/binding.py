@@ -15,7 +15,7 @@ MAX_ORDERS = 8
 
 DBG = {name: i for i, name in enumerate(
     ["LOGITS", "CAND_TOK", "CAND_LP", "LOGP_IN", "SCORE", "PNG", "CNT", "TOT", "SEL", "LOGP", "HIST_IN", "TRACE",
-     "HIDDEN"])}
+     "HIDDEN", "KCACHE", "VCACHE"])}
 
 _STATUS = {0: "SPD_OK", -1: "SPD_EINVAL", -2: "SPD_ESTATE", -3: "SPD_ERANGE", -4: "SPD_ENOMEM", -5: "SPD_ECUDA",
            -6: "SPD_ETABLE", -7: "SPD_ETIMEOUT"}
@@ -258,13 +258,16 @@ class SpdContext:
     def spd_launch_count(self) -> int:
         return int(self.lib.spd_launch_count(self.h))
 
-    def spd_debug_read(self, what: str) -> np.ndarray:
+    def spd_debug_read(self, what: str, positions: int = 0) -> np.ndarray:
+        """`positions` (KCACHE / VCACHE only) = cached positions so far: prefix length + tokens generated - 1."""
         k, c = self.k, self.cfg
         shapes = {"LOGITS": (np.float32, (c.vocab,)), "CAND_TOK": (np.int32, (k,)), "CAND_LP": (np.float32, (k,)),
                   "LOGP_IN": (np.float32, (k,)), "SCORE": (np.float32, (k * k,)), "PNG": (np.float32, (k * k,)),
                   "CNT": (np.int32, (k * k, 8)), "TOT": (np.int32, (k, 8)), "SEL": (np.int32, (k,)),
                   "LOGP": (np.float32, (k,)), "HIST_IN": (np.int32, (k, 8)),
                   "TRACE": (np.float32, (c.n_layers, 2, c.d_model)), "HIDDEN": (np.float32, (c.d_model,))}
+        if what in ("KCACHE", "VCACHE"):
+            shapes[what] = (np.float32, (c.n_layers, int(positions), c.d_model))
         dt, shp = shapes[what]
         out = np.zeros(shp, dt)
         _check(self.lib.spd_debug_read(self.h, DBG[what], out.ctypes.data, out.nbytes), "spd_debug_read")

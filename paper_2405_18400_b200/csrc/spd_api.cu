@@ -455,6 +455,24 @@ int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes) {
     case SPD_DBG_HIST_IN: return copy_rows(st + offsetof(spd::State, win_in), k, spd::kWin * 4, spd::kWin * 4);
     case SPD_DBG_TRACE: return copy(ctx->ws + ctx->lay.trace, (size_t)c.n_layers * 2 * c.d_model * 4);
     case SPD_DBG_HIDDEN: return copy(ctx->ws + ctx->lay.h, (size_t)c.d_model * 4);
+    case SPD_DBG_KCACHE:
+    case SPD_DBG_VCACHE: {
+      const int T = ctx->prefilled ? ctx->m + ctx->n_gen - 1 : 0;
+      const size_t rows = (size_t)c.n_layers, row_elems = (size_t)T * c.d_model, esz = c.kv_dtype ? 2 : 4;
+      if (bytes < rows * row_elems * 4) return SPD_ENOMEM;
+      if (T == 0) return SPD_OK;
+      const uint8_t *src = ctx->ws + (what == SPD_DBG_KCACHE ? ctx->lay.kcache : ctx->lay.vcache);
+      // the raw rows land in the tail of the caller's buffer, then are widened in place from the front
+      uint8_t *raw = static_cast<uint8_t *>(host_buf) + rows * row_elems * (4 - esz);
+      SPD_CUDA(cudaMemcpy2D(raw, row_elems * esz, src, (size_t)c.max_pos * c.d_model * esz, row_elems * esz, rows,
+                            cudaMemcpyDeviceToHost));
+      if (esz == 2) {
+        const uint16_t *in = reinterpret_cast<const uint16_t *>(raw);
+        uint32_t *out = static_cast<uint32_t *>(host_buf);
+        for (size_t i = 0; i < rows * row_elems; ++i) out[i] = (uint32_t)in[i] << 16;
+      }
+      return SPD_OK;
+    }
     default: return SPD_EINVAL;
   }
 }

@@ -21,9 +21,10 @@ def test_tiny_workload_stepwise(tiny_inputs, kv_dtype):
     for _ in range(wl.gen_tokens - 1):
         compare_step(ctx, orc, stats)
         assert np.abs(ctx.spd_debug_read("TRACE").astype(np.float64) - orc.trace()).max() < 1e-3
-    assert max(s["eps_z"] for s in stats) < 2e-4          # far inside the 2e-2 bound when quantisation points agree
-    if max(s["eps_z"] for s in stats) <= 2e-5:
-        assert max(s["dgamma"] for s in stats) <= GAMMA_TOL
+    errs = [s for s in stats if "eps_z" in s]
+    assert max(s["eps_z"] for s in errs) < 2e-4           # far inside the 2e-2 bound when quantisation points agree
+    if max(s["eps_z"] for s in errs) <= 2e-5:
+        assert max(s["dgamma"] for s in errs) <= GAMMA_TOL
     toks, lp, g = ctx.spd_generate(1, wl.gen_tokens + 1)
     ids_o, par_o, g_o = orc.step()
     assert np.array_equal(toks, orc.drafts()[:, len(prefix):])

@@ -139,3 +139,38 @@ def test_bf16_cache_holds_bf16_values(tiny_inputs):
         t = torch.from_numpy(np.ascontiguousarray(a))
         assert torch.equal(t.to(torch.bfloat16).to(torch.float32), t) and t.abs().max() > 0
     assert np.all(k[:, 16:] == 0)
+
+
+def test_cache_following_adopts_only_valid_roundings(tiny_inputs):
+    wl, weights, tables, prefix = tiny_inputs
+    cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "bf16")
+    a = so.Oracle(cfg, weights, tables)
+    a.prefill(prefix)
+    k, v = (x[:, :16].copy() for x in a.kv_cache())
+    z0 = a.logits()
+    b = so.Oracle(cfg, weights, tables)
+    b.follow_cache(k, v)
+    b.prefill(prefix)
+    assert b.follow_cache(None) == (0, 0) and np.array_equal(b.logits(), z0)      # its own values: nothing to adopt
+    # layer 0 keys moved one bf16 value up or down: adopted where that is the exact value's other neighbour,
+    # refused where it is two values away
+    k2 = k.copy()
+    bits = k2[0].view(np.uint32)
+    up = np.random.default_rng(0).random(bits.shape) < 0.5
+    bits[up] += np.uint32(1 << 16)
+    bits[~up] -= np.uint32(1 << 16)
+    c = so.Oracle(cfg, weights, tables)
+    c.follow_cache(k2, v)
+    c.prefill(prefix)
+    flips, bad = c.follow_cache(None)
+    got = c.kv_cache()[0][0, :16]
+    adopted, refused = int(np.count_nonzero(got == k2[0])), int(np.count_nonzero(got == k[0]))
+    assert adopted + refused == k2[0].size and adopted > 0.3 * k2[0].size and refused > 0.3 * k2[0].size
+    assert flips >= adopted and bad >= refused      # later layers, now fed different inputs, add to both counts
+    # values that are no rounding of the exact ones are refused and counted
+    k3 = k.copy()
+    k3[1, 3, :7] += 1.0
+    d = so.Oracle(cfg, weights, tables)
+    d.follow_cache(k3, v)
+    d.prefill(prefix)
+    assert d.follow_cache(None) == (0, 7) and np.array_equal(d.logits(), z0)
