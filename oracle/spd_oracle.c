@@ -76,6 +76,7 @@ typedef struct {
   double *trace;    /* [L][2][d]: last processed position's residual after attention / after FFN */
   const float *force_k, *force_v; /* [L][force_T][d] cache values to adopt where they are a valid rounding, or NULL */
   int force_T;
+  double force_slack;
   int64_t force_flips, force_bad;
   /* last step's intermediates */
   int32_t cand_tok[ORC_MAX_K];
@@ -173,15 +174,17 @@ static float quant_kv(const orc_config *c, double x) {
  * The cache value for the exact value x.  Rounding to the cache type is a decision that float
  * rounding can tip either way when x lies within rounding error of the midpoint of two
  * representable values.  When the tests supply another implementation's cache value `other`, it is adopted
- * if it is x rounded to its other neighbour (|other - x| below the spacing of the cache type in x's
- * binade); anything else is counted as a mismatch and not adopted.
+ * if it is a rounding of some value within `slack` of x (|other - x| below the spacing of the cache type
+ * in x's binade plus slack, slack being the caller's bound on the other side's float error in absolute
+ * terms: for values near zero that error exceeds the local spacing); anything else is counted as a
+ * mismatch and not adopted.
  */
 static float follow_kv(orc_ctx *o, double x, const float *other) {
   float own = quant_kv(&o->c, x);
   if (!other) return own;
   if (*other == own) return own;
   double spacing = x == 0.0 ? 0.0 : ldexp(1.0, ilogb(x) - (o->c.kv_dtype == 1 ? 7 : 23));
-  if (fabs((double)*other - x) < spacing) {
+  if (fabs((double)*other - x) < spacing + o->force_slack) {
     o->force_flips++;
     return *other;
   }
@@ -513,15 +516,17 @@ void orc_step_commit(orc_ctx *o, const int32_t *sel, const double *new_logP) {
 
 /*
  * Gives the next LM passes another implementation's cache contents ([L][T][d] keys and values as float32)
- * to follow wherever they are a valid rounding of this oracle's exact values; NULL switches it off.
+ * to follow wherever they are a valid rounding of this oracle's exact values (to within `slack`, see
+ * follow_kv); NULL switches it off.
  * flips / bad (either may be NULL) report how many values were adopted / refused since the last call.
  */
-void orc_follow_cache(orc_ctx *o, const float *k, const float *v, int T, int64_t *flips, int64_t *bad) {
+void orc_follow_cache(orc_ctx *o, const float *k, const float *v, int T, double slack, int64_t *flips, int64_t *bad) {
   if (flips) *flips = o->force_flips;
   if (bad) *bad = o->force_bad;
   o->force_k = k;
   o->force_v = v;
   o->force_T = T;
+  o->force_slack = slack;
   o->force_flips = o->force_bad = 0;
 }
 

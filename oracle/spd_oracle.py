@@ -60,7 +60,7 @@ def lib() -> C.CDLL:
         L.orc_step_commit.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_feed_token.argtypes = [C.c_void_p, C.c_int32]
         L.orc_set_logP.argtypes = [C.c_void_p, C.c_void_p]
-        L.orc_follow_cache.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_follow_cache.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_void_p]
         for name in ("orc_logits", "orc_trace", "orc_logP", "orc_gamma_now", "orc_cand_tok", "orc_cand_lp",
                      "orc_scores", "orc_png_last", "orc_cnt_last", "orc_tot_last", "orc_sel_last", "orc_drafts",
                      "orc_kcache", "orc_vcache"):
@@ -196,17 +196,18 @@ class Oracle:
         a = np.ascontiguousarray(logP, dtype=np.float64)
         lib().orc_set_logP(self.h, _ptr(a))
 
-    def follow_cache(self, k=None, v=None):
+    def follow_cache(self, k=None, v=None, slack: float = 0.0):
         """Follow the given cache contents (float32 [L, T, d]) in later passes; returns (adopted, refused)
-        counts accumulated since the previous call."""
+        counts accumulated since the previous call.  slack = absolute float error allowed for the other side."""
         flips, bad = C.c_int64(), C.c_int64()
         if k is None:
             self._fk = self._fv = None
-            lib().orc_follow_cache(self.h, None, None, 0, C.byref(flips), C.byref(bad))
+            lib().orc_follow_cache(self.h, None, None, 0, 0.0, C.byref(flips), C.byref(bad))
         else:
             self._fk = np.ascontiguousarray(k, dtype=np.float32)
             self._fv = np.ascontiguousarray(v, dtype=np.float32)
-            lib().orc_follow_cache(self.h, _ptr(self._fk), _ptr(self._fv), self._fk.shape[1], C.byref(flips), C.byref(bad))
+            lib().orc_follow_cache(self.h, _ptr(self._fk), _ptr(self._fv), self._fk.shape[1], float(slack), C.byref(flips),
+                                   C.byref(bad))
         return flips.value, bad.value
 
     def feed_token(self, tok: int) -> None:
