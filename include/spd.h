@@ -48,8 +48,7 @@ typedef struct spd_ctx spd_ctx; /* opaque; small host object owned by the librar
  * multi-head attention with rotary embedding on adjacent pairs (2i, 2i+1), angle
  * pos * rope_theta^(-2i/head_dim) -> residual -> RMSNorm -> SwiGLU feed-forward -> residual; final
  * RMSNorm; untied output projection.  head_dim = d_model / n_heads must be a multiple of 32, at
- * most 256; d_model and d_ffn multiples of 8; d_model <= 6144; vocab <= 65535; max_pos = positions the
- * KV cache holds.
+ * most 256; d_model and d_ffn multiples of 8; vocab <= 65535; max_pos = positions the KV cache holds.
  * Method: k drafts (1..SPD_MAX_K); n-gram orders n_min..n_max (2..SPD_MAX_N) with interpolation
  * weights lambda[n-2] (Eq. 5, Appendix B); alpha of Eq. 6; tau = softmax temperature applied to
  * the logits before anything else; delta of Eq. 7 (0 < delta <= 1; the paper gives no value).
@@ -230,10 +229,9 @@ int spd_score_static(const spd_config *cfg, const spd_ngram_table *tables, int32
 /* Number of kernel launches this context has enqueued so far. */
 int64_t spd_launch_count(const spd_ctx *ctx);
 
-/* Tuning knobs of the weight-streaming ring (bytes per stage, stages); 0 keeps the default (32768 bytes,
- * as many stages as fit).  A stage holds 4 whole rows, or 8 pieces of rows too long for that.  Takes effect
- * from the next launch.  SPD_EINVAL if stage_bytes is below 2048 or not a multiple of 128, or shared
- * memory would overflow. */
+/* Tuning knobs of the weight-streaming ring (bytes per stage, stages); 0 keeps the default.  Takes
+ * effect from the next launch.  SPD_EINVAL if a matrix row does not fit a stage or shared memory
+ * would overflow. */
 int spd_set_ring(spd_ctx *ctx, int32_t stage_bytes, int32_t n_stages);
 
 #ifdef __cplusplus

@@ -28,18 +28,13 @@ int cuda_fail(cudaError_t e, const char *what) {
     if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
   } while (0)
 
-constexpr size_t kPartBytes = sizeof(float) * 2 * spd::kTile * spd::kPartStride;  // row partials, after the ring
-constexpr size_t kMinFragBytes = 26880;  // the fragment area also serves the attention merge, the tail and the
-                                         // per-warp fragment prefetch buffers (2 x 7 warps x 5 x 12 x 32 bytes)
+constexpr size_t kPartBytes = 20480;  // per-block scratch after the ring: row partials / attention merge / tail
 constexpr size_t kSmemLimit = 232448; // 227 KB opt-in maximum per block on sm_100
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// x as tensor-core A fragments: 12 lanes x 8 words per 64-column pair-block
-size_t frag_bytes(int cols) { return (size_t)((cols + 63) / 64) * 12 * 8 * 4; }
-
 struct Layout {
-  size_t kcache, vcache, rope, layers, h, q, ufrag, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
+  size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
       trace, total;
 };
 
@@ -50,7 +45,7 @@ bool valid_config(const spd_config *c) {
   const int hd = c->d_model / c->n_heads;
   if (hd % 32 || hd > 256) return false;
   if (c->vocab > 65535) return false;
-  if (c->d_model > spd::kMaxVec * spd::kConsumerThreads * 8) return false;
+  if (c->d_model > spd::kMaxVec * spd::kConsumerThreads * 8 || c->d_ffn > spd::kMaxVec * spd::kConsumerThreads * 8) return false;
   if (c->k < 1 || c->k > SPD_MAX_K) return false;
   if (c->n_min < 2 || c->n_max > SPD_MAX_N) return false;
   if (!(c->tau > 0.f) || !(c->delta > 0.f) || c->delta > 1.f || !(c->alpha >= 0.f) || c->alpha > 1.f) return false;
@@ -76,7 +71,7 @@ Layout make_layout(const spd_config &c, int grid) {
   L.layers = take((size_t)c.n_layers * sizeof(spd::LayerW));
   L.h = take((size_t)c.d_model * 4);
   L.q = take((size_t)c.d_model * 4);
-  L.ufrag = take(frag_bytes(c.d_ffn));
+  L.u = take((size_t)c.d_ffn * 4);
   L.logits = take((size_t)c.vocab * 4);
   L.opart = take((size_t)c.n_heads * spd::kMaxSplit * hd * 4);
   L.oml = take((size_t)c.n_heads * spd::kMaxSplit * sizeof(float2));
@@ -113,18 +108,12 @@ struct spd_ctx {
 
 namespace {
 
-// shared memory after the ring: row partials, then x as fragments (also the attention and tail scratch)
-size_t scratch_bytes(const spd_config &c) {
-  size_t frag = frag_bytes(c.d_model);
-  if (frag < kMinFragBytes) frag = kMinFragBytes;
-  return kPartBytes + align_up(frag, 128);
-}
-
-// A stage holds 4 whole rows (or 8 row pieces of a segment); 32 KB by default.
 int pick_ring(const spd_config &c, int32_t stage_bytes, int32_t n_stages, int32_t *out_stage, int32_t *out_n) {
+  const size_t maxrow = (size_t)2 * (c.d_model > c.d_ffn ? c.d_model : c.d_ffn);
   size_t sb = stage_bytes > 0 ? (size_t)stage_bytes : 32768;
-  if (sb % 128 || sb < 2048) return SPD_EINVAL;
-  const size_t avail = kSmemLimit - scratch_bytes(c) - 2048;  // static shared memory and alignment slack
+  if (stage_bytes <= 0 && sb < maxrow) sb = align_up(maxrow, 1024);
+  if (sb % 128 || sb < maxrow) return SPD_EINVAL;
+  const size_t avail = kSmemLimit - kPartBytes - 2048;  // static shared memory and alignment slack
   int ns = n_stages > 0 ? n_stages : (int)(avail / sb);
   if (ns > spd::kMaxStages) ns = spd::kMaxStages;
   if (ns < 2 || (size_t)ns * sb > avail) return SPD_EINVAL;
@@ -242,7 +231,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   std::memset(&kp, 0, sizeof kp);
   int rc = pick_ring(*cfg, 0, 0, &kp.stage_bytes, &kp.n_stages);
   if (rc) return fail(rc);
-  ctx->dyn_smem = (size_t)kp.stage_bytes * kp.n_stages + scratch_bytes(*cfg);
+  ctx->dyn_smem = (size_t)kp.stage_bytes * kp.n_stages + kPartBytes;
   int per_sm = 0;
   e = spd_internal_prepare(ctx->dyn_smem, &per_sm);
   if (e != cudaSuccess) return fail(cuda_fail(e, "kernel attributes"));
@@ -271,7 +260,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.rope = reinterpret_cast<const float2 *>(ws + lay.rope);
   kp.layers = reinterpret_cast<const spd::LayerW *>(ws + lay.layers);
   kp.h = reinterpret_cast<float *>(ws + lay.h); kp.q = reinterpret_cast<float *>(ws + lay.q);
-  kp.ufrag = reinterpret_cast<unsigned short *>(ws + lay.ufrag); kp.logits = reinterpret_cast<float *>(ws + lay.logits);
+  kp.u = reinterpret_cast<float *>(ws + lay.u); kp.logits = reinterpret_cast<float *>(ws + lay.logits);
   kp.opart = reinterpret_cast<float *>(ws + lay.opart); kp.oml = reinterpret_cast<float2 *>(ws + lay.oml);
   kp.pk_val = reinterpret_cast<float *>(ws + lay.pk_val); kp.pk_id = reinterpret_cast<int32_t *>(ws + lay.pk_id);
   kp.pk_ms = reinterpret_cast<float2 *>(ws + lay.pk_ms);
@@ -300,7 +289,6 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   e = cudaMemcpyAsync(ws + lay.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ws + lay.layers, layers.data(), layers.size() * sizeof(spd::LayerW), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.state, 0, sizeof(spd::State), s);
-  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.ufrag, 0, frag_bytes(cfg->d_ffn), s);  // columns past d_ffn stay zero
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.trace, 0, (size_t)cfg->n_layers * 2 * cfg->d_model * 4, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return fail(cuda_fail(e, "workspace initialisation"));
@@ -319,7 +307,7 @@ int spd_set_ring(spd_ctx *ctx, int32_t stage_bytes, int32_t n_stages) {
   int rc = pick_ring(ctx->cfg, stage_bytes, n_stages, &sb, &ns);
   if (rc) return rc;
   if ((rc = set_device(ctx))) return rc;
-  const size_t dyn = (size_t)sb * ns + scratch_bytes(ctx->cfg);
+  const size_t dyn = (size_t)sb * ns + kPartBytes;
   int per_sm = 0;
   SPD_CUDA(spd_internal_prepare(dyn > ctx->dyn_smem ? dyn : ctx->dyn_smem, &per_sm));
   if (per_sm < 1) return SPD_EINVAL;

@@ -79,8 +79,7 @@ __device__ __forceinline__ uint4 lds128(const void *p) {
 struct Blk {
   const KParams *p;
   uint8_t *ring;
-  float *part;       // [2][kTile][kConsumerWarps] row partials
-  uint4 *xf;         // A fragments of x; doubles as scratch of the attention phase and of the tail
+  float *part;       // [2][kTile][kConsumerWarps]
   uint64_t *full, *empty;
   float *red;        // [64] reduction scratch
   volatile int *dead;
@@ -144,121 +143,53 @@ __device__ __forceinline__ void cta_rows(int R, int gran, int &r0, int &r1) {
   r1 = (int)(U * (blockIdx.x + 1) / gridDim.x) * gran;
 }
 
-// ---------------------------------------------------------------- how a matrix is cut into ring chunks
-// A block's rows are taken in groups of 4: the 8 columns (n) of one tensor-core tile are the 4 rows
-// times the two 32-column halves of a 64-column "pair-block", so that the 8 lanes of a quarter-warp read
-// 128 contiguous bytes of shared memory (no padding, no bank conflicts) and a group of full rows is one
-// contiguous bulk copy.  Rows of up to `full` columns go through the ring whole (one chunk = one group);
-// longer rows are cut into segments of at most 2048 columns (one chunk = two groups x one segment, one
-// bulk copy per row piece) and walked tile by tile (32 rows), segment by segment, so that a warp keeps
-// one accumulator set per group of the tile and reloads its slices of x per segment.
-struct MatPlan {
-  int r0, r1;      // this block's rows
-  int C;           // columns
-  int seg_cols;    // columns per segment (multiple of 64 unless the row is a single segment)
-  int nseg;
-  int tile_rows;   // rows between two epilogues
-  uint32_t pitch;  // bytes between row pieces inside a stage
-  uint32_t rowbytes;
-};
-
-__device__ __forceinline__ MatPlan make_plan(const KParams &p, int R, int C, int gran) {
-  MatPlan m;
-  cta_rows(R, gran, m.r0, m.r1);
-  m.C = C;
-  m.rowbytes = (uint32_t)C * 2u;
-  int full = (p.stage_bytes / (kGroupRows * 2)) / 64 * 64;
-  if (full > kMaxWholeCols) full = kMaxWholeCols;
-  if (C <= full) {
-    m.seg_cols = C;
-    m.nseg = 1;
-    m.tile_rows = kTile;
-    m.pitch = m.rowbytes;
-  } else {
-    int sc = (p.stage_bytes / (2 * kGroupRows * 2)) / 64 * 64;
-    if (sc > kMaxSegCols) sc = kMaxSegCols;
-    m.seg_cols = sc;
-    m.nseg = (C + sc - 1) / sc;
-    m.tile_rows = kSegTile;
-    m.pitch = (uint32_t)sc * 2u;
-  }
-  return m;
+__device__ __forceinline__ int rows_per_chunk(const KParams &p, int C) {
+  int rpc = p.stage_bytes / (C * 2);
+  return rpc > kMaxRowsPerChunk ? kMaxRowsPerChunk : rpc;
 }
 
-// The matrices of one timestep in the order they are used: phase 4l+0..3 = layer l's QKV, O, gate/up,
-// down projections; phase 4L = the LM head.
-struct PhaseDesc {
-  const __nv_bfloat16 *W;
-  int R, C, gran;
-};
-__device__ __forceinline__ PhaseDesc phase_desc(const KParams &p, int ph) {
-  PhaseDesc d;
-  if (ph == 4 * p.L) {
-    d.W = p.lm_head; d.R = p.V; d.C = p.d; d.gran = 1;
-    return d;
-  }
-  const LayerW &lw = p.layers[ph >> 2];
-  switch (ph & 3) {
-    case 0: d.W = lw.wqkv; d.R = 3 * p.d; d.C = p.d; d.gran = 2; break;
-    case 1: d.W = lw.wo; d.R = p.d; d.C = p.d; d.gran = 1; break;
-    case 2: d.W = lw.wgate_up; d.R = 2 * p.f; d.C = p.d; d.gran = 2; break;
-    default: d.W = lw.wdown; d.R = p.d; d.C = p.f; d.gran = 1; break;
-  }
-  return d;
-}
-
-// ---------------------------------------------------------------- producer (one warp)
+// ---------------------------------------------------------------- producer
 struct Producer {
   uint32_t stage, phase;
   uint32_t issued;  // chunks issued so far (saturating at n_stages for the drain)
 };
 
-// Lane 0 waits for the stage and arms its barrier; then one bulk copy for a group of whole rows, or one
-// per row piece (lanes 0..nrows-1) for a segment.
-__device__ __forceinline__ bool produce_chunk(Blk &b, Producer &pr, const uint8_t *W, const MatPlan &m, int row0, int nrows,
-                                              int seg, int lane) {
+__device__ __forceinline__ void produce_matrix(Blk &b, Producer &pr, const __nv_bfloat16 *W, int R, int C, int gran) {
   const KParams &p = *b.p;
-  const uint32_t piece = m.nseg == 1 ? m.rowbytes : (uint32_t)min(m.seg_cols, m.C - seg * m.seg_cols) * 2u;
-  int dead = 0;
-  if (lane == 0) {
-    wait_mbar(b, &b.empty[pr.stage], pr.phase ^ 1u, 200);
-    dead = *b.dead;
-    if (!dead) mbar_expect_tx(&b.full[pr.stage], piece * (uint32_t)nrows);
-  }
-  dead = __shfl_sync(0xffffffffu, dead, 0);
-  if (dead) return false;
-  uint8_t *dst = b.ring + (size_t)pr.stage * p.stage_bytes;
-  if (m.nseg == 1) {
-    if (lane == 0) bulk_load(dst, W + (size_t)row0 * m.rowbytes, piece * (uint32_t)nrows, &b.full[pr.stage]);
-  } else if (lane < nrows) {
-    bulk_load(dst + (size_t)lane * m.pitch, W + (size_t)(row0 + lane) * m.rowbytes + (size_t)seg * m.seg_cols * 2u, piece,
-              &b.full[pr.stage]);
-  }
-  if (pr.issued < (uint32_t)p.n_stages) ++pr.issued;
-  if (++pr.stage == (uint32_t)p.n_stages) { pr.stage = 0; pr.phase ^= 1u; }
-  return true;
-}
-
-__device__ __forceinline__ void producer_main(Blk &b) {
-  const KParams &p = *b.p;
-  const int lane = threadIdx.x & 31;
-  Producer pr{0u, 0u, 0u};
-  bool ok = true;
-  for (int it = 0; it < p.n_iters && ok; ++it) {
-    const int nph = (p.mode == kModeDecode || it == p.n_iters - 1) ? 4 * p.L + 1 : 4 * p.L;
-    for (int ph = 0; ph < nph && ok; ++ph) {
-      const PhaseDesc pd = phase_desc(p, ph);
-      const MatPlan m = make_plan(p, pd.R, pd.C, pd.gran);
-      const uint8_t *W = reinterpret_cast<const uint8_t *>(pd.W);
-      const int crow = m.nseg == 1 ? kGroupRows : 2 * kGroupRows;  // rows per chunk
-      for (int t0 = m.r0; t0 < m.r1 && ok; t0 += m.tile_rows) {
-        const int t1 = min(t0 + m.tile_rows, m.r1);
-        for (int s = 0; s < m.nseg && ok; ++s)
-          for (int g0 = t0; g0 < t1 && ok; g0 += crow) ok = produce_chunk(b, pr, W, m, g0, min(crow, t1 - g0), s, lane);
-      }
+  int r0, r1;
+  cta_rows(R, gran, r0, r1);
+  const int rpc = rows_per_chunk(p, C);
+  const uint32_t rowbytes = (uint32_t)C * 2u;
+  for (int t0 = r0; t0 < r1; t0 += kTile) {
+    const int t1 = min(t0 + kTile, r1);
+    for (int r = t0; r < t1; r += rpc) {
+      const int n = min(rpc, t1 - r);
+      wait_mbar(b, &b.empty[pr.stage], pr.phase ^ 1u, 200);
+      if (*b.dead) return;
+      const uint32_t bytes = (uint32_t)n * rowbytes;
+      mbar_expect_tx(&b.full[pr.stage], bytes);
+      bulk_load(b.ring + (size_t)pr.stage * p.stage_bytes, (const uint8_t *)W + (size_t)r * rowbytes, bytes,
+                &b.full[pr.stage]);
+      if (pr.issued < (uint32_t)p.n_stages) ++pr.issued;
+      if (++pr.stage == (uint32_t)p.n_stages) { pr.stage = 0; pr.phase ^= 1u; }
     }
   }
-  if (!ok && lane == 0) {
+}
+
+__device__ void producer_main(Blk &b) {
+  const KParams &p = *b.p;
+  Producer pr{0u, 0u, 0u};
+  for (int it = 0; it < p.n_iters && !*b.dead; ++it) {
+    for (int l = 0; l < p.L && !*b.dead; ++l) {
+      const LayerW lw = p.layers[l];
+      produce_matrix(b, pr, lw.wqkv, 3 * p.d, p.d, 2);
+      produce_matrix(b, pr, lw.wo, p.d, p.d, 1);
+      produce_matrix(b, pr, lw.wgate_up, 2 * p.f, p.d, 2);
+      produce_matrix(b, pr, lw.wdown, p.d, p.f, 1);
+    }
+    if (p.mode == kModeDecode || it == p.n_iters - 1) produce_matrix(b, pr, p.lm_head, p.V, p.d, 1);
+  }
+  if (*b.dead) {
     // Giving up: nothing more is issued; wait (bounded) until every copy already issued has landed,
     // so that no copy writes into shared memory after the block has gone.
     uint32_t s = pr.stage, ph = pr.phase;
@@ -269,95 +200,103 @@ __device__ __forceinline__ void producer_main(Blk &b) {
       while (!mbar_try_wait(&b.full[s], ph) && globaltimer() - t0 < kWaitNs) {}
     }
   }
-  __syncwarp();
 }
 
-// ---------------------------------------------------------------- consumer: tensor-core row products
-// y[r] = sum_c W[r][c] x[c] for the 4 rows of a group is computed as D = A * B on mma.sync m16n8k16 (bf16 in,
-// float32 accumulate).  B column n = 2r + h holds row r's weights of half h of each 64-column pair-block;
-// A rows 0..2 hold the three bf16 terms of x (x = hi + mid + lo exactly to float32 precision) for half 0,
-// rows 8..10 the same for half 1.  A lane's 16-byte shared-memory load (8 consecutive weights of its
-// row and half) feeds two multiplies; which k index a column lands on is free as long as A agrees, so no
-// ldmatrix shuffle is needed.  The tensor core is used only because it multiplies 256 weights per
-// instruction where the plain path needs 17 instructions per 8 weights; the work stays HBM-bound.
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t a0, const uint32_t a1, const uint32_t a2,
-                                         const uint32_t a3, const uint32_t b0, const uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+// ---------------------------------------------------------------- consumer: row dot products
+__device__ __forceinline__ float dot8(const uint4 w, const float (&x)[8], float acc) {
+  acc = fmaf(__uint_as_float(w.x << 16), x[0], acc);
+  acc = fmaf(__uint_as_float(w.x & 0xffff0000u), x[1], acc);
+  acc = fmaf(__uint_as_float(w.y << 16), x[2], acc);
+  acc = fmaf(__uint_as_float(w.y & 0xffff0000u), x[3], acc);
+  acc = fmaf(__uint_as_float(w.z << 16), x[4], acc);
+  acc = fmaf(__uint_as_float(w.z & 0xffff0000u), x[5], acc);
+  acc = fmaf(__uint_as_float(w.w << 16), x[6], acc);
+  acc = fmaf(__uint_as_float(w.w & 0xffff0000u), x[7], acc);
+  return acc;
 }
 
-__device__ __forceinline__ uint32_t bf16_bits(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v)); }
-// term `part` (0 hi, 1 mid, 2 lo) of the exact three-way bf16 split of v
-__device__ __forceinline__ uint32_t split_term(float v, int part) {
-  const uint32_t h = bf16_bits(v);
-  if (part == 0) return h;
-  float r = v - __uint_as_float(h << 16);
-  const uint32_t m = bf16_bits(r);
-  if (part == 1) return m;
-  r -= __uint_as_float(m << 16);
-  return bf16_bits(r);
-}
-
-// Fragment store: for pair-block P, A-lane l = term * 4 + q (l < 12), eight 32-bit words
-//   [0] half 0 cols (8q+0, 8q+1)   [1] half 1 same   [2] half 0 cols (8q+2, 8q+3)   [3] half 1 same    (first multiply)
-//   [4] half 0 cols (8q+4, 8q+5)   [5] half 1 same   [6] half 0 cols (8q+6, 8q+7)   [7] half 1 same    (second multiply)
-// i.e. exactly the a0..a3 registers of the two multiplies that consume one 16-byte weight load.
-__device__ __forceinline__ void load_frag(const uint4 *frag, int P, int lane, uint32_t (&a)[8]) {
-  if (lane < 12) {
-    const uint4 lo = frag[(size_t)(P * 12 + lane) * 2], hi = frag[(size_t)(P * 12 + lane) * 2 + 1];
-    a[0] = lo.x; a[1] = lo.y; a[2] = lo.z; a[3] = lo.w;
-    a[4] = hi.x; a[5] = hi.y; a[6] = hi.z; a[7] = hi.w;
+// Sums NR per-lane accumulators over the warp with a folding butterfly.  Afterwards lane
+// r * (32 / NR) holds the total of accumulator r.
+template <int NR>
+__device__ __forceinline__ float warp_fold(float (&a)[NR], int lane) {
+  if constexpr (NR == 8) {
+    float b4[4];
+    const bool up = lane & 16;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float send = up ? a[i] : a[i + 4];
+      const float keep = up ? a[i + 4] : a[i];
+      b4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+    float b2[2];
+    const bool up2 = lane & 8;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float send = up2 ? b4[i] : b4[i + 2];
+      const float keep = up2 ? b4[i + 2] : b4[i];
+      b2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+    const bool up3 = lane & 4;
+    float v = (up3 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up3 ? b2[0] : b2[1], 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
+  } else if constexpr (NR == 4) {
+    float b2[2];
+    const bool up = lane & 16;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float send = up ? a[i] : a[i + 2];
+      const float keep = up ? a[i + 2] : a[i];
+      b2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+    const bool up2 = lane & 8;
+    float v = (up2 ? b2[1] : b2[0]) + __shfl_xor_sync(0xffffffffu, up2 ? b2[0] : b2[1], 8);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
+  } else if constexpr (NR == 2) {
+    const bool up = lane & 16;
+    float v = (up ? a[1] : a[0]) + __shfl_xor_sync(0xffffffffu, up ? a[0] : a[1], 16);
+    v += __shfl_xor_sync(0xffffffffu, v, 8);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
   } else {
+    float v = a[0];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) a[e] = 0u;
-  }
-}
-__device__ __forceinline__ void load_frag_global(const uint4 *frag, int P, int lane, uint32_t (&a)[8]) {
-  if (lane < 12) {
-    const uint4 lo = __ldcg(frag + (size_t)(P * 12 + lane) * 2), hi = __ldcg(frag + (size_t)(P * 12 + lane) * 2 + 1);
-    a[0] = lo.x; a[1] = lo.y; a[2] = lo.z; a[3] = lo.w;
-    a[4] = hi.x; a[5] = hi.y; a[6] = hi.z; a[7] = hi.w;
-  } else {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) a[e] = 0u;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
   }
 }
 
-// Thread `v` holds columns [8v, 8v+8) of x (zeros past the end of the row): writes their three bf16
-// terms into the fragment store.
-__device__ __forceinline__ void write_frags(uint32_t *frag, int v, const float (&x)[8]) {
-  const int P = v >> 3, h = (v >> 2) & 1, q = v & 3;
-  uint32_t t[3][8];
+// One chunk of n (<= NR) rows in a ring stage: every thread multiplies its column vectors, the warp
+// folds, and the warp's partial of row j goes to part[(trow + j) * warps + warp].
+template <int NR>
+__device__ __forceinline__ void consume_chunk(const uint8_t *stage, int n, int rowbytes, int nv,
+                                              const float (&xr)[kMaxVec][8], float *part_rows, int warp, int lane) {
+  float acc[NR];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    t[0][e] = bf16_bits(x[e]);
-    float r = x[e] - __uint_as_float(t[0][e] << 16);
-    t[1][e] = bf16_bits(r);
-    r -= __uint_as_float(t[1][e] << 16);
-    t[2][e] = bf16_bits(r);
+  for (int r = 0; r < NR; ++r) acc[r] = 0.f;
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) {
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {
+        if (r < n) {
+          const uint4 w = lds128(stage + (size_t)r * rowbytes + (size_t)v * 16);
+          acc[r] = dot8(w, xr[i], acc[r]);
+        }
+      }
+    }
   }
-#pragma unroll
-  for (int k = 0; k < 3; ++k) {
-    uint32_t *w = frag + (size_t)((P * 12 + k * 4 + q) * 8) + h;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) w[2 * e] = t[k][2 * e] | (t[k][2 * e + 1] << 16);
-  }
-}
-
-// This lane's 16 bytes of weights for pair-block column offset `pcol` (columns from the start of the
-// row piece) of group row r, half h; zeros past the end of the row.
-__device__ __forceinline__ uint4 load_b(uint32_t row_addr, int pcol, int cols_left) {
-  uint4 w = make_uint4(0u, 0u, 0u, 0u);
-  if (pcol < cols_left) asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w) : "r"(row_addr + (uint32_t)pcol * 2u));
-  return w;
-}
-
-// Adds the split rows of both halves and leaves the warp's partial sums of the group's rows in part[].
-__device__ __forceinline__ void group_finish(float v, float *part_rows, int nrows, int warp, int lane) {
-  const float t1 = __shfl_down_sync(0xffffffffu, v, 4), t2 = __shfl_down_sync(0xffffffffu, v, 8);
-  v += t1 + t2;
-  if (lane < 4 && lane < nrows) part_rows[lane * kPartStride + warp] = v;
+  const float v = warp_fold<NR>(acc, lane);
+  constexpr int kStride = 32 / NR;
+  const int j = lane / kStride;
+  if ((lane % kStride) == 0 && j < n) part_rows[j * kConsumerWarps + warp] = v;
 }
 
 enum Epi { kEpiQKV = 0, kEpiAddH = 1, kEpiSwiGLU = 2, kEpiLogits = 3 };
@@ -367,9 +306,16 @@ struct EpiArgs {
 };
 
 __device__ __forceinline__ float part_sum(const float *row) {
+  const float4 *q = reinterpret_cast<const float4 *>(row);
   float s = 0.f;
 #pragma unroll
-  for (int i = 0; i < kConsumerWarps; ++i) s += row[i];
+  for (int i = 0; i < kConsumerWarps / 4; ++i) {
+    const float4 a = q[i];
+    s += a.x;
+    s += a.y;
+    s += a.z;
+    s += a.w;
+  }
   return s;
 }
 
@@ -387,8 +333,8 @@ __device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, co
     // rows come in pairs (2i, 2i+1) of one head: rotate q and k, append k and v to the cache
     if (tid * 2 < rows) {
       const int r = t0 + tid * 2;
-      float a = part_sum(part + (size_t)(tid * 2) * kPartStride);
-      float c = part_sum(part + (size_t)(tid * 2 + 1) * kPartStride);
+      float a = part_sum(part + (size_t)(tid * 2) * kConsumerWarps);
+      float c = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps);
       const int sec = r / p.d, col = r - sec * p.d;
       if (sec < 2) {
         const float2 cs = p.rope[(size_t)ea.pos * (p.hd / 2) + (col % p.hd) / 2];
@@ -411,181 +357,50 @@ __device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, co
   } else if (kind == kEpiAddH) {
     if (tid < rows) {
       const int r = t0 + tid;
-      const float y = __ldcg(p.h + r) + part_sum(part + (size_t)tid * kPartStride);
+      const float y = __ldcg(p.h + r) + part_sum(part + (size_t)tid * kConsumerWarps);
       p.h[r] = y;
       if (p.trace) p.trace[((size_t)ea.layer * 2 + ea.which) * p.d + r] = y;
     }
   } else if (kind == kEpiSwiGLU) {
     if (tid * 2 < rows) {
-      const float g = part_sum(part + (size_t)(tid * 2) * kPartStride);
-      const float up = part_sum(part + (size_t)(tid * 2 + 1) * kPartStride);
-      const float u = g / (1.f + __expf(-g)) * up;
-      // stored as the three bf16 terms, at the place the down projection's A fragments are read from
-      const int j = (t0 >> 1) + tid;
-      const int P = j >> 6, h = (j >> 5) & 1, q = (j >> 3) & 3, e = j & 7;
-#pragma unroll
-      for (int t = 0; t < 3; ++t)
-        p.ufrag[((size_t)((P * 12 + t * 4 + q) * 8) + (e >> 1) * 2 + h) * 2 + (e & 1)] = (unsigned short)split_term(u, t);
+      const float g = part_sum(part + (size_t)(tid * 2) * kConsumerWarps);
+      const float up = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps);
+      p.u[(t0 >> 1) + tid] = g / (1.f + __expf(-g)) * up;
     }
   } else {
-    if (tid < rows) p.logits[t0 + tid] = part_sum(part + (size_t)tid * kPartStride);
+    if (tid < rows) p.logits[t0 + tid] = part_sum(part + (size_t)tid * kConsumerWarps);
   }
 }
 
-// Asynchronous copy of this warp's fragments of segment `seg` from global memory into its private buffer
-// (entry j of the buffer = the warp's j-th pair-block of the segment).
-__device__ __forceinline__ void prefetch_frags(const uint4 *gfrag, uint4 *dst, int seg, int pb_seg, int seg_cols, int C, int warp,
-                                               int lane) {
-  if (lane < 12) {
-#pragma unroll
-    for (int j = 0; j < kSegPB; ++j) {
-      const int Pl = warp + kConsumerWarps * j;
-      if (Pl < pb_seg && seg * seg_cols + Pl * 64 < C) {
-        const uint4 *src = gfrag + (size_t)((seg * pb_seg + Pl) * 12 + lane) * 2;
-        const uint32_t d = smem_u32(dst + (size_t)(j * 12 + lane) * 2);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d + 16u), "l"(src + 1) : "memory");
-      }
-    }
-  }
-}
-
-enum XSrc { kXSmem = 0, kXGlobal = 1 };  // A fragments in the block's shared memory / in global memory (FFN activation)
-
-__device__ __forceinline__ void stage_done(Blk &b, int lane) {
-  __syncwarp();
-  if (lane == 0) mbar_arrive(&b.empty[b.c_stage]);
-  if (++b.c_stage == (uint32_t)b.p->n_stages) { b.c_stage = 0; b.c_phase ^= 1u; }
-}
-
-// Streams this block's rows of one matrix through the ring.
-__device__ __forceinline__ void consume_matrix(Blk &b, int R, int C, int gran, int xsrc, int kind, const EpiArgs &ea) {
+// Streams this block's rows of one matrix through the ring against the register-resident x.
+__device__ __forceinline__ void consume_matrix(Blk &b, int R, int C, int gran, const float (&xr)[kMaxVec][8], int kind,
+                                               const EpiArgs &ea) {
   const KParams &p = *b.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r_in_group = lane >> 3, h = (lane >> 2) & 1, q = lane & 3;
-  const int lane_col = h * 32 + q * 8;  // this lane's column inside a pair-block
-  const MatPlan m = make_plan(p, R, C, gran);
-  const uint4 *gfrag = reinterpret_cast<const uint4 *>(p.ufrag);
+  int r0, r1;
+  cta_rows(R, gran, r0, r1);
+  const int rpc = rows_per_chunk(p, C);
+  const int rowbytes = C * 2, nv = C / 8;
   int buf = 0;
-  if (m.nseg == 1) {
-    // whole rows: the warp's slices of x stay in registers for the phase
-    uint32_t xa[kMaxPB][8];
-#pragma unroll
-    for (int j = 0; j < kMaxPB; ++j) {
-      const int P = warp + kConsumerWarps * j;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) xa[j][e] = 0u;
-      if (P * 64 < C) {
-        if (xsrc == kXSmem) load_frag(b.xf, P, lane, xa[j]);
-        else load_frag_global(gfrag, P, lane, xa[j]);
-      }
+  for (int t0 = r0; t0 < r1; t0 += kTile) {
+    const int t1 = min(t0 + kTile, r1);
+    float *part = b.part + (size_t)buf * kTile * kConsumerWarps;
+    for (int r = t0; r < t1; r += rpc) {
+      const int n = min(rpc, t1 - r);
+      wait_mbar(b, &b.full[b.c_stage], b.c_phase, 300);
+      const uint8_t *stage = b.ring + (size_t)b.c_stage * p.stage_bytes;
+      float *prow = part + (size_t)(r - t0) * kConsumerWarps;
+      if (n > 4) consume_chunk<8>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      else if (n > 2) consume_chunk<4>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      else if (n > 1) consume_chunk<2>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      else consume_chunk<1>(stage, n, rowbytes, nv, xr, prow, warp, lane);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&b.empty[b.c_stage]);
+      if (++b.c_stage == (uint32_t)p.n_stages) { b.c_stage = 0; b.c_phase ^= 1u; }
     }
-    for (int t0 = m.r0; t0 < m.r1; t0 += m.tile_rows) {
-      const int t1 = min(t0 + m.tile_rows, m.r1);
-      float *part = b.part + (size_t)buf * kTile * kPartStride;
-      for (int g0 = t0; g0 < t1; g0 += kGroupRows) {
-        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f}, d2[4] = {0.f, 0.f, 0.f, 0.f}, d3[4] = {0.f, 0.f, 0.f, 0.f};
-        wait_mbar(b, &b.full[b.c_stage], b.c_phase, 300);
-        const uint32_t row_addr = smem_u32(b.ring + (size_t)b.c_stage * p.stage_bytes) + (uint32_t)r_in_group * m.pitch;
-#pragma unroll
-        for (int j0 = 0; j0 < kMaxPB; j0 += 5) {
-          uint4 w[5];
-#pragma unroll
-          for (int j = 0; j < 5; ++j) {
-            const int pc = (warp + kConsumerWarps * (j0 + j)) * 64;
-            if (pc < C) w[j] = load_b(row_addr, pc + lane_col, C);  // warp-uniform condition
-          }
-#pragma unroll
-          for (int j = 0; j < 5; ++j) {
-            const int pc = (warp + kConsumerWarps * (j0 + j)) * 64;
-            if (pc < C) {
-              if (j & 1) {
-                mma_bf16(d2, xa[j0 + j][0], xa[j0 + j][1], xa[j0 + j][2], xa[j0 + j][3], w[j].x, w[j].y);
-                mma_bf16(d3, xa[j0 + j][4], xa[j0 + j][5], xa[j0 + j][6], xa[j0 + j][7], w[j].z, w[j].w);
-              } else {
-                mma_bf16(d0, xa[j0 + j][0], xa[j0 + j][1], xa[j0 + j][2], xa[j0 + j][3], w[j].x, w[j].y);
-                mma_bf16(d1, xa[j0 + j][4], xa[j0 + j][5], xa[j0 + j][6], xa[j0 + j][7], w[j].z, w[j].w);
-              }
-            }
-          }
-        }
-        stage_done(b, lane);
-        group_finish((d0[0] + d1[0]) + (d2[0] + d3[0]) + ((d0[3] + d1[3]) + (d2[3] + d3[3])), part + (size_t)(g0 - t0) * kPartStride, min(kGroupRows, t1 - g0), warp, lane);
-      }
-      named_sync(1, kConsumerThreads);
-      epilogue(b, kind, ea, part, t0, t1);
-      buf ^= 1;
-    }
-  } else {
-    // long rows: per tile of 32 rows, segment by segment.  When x comes from global memory each warp
-    // copies its slices of the next segment into a private shared-memory buffer (cp.async, no registers
-    // held) while the current segment is multiplied; the fragment area is free for that in such phases.
-    const int pb_seg = m.seg_cols / 64;
-    uint4 *pre = b.xf + (size_t)warp * (kSegPB * 12 * 2);  // [2 buffers][warps][kSegPB][12 lanes][2]
-    constexpr int kPreBuf = kConsumerWarps * kSegPB * 12 * 2;
-    for (int t0 = m.r0; t0 < m.r1; t0 += m.tile_rows) {
-      const int t1 = min(t0 + m.tile_rows, m.r1);
-      float *part = b.part + (size_t)buf * kTile * kPartStride;
-      float acc[kSegTile / kGroupRows][4];
-#pragma unroll
-      for (int g = 0; g < kSegTile / kGroupRows; ++g) acc[g][0] = acc[g][1] = acc[g][2] = acc[g][3] = 0.f;
-      if (xsrc == kXGlobal) prefetch_frags(gfrag, pre, 0, pb_seg, m.seg_cols, C, warp, lane);
-      for (int s = 0; s < m.nseg; ++s) {
-        const int seg_len = min(m.seg_cols, C - s * m.seg_cols);
-        uint32_t xa[kSegPB][8];
-        if (xsrc == kXGlobal) {
-          asm volatile("cp.async.wait_all;" ::: "memory");
-          __syncwarp();
-        }
-#pragma unroll
-        for (int j = 0; j < kSegPB; ++j) {
-          const int Pl = warp + kConsumerWarps * j;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) xa[j][e] = 0u;
-          if (Pl < pb_seg && s * m.seg_cols + Pl * 64 < C) {
-            if (xsrc == kXSmem) load_frag(b.xf, s * pb_seg + Pl, lane, xa[j]);
-            else load_frag(pre + (size_t)(s & 1) * kPreBuf, j, lane, xa[j]);
-          }
-        }
-        if (xsrc == kXGlobal && s + 1 < m.nseg)
-          prefetch_frags(gfrag, pre + (size_t)((s + 1) & 1) * kPreBuf, s + 1, pb_seg, m.seg_cols, C, warp, lane);
-#pragma unroll
-        for (int c = 0; c < kSegTile / (2 * kGroupRows); ++c) {
-          if (t0 + c * 2 * kGroupRows < t1) {
-            wait_mbar(b, &b.full[b.c_stage], b.c_phase, 300);
-            const uint32_t base = smem_u32(b.ring + (size_t)b.c_stage * p.stage_bytes) + (uint32_t)r_in_group * m.pitch;
-#pragma unroll
-            for (int gg = 0; gg < 2; ++gg) {
-              if (t0 + (2 * c + gg) * kGroupRows < t1) {
-                uint4 w[kSegPB];
-#pragma unroll
-                for (int j = 0; j < kSegPB; ++j) {
-                  const int pc = (warp + kConsumerWarps * j) * 64;
-                  if (pc < seg_len) w[j] = load_b(base + (uint32_t)(gg * kGroupRows) * m.pitch, pc + lane_col, seg_len);
-                }
-#pragma unroll
-                for (int j = 0; j < kSegPB; ++j) {
-                  const int pc = (warp + kConsumerWarps * j) * 64;
-                  if (pc < seg_len) {
-                    mma_bf16(acc[2 * c + gg], xa[j][0], xa[j][1], xa[j][2], xa[j][3], w[j].x, w[j].y);
-                    mma_bf16(acc[2 * c + gg], xa[j][4], xa[j][5], xa[j][6], xa[j][7], w[j].z, w[j].w);
-                  }
-                }
-              }
-            }
-            stage_done(b, lane);
-          }
-        }
-      }
-#pragma unroll
-      for (int g = 0; g < kSegTile / kGroupRows; ++g)
-        if (t0 + g * kGroupRows < t1)
-          group_finish(acc[g][0] + acc[g][3], part + (size_t)(g * kGroupRows) * kPartStride, min(kGroupRows, t1 - t0 - g * kGroupRows),
-                       warp, lane);
-      named_sync(1, kConsumerThreads);
-      epilogue(b, kind, ea, part, t0, t1);
-      buf ^= 1;
-    }
+    named_sync(1, kConsumerThreads);
+    epilogue(b, kind, ea, part, t0, t1);
+    buf ^= 1;
   }
 }
 
@@ -610,24 +425,18 @@ __device__ __forceinline__ void load8(const float *src, float (&x)[8]) {
   x[4] = c.x; x[5] = c.y; x[6] = c.z; x[7] = c.w;
 }
 
-// x = RMSNorm(h) * gain, left as A fragments in the block's shared memory (pair-blocks past the end of
-// the row are zero-filled)
-__device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const __nv_bfloat16 *gain, int C) {
-  const int nv = C / 8, nv_pad = (C + 63) / 64 * 8;
-  float xv[kMaxVec][8];
-  uint4 gv[kMaxVec];
+// x = RMSNorm(h) * gain, each thread keeping its own column vectors
+__device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const __nv_bfloat16 *gain, int C,
+                                              float (&xr)[kMaxVec][8]) {
+  const int nv = C / 8;
   float ss = 0.f;
 #pragma unroll
   for (int i = 0; i < kMaxVec; ++i) {
     const int v = (int)threadIdx.x + i * kConsumerThreads;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) xv[i][e] = 0.f;
-    gv[i] = make_uint4(0u, 0u, 0u, 0u);
     if (v < nv) {
-      load8(h + (size_t)v * 8, xv[i]);
-      gv[i] = *reinterpret_cast<const uint4 *>(gain + (size_t)v * 8);
+      load8(h + (size_t)v * 8, xr[i]);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) ss = fmaf(xv[i][e], xv[i][e], ss);
+      for (int e = 0; e < 8; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
     }
   }
   ss = block_sum(b, ss);
@@ -635,59 +444,61 @@ __device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const __nv
 #pragma unroll
   for (int i = 0; i < kMaxVec; ++i) {
     const int v = (int)threadIdx.x + i * kConsumerThreads;
-    if (v < nv_pad) {
-      const uint32_t gw[4] = {gv[i].x, gv[i].y, gv[i].z, gv[i].w};
+    if (v < nv) {
+      const uint4 g = *reinterpret_cast<const uint4 *>(gain + (size_t)v * 8);
+      const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        xv[i][2 * e] = xv[i][2 * e] * rs * __uint_as_float(gw[e] << 16);
-        xv[i][2 * e + 1] = xv[i][2 * e + 1] * rs * __uint_as_float(gw[e] & 0xffff0000u);
+        xr[i][2 * e] = xr[i][2 * e] * rs * __uint_as_float(gw[e] << 16);
+        xr[i][2 * e + 1] = xr[i][2 * e + 1] * rs * __uint_as_float(gw[e] & 0xffff0000u);
       }
-      write_frags(reinterpret_cast<uint32_t *>(b.xf), v, xv[i]);
     }
   }
-  named_sync(1, kConsumerThreads);
+}
+
+__device__ __forceinline__ void prologue_plain(const float *src, int C, float (&xr)[kMaxVec][8]) {
+  const int nv = C / 8;
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) load8(src + (size_t)v * 8, xr[i]);
+  }
 }
 
 __device__ __forceinline__ int attn_splits(const KParams &p, int T) {
   int ms = (int)gridDim.x / p.H;
   ms = ms < 1 ? 1 : (ms > kMaxSplit ? kMaxSplit : ms);
-  int ns = (T + 7) / 8;  // short contexts are still spread over all blocks: the phase is latency-bound
+  int ns = (T + 63) / 64;
   return ns < 1 ? 1 : (ns > ms ? ms : ns);
 }
 
-// x = attention output (the per-split partial sums of each head merged), left as A fragments
-__device__ __forceinline__ void prologue_attn(Blk &b, int T) {
-  const KParams &p = *b.p;
-  const int nv = p.d / 8, nv_pad = (p.d + 63) / 64 * 8, ns = attn_splits(p, T);
+// x = attention output: merges the per-split partial sums of each head
+__device__ __forceinline__ void prologue_attn(const KParams &p, int T, float (&xr)[kMaxVec][8]) {
+  const int nv = p.d / 8, ns = attn_splits(p, T);
 #pragma unroll
   for (int i = 0; i < kMaxVec; ++i) {
     const int v = (int)threadIdx.x + i * kConsumerThreads;
-    if (v < nv_pad) {
-      float acc[8];
+    if (v < nv) {
+      const int col = v * 8, head = col / p.hd, c = col - head * p.hd;
+      float M = -CUDART_INF_F;
+      for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&p.oml[head * ns + s]).x);
+      float den = 0.f, acc[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-      if (v < nv) {
-        const int col = v * 8, head = col / p.hd, c = col - head * p.hd;
-        float M = -CUDART_INF_F;
-        for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&p.oml[head * ns + s]).x);
-        float den = 0.f;
-        for (int s = 0; s < ns; ++s) {
-          const float2 ml = __ldcg(&p.oml[head * ns + s]);
-          const float w = __expf(ml.x - M);
-          den = fmaf(ml.y, w, den);
-          float o[8];
-          load8(p.opart + (size_t)(head * ns + s) * p.hd + c, o);
+      for (int s = 0; s < ns; ++s) {
+        const float2 ml = __ldcg(&p.oml[head * ns + s]);
+        const float w = __expf(ml.x - M);
+        den = fmaf(ml.y, w, den);
+        float o[8];
+        load8(p.opart + (size_t)(head * ns + s) * p.hd + c, o);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[e] = fmaf(o[e], w, acc[e]);
-        }
-        const float inv = 1.f / den;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] *= inv;
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(o[e], w, acc[e]);
       }
-      write_frags(reinterpret_cast<uint32_t *>(b.xf), v, acc);
+      const float inv = 1.f / den;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xr[i][e] = acc[e] * inv;
     }
   }
-  named_sync(1, kConsumerThreads);
 }
 
 // ---------------------------------------------------------------- attention over the shared cache
@@ -699,14 +510,14 @@ __device__ __forceinline__ float load_kv(const KParams &p, const void *cache, si
   return __ldcg(reinterpret_cast<const float *>(cache) + idx);
 }
 
-__device__ __forceinline__ void attention_phase(Blk &b, int layer, int pos) {
+__device__ void attention_phase(Blk &b, int layer, int pos) {
   const KParams &p = *b.p;
   const int T = pos + 1, ns = attn_splits(p, T), items = p.H * ns;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int epl = p.hd / 32;  // elements per lane, <= 8
   const float scale = 1.f / sqrtf((float)p.hd);
-  float *s_acc = reinterpret_cast<float *>(b.xf);  // [warps][256]
-  float *s_m = s_acc + kConsumerWarps * 256;       // [warps]
+  float *s_acc = b.part;                           // [warps][hd]
+  float *s_m = b.part + kConsumerWarps * 256;      // [warps]
   float *s_l = s_m + kConsumerWarps;               // [warps]
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int head = item / ns, sp = item - head * ns;
@@ -718,36 +529,27 @@ __device__ __forceinline__ void attention_phase(Blk &b, int layer, int pos) {
       acc[e] = 0.f;
     }
     float m = -CUDART_INF_F, l = 0.f;
-    // four positions per round: their loads are independent and go out together
-    for (int tb = t0 + warp * 4; tb < t1; tb += kConsumerWarps * 4) {
-      float kk[4][8], vv[4][8];
+    for (int t = t0 + warp; t < t1; t += kConsumerWarps) {
+      const size_t base = ((size_t)layer * p.max_pos + t) * p.d + head * p.hd + lane * epl;
+      float dot = 0.f, vv[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int t = min(tb + u, t1 - 1);
-        const size_t base = ((size_t)layer * p.max_pos + t) * p.d + head * p.hd + lane * epl;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          kk[u][e] = e < epl ? load_kv(p, p.kcache, base + e) : 0.f;
-          vv[u][e] = e < epl ? load_kv(p, p.vcache, base + e) : 0.f;
+      for (int e = 0; e < 8; ++e) {
+        if (e < epl) {
+          dot = fmaf(q[e], load_kv(p, p.kcache, base + e), dot);
+          vv[e] = load_kv(p, p.vcache, base + e);
+        } else {
+          vv[e] = 0.f;
         }
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (tb + u < t1) {  // warp-uniform
-          float dot = 0.f;
+      for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      const float s = dot * scale;
+      const float mn = fmaxf(m, s);
+      const float c = __expf(m - mn), pw = __expf(s - mn);
+      l = l * c + pw;
 #pragma unroll
-          for (int e = 0; e < 8; ++e) dot = fmaf(q[e], kk[u][e], dot);
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          const float s = dot * scale;
-          const float mn = fmaxf(m, s);
-          const float c = __expf(m - mn), pw = __expf(s - mn);
-          l = l * c + pw;
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[e] = acc[e] * c + pw * vv[u][e];
-          m = mn;
-        }
-      }
+      for (int e = 0; e < 8; ++e) acc[e] = acc[e] * c + pw * vv[e];
+      m = mn;
     }
 #pragma unroll
     for (int e = 0; e < 8; ++e)
@@ -757,7 +559,7 @@ __device__ __forceinline__ void attention_phase(Blk &b, int layer, int pos) {
       s_l[warp] = l;
     }
     named_sync(1, kConsumerThreads);
-    for (int dim = threadIdx.x; dim < p.hd; dim += kConsumerThreads) {
+    if ((int)threadIdx.x < p.hd) {
       float M = -CUDART_INF_F;
 #pragma unroll
       for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, s_m[w]);
@@ -766,10 +568,10 @@ __device__ __forceinline__ void attention_phase(Blk &b, int layer, int pos) {
       for (int w = 0; w < kConsumerWarps; ++w) {
         const float wgt = s_m[w] == -CUDART_INF_F ? 0.f : __expf(s_m[w] - M);
         L = fmaf(s_l[w], wgt, L);
-        A = fmaf(s_acc[w * 256 + dim], wgt, A);
+        A = fmaf(s_acc[w * 256 + threadIdx.x], wgt, A);
       }
-      p.opart[(size_t)item * p.hd + dim] = A;
-      if (dim == 0) p.oml[item] = make_float2(M, L);
+      p.opart[(size_t)item * p.hd + threadIdx.x] = A;
+      if (threadIdx.x == 0) p.oml[item] = make_float2(M, L);
     }
     named_sync(1, kConsumerThreads);
   }
@@ -789,7 +591,7 @@ __device__ __forceinline__ void warp_best(float &v, int &i) {
 }
 
 // Warp 0 of each block: the k best logits among rows [r0, r1) and (max, sum exp) of z / tau over them.
-__device__ __forceinline__ void block_topk(const KParams &p, int r0, int r1) {
+__device__ void block_topk(const KParams &p, int r0, int r1) {
   const int lane = threadIdx.x & 31;
   float pv = 0.f;
   int pi = -1;
@@ -827,7 +629,7 @@ __device__ __forceinline__ void block_topk(const KParams &p, int r0, int r1) {
 }
 
 // ---------------------------------------------------------------- the method's tail (block 0)
-__device__ __forceinline__ int probe(State *st, volatile int *dead, const SpdSlot *tab, uint64_t mask, uint32_t w0, uint32_t w1, uint32_t w2) {
+__device__ __forceinline__ int probe(Blk &b, const SpdSlot *tab, uint64_t mask, uint32_t w0, uint32_t w1, uint32_t w2) {
   uint64_t idx = spd_key_hash(w0, w1, w2) & mask;
   const uint64_t limit = mask + 1 < 16384 ? mask + 1 : 16384;
   for (uint64_t i = 0; i < limit; ++i) {
@@ -836,18 +638,13 @@ __device__ __forceinline__ int probe(State *st, volatile int *dead, const SpdSlo
     if (s.x == w0 && s.y == w1 && s.z == w2) return (int)s.w;
     idx = (idx + 1) & mask;
   }
-  if (mask + 1 > limit) {
-    if (atomicCAS(&st->err, 0, kErrTable) == 0) st->err_info = 400;
-    atomicExch(&st->abort_flag, 1u);
-    *dead = 1;
-  }
+  if (mask + 1 > limit) give_up(b, kErrTable, 400);
   return 0;
 }
 
 // KeepTopK over the whole vocabulary from the blocks' partial lists (Algorithm 1), with
 // log-probabilities under temperature tau.  Warp 0.
-__device__ __noinline__ void tail_keep_topk(const KParams *pp) {
-  const KParams &p = *pp;
+__device__ void tail_keep_topk(const KParams &p) {
   const int lane = threadIdx.x & 31;
   State *st = p.st;
   const int ncand = (int)gridDim.x * p.k;
@@ -889,13 +686,11 @@ __device__ __noinline__ void tail_keep_topk(const KParams *pp) {
 
 // Scores the k*k options, keeps the k best, updates the draft state.  `first` = first timestep: draft i
 // simply takes kept token i (Eq. 1).  All consumer threads of block 0.
-// Kept out of line (it runs once per timestep on one block) so that its registers do not weigh on the
-// streaming loops; everything it needs comes by value or through the parameter block.
-__device__ __noinline__ void tail_score_select(const KParams *pp, uint4 *scratch, volatile int *dead, bool first, int step) {
-  const KParams &p = *pp;
+__device__ void tail_score_select(Blk &b, bool first, int step) {
+  const KParams &p = *b.p;
   State *st = p.st;
   const int tid = threadIdx.x, k = p.k, nt = p.n_tables;
-  int *s_cnt = reinterpret_cast<int *>(scratch);          // [k*k][8]
+  int *s_cnt = reinterpret_cast<int *>(b.part);           // [k*k][8]
   int *s_tot = s_cnt + kMaxK * kMaxK * kMaxTables;         // [k][8]
   float *s_png = reinterpret_cast<float *>(s_tot + kMaxK * kMaxTables);  // [k*k]
   float *s_score = s_png + kMaxK * kMaxK;                  // [k*k]
@@ -944,36 +739,36 @@ __device__ __noinline__ void tail_score_select(const KParams *pp, uint4 *scratch
         if (j >= 0) key[len++] = st->cand_tok[j];
         uint32_t w0, w1, w2;
         spd_pack_key(key, len, w0, w1, w2);
-        res = j >= 0 ? probe(st, dead, tb.ngram, tb.ngram_mask, w0, w1, w2) : probe(st, dead, tb.ctx, tb.ctx_mask, w0, w1, w2);
+        res = j >= 0 ? probe(b, tb.ngram, tb.ngram_mask, w0, w1, w2) : probe(b, tb.ctx, tb.ctx_mask, w0, w1, w2);
       }
       if (j >= 0) s_cnt[(i * k + j) * kMaxTables + ti] = res;
       else s_tot[i * kMaxTables + ti] = res;
     }
     named_sync(1, kConsumerThreads);
-    for (int o = tid; o < k * k; o += kConsumerThreads) {  // option o = i * k + j
-      const int i = o / k;
+    if (tid < k * k) {
+      const int i = tid / k;
       float png = 0.f;
       for (int ti = 0; ti < nt; ++ti) {
-        const int c = s_cnt[o * kMaxTables + ti], t = s_tot[i * kMaxTables + ti];
-        st->cnt[o][ti] = c;
-        if (o % k == 0) st->tot[i][ti] = t;
+        const int c = s_cnt[tid * kMaxTables + ti], t = s_tot[i * kMaxTables + ti];
+        st->cnt[tid][ti] = c;
+        if (tid % k == 0) st->tot[i][ti] = t;
         if (t > 0) png = fmaf(p.lambda[p.tab[ti].n - 2], (float)c / (float)t, png);
       }
-      s_png[o] = png;
-      st->png[o] = png;
+      s_png[tid] = png;
+      st->png[tid] = png;
     }
     named_sync(1, kConsumerThreads);
-    for (int o = tid; o < k * k; o += kConsumerThreads) {
-      const int i = o / k, j = o - i * k;
+    if (tid < k * k) {
+      const int i = tid / k, j = tid - i * k;
       bool overlap = false;
       for (int jj = 0; jj < k; ++jj) overlap |= s_png[i * k + jj] > 0.f;
       const float base = st->logP[i] + (1.f - p.alpha) * st->cand_lp[j];
       float sc;
-      if (!overlap) sc = base + p.log_delta;                               // Eq. 7
-      else if (s_png[o] > 0.f) sc = base + p.alpha * logf(s_png[o]);       // Eq. 6
-      else sc = -CUDART_INF_F;                                             // token absent from the n-gram distribution
-      s_score[o] = sc;
-      st->score[o] = sc;
+      if (!overlap) sc = base + p.log_delta;                                   // Eq. 7
+      else if (s_png[tid] > 0.f) sc = base + p.alpha * logf(s_png[tid]);       // Eq. 6
+      else sc = -CUDART_INF_F;                                                 // token absent from the n-gram distribution
+      s_score[tid] = sc;
+      st->score[tid] = sc;
     }
     named_sync(1, kConsumerThreads);
     if (tid < 32) {
@@ -1047,7 +842,7 @@ __device__ __noinline__ void tail_score_select(const KParams *pp, uint4 *scratch
 }
 
 // Next LM input (block 0): the token embedding in prefill, the superposed embedding of Eq. 3 in decode.
-__device__ __forceinline__ void embed_input(const KParams &p, int it) {
+__device__ void embed_input(const KParams &p, int it) {
   const State *st = p.st;
   if (p.mode == kModePrefill) {
     const int tok = p.prefix[it];
@@ -1063,50 +858,47 @@ __device__ __forceinline__ void embed_input(const KParams &p, int it) {
 }
 
 // ---------------------------------------------------------------- consumer main loop
-__device__ __forceinline__ void consumer_main(Blk &b) {
+__device__ void consumer_main(Blk &b) {
   const KParams &p = *b.p;
+  float xr[kMaxVec][8];
   for (int it = 0; it < p.n_iters; ++it) {
     const int pos = p.pos0 + it;
     if (blockIdx.x == 0) embed_input(p, it);
     if (grid_barrier(b)) return;
-    const bool head = p.mode == kModeDecode || it == p.n_iters - 1;
-    const int nph = head ? 4 * p.L + 1 : 4 * p.L;
-    for (int ph = 0; ph < nph; ++ph) {
-      const PhaseDesc pd = phase_desc(p, ph);
-      const int l = ph >> 2, j = ph == 4 * p.L ? 4 : (ph & 3);
-      EpiArgs ea{l, pos, j == 3 ? 1 : 0};
-      int kind, xsrc = kXSmem;
-      if (j == 0) {
-        prologue_norm(b, p.h, p.layers[l].attn_norm, p.d);
-        kind = kEpiQKV;
-      } else if (j == 1) {
-        attention_phase(b, l, pos);
-        if (grid_barrier(b)) return;
-        prologue_attn(b, pos + 1);
-        kind = kEpiAddH;
-      } else if (j == 2) {
-        prologue_norm(b, p.h, p.layers[l].ffn_norm, p.d);
-        kind = kEpiSwiGLU;
-      } else if (j == 3) {
-        xsrc = kXGlobal;
-        kind = kEpiAddH;
-      } else {
-        prologue_norm(b, p.h, p.final_norm, p.d);
-        kind = kEpiLogits;
-      }
-      consume_matrix(b, pd.R, pd.C, pd.gran, xsrc, kind, ea);
-      if (j == 4) {
-        named_sync(1, kConsumerThreads);
-        int r0, r1;
-        cta_rows(p.V, 1, r0, r1);
-        if (threadIdx.x < 32) block_topk(p, r0, r1);
-      }
+    for (int l = 0; l < p.L; ++l) {
+      const LayerW lw = p.layers[l];
+      EpiArgs ea{l, pos, 0};
+      prologue_norm(b, p.h, lw.attn_norm, p.d, xr);
+      consume_matrix(b, 3 * p.d, p.d, 2, xr, kEpiQKV, ea);
+      if (grid_barrier(b)) return;
+      attention_phase(b, l, pos);
+      if (grid_barrier(b)) return;
+      prologue_attn(p, pos + 1, xr);
+      consume_matrix(b, p.d, p.d, 1, xr, kEpiAddH, ea);
+      if (grid_barrier(b)) return;
+      prologue_norm(b, p.h, lw.ffn_norm, p.d, xr);
+      consume_matrix(b, 2 * p.f, p.d, 2, xr, kEpiSwiGLU, ea);
+      if (grid_barrier(b)) return;
+      prologue_plain(p.u, p.f, xr);
+      ea.which = 1;
+      consume_matrix(b, p.d, p.f, 1, xr, kEpiAddH, ea);
       if (grid_barrier(b)) return;
     }
-    if (head && blockIdx.x == 0) {
-      if (threadIdx.x < 32) tail_keep_topk(b.p);
-      const bool first = p.mode == kModePrefill;
-      tail_score_select(b.p, b.xf, b.dead, first, first ? 0 : p.step0 + it);
+    const bool last = it == p.n_iters - 1;
+    if (p.mode == kModeDecode || last) {
+      EpiArgs ea{0, pos, 0};
+      prologue_norm(b, p.h, p.final_norm, p.d, xr);
+      consume_matrix(b, p.V, p.d, 1, xr, kEpiLogits, ea);
+      named_sync(1, kConsumerThreads);
+      int r0, r1;
+      cta_rows(p.V, 1, r0, r1);
+      if (threadIdx.x < 32) block_topk(p, r0, r1);
+      if (grid_barrier(b)) return;
+      if (blockIdx.x == 0) {
+        if (threadIdx.x < 32) tail_keep_topk(p);
+        const bool first = p.mode == kModePrefill;
+        tail_score_select(b, first, first ? 0 : p.step0 + it);
+      }
     }
   }
 }
@@ -1120,7 +912,6 @@ __global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_co
   b.p = &p;
   b.ring = smem;
   b.part = reinterpret_cast<float *>(smem + (size_t)p.n_stages * p.stage_bytes);
-  b.xf = reinterpret_cast<uint4 *>(smem + (size_t)p.n_stages * p.stage_bytes + sizeof(float) * 2 * kTile * kPartStride);
   b.full = s_full;
   b.empty = s_empty;
   b.red = s_red;
@@ -1139,18 +930,13 @@ __global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_co
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // the ring starts zeroed: rows of a last, short group that no copy writes are still multiplied (into
-  // columns nobody reads), so they must hold finite values
-  for (size_t i = threadIdx.x; i < (size_t)p.n_stages * p.stage_bytes / 16; i += blockDim.x)
-    reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0u, 0u, 0u, 0u);
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
   if (p.mode == kModeScoreOnly) {
-    if (blockIdx.x == 0 && threadIdx.x < kConsumerThreads) tail_score_select(b.p, b.xf, b.dead, false, p.step0);
+    if (blockIdx.x == 0 && threadIdx.x < kConsumerThreads) tail_score_select(b, false, p.step0);
     return;
   }
   if (threadIdx.x >= kConsumerThreads) {
-    producer_main(b);
+    if (threadIdx.x == kConsumerThreads) producer_main(b);
   } else {
     consumer_main(b);
   }

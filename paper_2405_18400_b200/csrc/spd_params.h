@@ -10,19 +10,13 @@ namespace spd {
 constexpr int kMaxK = 16;
 constexpr int kMaxTables = 8;
 constexpr int kWin = 8;             // tokens of history kept per draft (n_max - 1 <= 5 are used)
-constexpr int kConsumerWarps = 7;   // warps that multiply; one more warp streams weights (8 warps: 255 registers each)
+constexpr int kConsumerWarps = 16;  // warps that multiply; one more warp streams weights
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
-constexpr int kPartStride = 8;      // floats between the rows of the partial-sum buffer (>= kConsumerWarps)
-constexpr int kTile = 64;           // rows between two epilogues (rows that pass the ring whole)
-constexpr int kSegTile = 32;        // the same for rows cut into segments
-constexpr int kGroupRows = 4;       // rows per tensor-core tile
-constexpr int kMaxPB = 10;          // 64-column pair-blocks a warp owns in a whole row: columns <= 4096 over 7 warps
-constexpr int kSegPB = 5;           // the same inside a segment: segments of at most 2048 columns
-constexpr int kMaxWholeCols = 4096;  // rows up to this many columns pass the ring whole
-constexpr int kMaxSegCols = 2048;    // longer rows are cut into segments of at most this many columns
+constexpr int kTile = 128;          // rows between two epilogues
+constexpr int kMaxRowsPerChunk = 8;
 constexpr int kMaxStages = 16;
-constexpr int kMaxVec = 4;          // 8-column vectors per thread in a prologue: d_model <= 6144 over 224 threads
+constexpr int kMaxVec = 4;          // 16-byte column vectors per thread: columns <= 4 * 512 * 8
 constexpr int kMaxSplit = 8;        // attention splits per head
 
 enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2 };
@@ -73,8 +67,7 @@ struct KParams {
   // workspace
   void *kcache, *vcache;     // [L][max_pos][d] float or bf16
   const float2 *rope;        // [max_pos][hd/2] (cos, sin)
-  float *h, *q, *logits;     // [d], [d], [V]
-  unsigned short *ufrag;     // FFN activation as tensor-core A fragments: [ceil(f/64)][12][8] 32-bit words
+  float *h, *q, *u, *logits; // [d], [d], [f], [V]
   float *opart;              // [H * kMaxSplit][hd] unnormalised attention partials
   float2 *oml;               // [H * kMaxSplit] (running max, running sum)
   float *pk_val;             // [grid][k] per-block top logits

