@@ -510,8 +510,107 @@ __device__ __forceinline__ float load_kv(const KParams &p, const void *cache, si
   return __ldcg(reinterpret_cast<const float *>(cache) + idx);
 }
 
+// Fast path of the attention phase for a bf16 cache and head_dim 128 (a cache row of a head is 256 bytes):
+// half a warp takes one position with 16-byte loads, and each warp keeps eight positions in flight, so a
+// long context costs a few dependent memory round trips instead of one per position.  Each half-warp runs
+// its own online softmax; halves, then warps, are merged at the end exactly like the general path.
+__device__ void attention_phase_bf16_hd128(Blk &b, int layer, int pos) {
+  const KParams &p = *b.p;
+  const int T = pos + 1, ns = attn_splits(p, T), items = p.H * ns;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
+  const float scale = 1.f / sqrtf(128.f);
+  float *s_acc = b.part;                           // [warps][128]
+  float *s_m = b.part + kConsumerWarps * 256;      // [warps]
+  float *s_l = s_m + kConsumerWarps;               // [warps]
+  const __nv_bfloat16 *kc = reinterpret_cast<const __nv_bfloat16 *>(p.kcache);
+  const __nv_bfloat16 *vc = reinterpret_cast<const __nv_bfloat16 *>(p.vcache);
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int head = item / ns, sp = item - head * ns;
+    const int t0 = (int)((long long)T * sp / ns), t1 = (int)((long long)T * (sp + 1) / ns);
+    float q[8], acc[8];
+    load8(p.q + head * 128 + l16 * 8, q);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    float m = -CUDART_INF_F, l = 0.f;
+    const size_t col = (size_t)head * 128 + l16 * 8;
+    for (int tb = t0 + warp * 8; tb < t1; tb += kConsumerWarps * 8) {
+      uint4 kq[4], vq[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int t = min(tb + 2 * u + half, t1 - 1);  // clamped: the extra loads are discarded below
+        const size_t off = ((size_t)layer * p.max_pos + t) * p.d + col;
+        kq[u] = __ldcg(reinterpret_cast<const uint4 *>(kc + off));
+        vq[u] = __ldcg(reinterpret_cast<const uint4 *>(vc + off));
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t kw[4] = {kq[u].x, kq[u].y, kq[u].z, kq[u].w};
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          dot = fmaf(q[2 * e], __uint_as_float(kw[e] << 16), dot);
+          dot = fmaf(q[2 * e + 1], __uint_as_float(kw[e] & 0xffff0000u), dot);
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        if (tb + 2 * u + half < t1) {  // uniform within the half-warp
+          const float s = dot * scale;
+          const float mn = fmaxf(m, s);
+          const float c = __expf(m - mn), pw = __expf(s - mn);
+          l = l * c + pw;
+          const uint32_t vw[4] = {vq[u].x, vq[u].y, vq[u].z, vq[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            acc[2 * e] = acc[2 * e] * c + pw * __uint_as_float(vw[e] << 16);
+            acc[2 * e + 1] = acc[2 * e + 1] * c + pw * __uint_as_float(vw[e] & 0xffff0000u);
+          }
+          m = mn;
+        }
+      }
+    }
+    // merge the two half-warps
+    {
+      const float mo = __shfl_xor_sync(0xffffffffu, m, 16), lo = __shfl_xor_sync(0xffffffffu, l, 16);
+      const float M = fmaxf(m, mo);
+      const float w_self = m == -CUDART_INF_F ? 0.f : __expf(m - M), w_oth = mo == -CUDART_INF_F ? 0.f : __expf(mo - M);
+      l = l * w_self + lo * w_oth;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = acc[e] * w_self + __shfl_xor_sync(0xffffffffu, acc[e], 16) * w_oth;
+      m = M;
+    }
+    if (half == 0) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s_acc[warp * 256 + l16 * 8 + e] = acc[e];
+    }
+    if (lane == 0) {
+      s_m[warp] = m;
+      s_l[warp] = l;
+    }
+    named_sync(1, kConsumerThreads);
+    if (threadIdx.x < 128) {
+      float M = -CUDART_INF_F;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, s_m[w]);
+      float L = 0.f, A = 0.f;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) {
+        const float wgt = s_m[w] == -CUDART_INF_F ? 0.f : __expf(s_m[w] - M);
+        L = fmaf(s_l[w], wgt, L);
+        A = fmaf(s_acc[w * 256 + threadIdx.x], wgt, A);
+      }
+      p.opart[(size_t)item * 128 + threadIdx.x] = A;
+      if (threadIdx.x == 0) p.oml[item] = make_float2(M, L);
+    }
+    named_sync(1, kConsumerThreads);
+  }
+}
+
 __device__ void attention_phase(Blk &b, int layer, int pos) {
   const KParams &p = *b.p;
+  if (p.kv_bf16 && p.hd == 128) {
+    attention_phase_bf16_hd128(b, layer, pos);
+    return;
+  }
   const int T = pos + 1, ns = attn_splits(p, T), items = p.H * ns;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int epl = p.hd / 32;  // elements per lane, <= 8
