@@ -325,7 +325,8 @@ __device__ __forceinline__ void store_kv(const KParams &p, void *cache, size_t i
 }
 
 // Finishes rows [t0, t1) of the current matrix from the warps' partial sums.
-__device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, const float *part, int t0, int t1) {
+__device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, const float *part, int t0, int t1, bool have_h,
+                                         float h_pre) {
   const KParams &p = *b.p;
   const int tid = threadIdx.x;
   const int rows = t1 - t0;
@@ -357,7 +358,7 @@ __device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, co
   } else if (kind == kEpiAddH) {
     if (tid < rows) {
       const int r = t0 + tid;
-      const float y = __ldcg(p.h + r) + part_sum(part + (size_t)tid * kConsumerWarps);
+      const float y = (have_h ? h_pre : __ldcg(p.h + r)) + part_sum(part + (size_t)tid * kConsumerWarps);
       p.h[r] = y;
       if (p.trace) p.trace[((size_t)ea.layer * 2 + ea.which) * p.d + r] = y;
     }
@@ -381,6 +382,9 @@ __device__ __forceinline__ void consume_matrix(Blk &b, int R, int C, int gran, c
   cta_rows(R, gran, r0, r1);
   const int rpc = rows_per_chunk(p, C);
   const int rowbytes = C * 2, nv = C / 8;
+  // the residual rows this thread will update in the first tile are fetched now, off the critical path
+  float h_pre = 0.f;
+  if (kind == kEpiAddH && r0 + (int)threadIdx.x < min(r0 + kTile, r1)) h_pre = __ldcg(p.h + r0 + threadIdx.x);
   int buf = 0;
   for (int t0 = r0; t0 < r1; t0 += kTile) {
     const int t1 = min(t0 + kTile, r1);
@@ -399,7 +403,7 @@ __device__ __forceinline__ void consume_matrix(Blk &b, int R, int C, int gran, c
       if (++b.c_stage == (uint32_t)p.n_stages) { b.c_stage = 0; b.c_phase ^= 1u; }
     }
     named_sync(1, kConsumerThreads);
-    epilogue(b, kind, ea, part, t0, t1);
+    epilogue(b, kind, ea, part, t0, t1, t0 == r0, h_pre);
     buf ^= 1;
   }
 }
