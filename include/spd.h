@@ -139,6 +139,16 @@ int spd_step(spd_ctx *ctx, int32_t *out_ids, int32_t *out_parent, float *out_gam
 int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *out_len, float *out_logp,
                  float *out_gamma);
 
+/*
+ * Reset (Section 5.3 "Superposed Decoding Resets"): one of the k drafts is chosen - by the caller; the paper
+ * samples one every s timesteps - and draft generation restarts from it.  The chosen draft's tokens are
+ * appended to the prefix, the cache positions that were filled from superposed inputs are recomputed from
+ * those tokens (the original prefix's positions are kept), and the first timestep (Eq. 1) runs on the longer
+ * prefix.  Afterwards the context is exactly as after spd_prefill on prefix + chosen draft.  draft: 0..k-1;
+ * out_ids / out_gamma as for spd_prefill.  SPD_ESTATE before spd_prefill.  Synchronises the stream.
+ */
+int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma);
+
 /* Same as spd_generate but only enqueues the launch: no synchronisation, no outputs.  For callers
  * that time the launch with their own CUDA events; follow with spd_sync. */
 int spd_generate_async(spd_ctx *ctx, int32_t n_steps);

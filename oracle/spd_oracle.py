@@ -169,6 +169,11 @@ class Oracle:
             raise ValueError("orc_prefill: bad arguments")
         return out, g
 
+    def reset(self, draft: int):
+        """Section 5.3: generation restarts from one draft.  By definition: the first timestep on the prefix
+        followed by that draft's tokens, everything recomputed from scratch."""
+        return self.prefill(self.drafts()[int(draft)].tolist())
+
     def step(self):
         ids = np.zeros(self.k, np.int32)
         par = np.zeros(self.k, np.int32)

@@ -65,7 +65,7 @@ _lib: Optional[C.CDLL] = None
 
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
-           "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static"]
+           "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset"]
 
 
 def load_library() -> C.CDLL:
@@ -88,6 +88,7 @@ def load_library() -> C.CDLL:
                              C.c_size_t, C.POINTER(C.c_void_p)]
     L.spd_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.spd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.spd_reset.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.spd_generate.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_generate_async.argtypes = [C.c_void_p, C.c_int32]
     L.spd_sync.argtypes = [C.c_void_p]
@@ -226,6 +227,12 @@ class SpdContext:
         ids = np.zeros(self.k, np.int32)
         g = np.zeros(self.k, np.float32)
         _check(self.lib.spd_prefill(self.h, a.ctypes.data, a.shape[0], ids.ctypes.data, g.ctypes.data), "spd_prefill")
+        return ids, g
+
+    def spd_reset(self, draft: int):
+        ids = np.zeros(self.k, np.int32)
+        g = np.zeros(self.k, np.float32)
+        _check(self.lib.spd_reset(self.h, int(draft), ids.ctypes.data, g.ctypes.data), "spd_reset")
         return ids, g
 
     def spd_step(self):

@@ -102,6 +102,7 @@ struct spd_ctx {
   size_t dyn_smem;
   bool prefilled;
   int32_t m;       // prefix length
+  std::vector<int32_t> prefix;  // host copy of the prefix (spd_reset extends it)
   int32_t n_gen;   // tokens generated per draft
   int64_t launches;
 };
@@ -344,7 +345,59 @@ int spd_prefill(spd_ctx *ctx, const int32_t *prefix_ids, int32_t m, int32_t *out
   ctx->prefilled = true;
   ctx->m = m;
   ctx->n_gen = 1;
+  ctx->prefix.assign(prefix_ids, prefix_ids + m);
   for (int i = 0; i < c.k; ++i) {
+    if (out_ids) out_ids[i] = ids[i];
+    if (out_gamma) out_gamma[i] = gamma[i];
+  }
+  return SPD_OK;
+}
+
+int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma) {
+  if (!ctx) return SPD_EINVAL;
+  if (!ctx->prefilled) return SPD_ESTATE;
+  const spd_config &c = ctx->cfg;
+  if (draft < 0 || draft >= c.k) return SPD_ERANGE;
+  const int k = c.k, n = ctx->n_gen, m = ctx->m;
+  if (m + n >= c.max_pos) return SPD_ERANGE;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  // the chosen draft's tokens, by its parent links
+  std::vector<int32_t> tok((size_t)n * k), par((size_t)n * k), seq(n);
+  SPD_CUDA(cudaMemcpyAsync(tok.data(), ctx->ws + ctx->lay.hist_tok, tok.size() * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  SPD_CUDA(cudaMemcpyAsync(par.data(), ctx->ws + ctx->lay.hist_par, par.size() * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  if ((rc = spd_sync(ctx))) return rc;
+  for (int s = n - 1, cur = draft; s >= 0; --s) {
+    seq[s] = tok[(size_t)s * k + cur];
+    cur = par[(size_t)s * k + cur];
+  }
+  ctx->prefix.insert(ctx->prefix.end(), seq.begin(), seq.end());
+  const int m2 = m + n;
+  // fresh draft state on the longer prefix; positions 0..m-1 of the cache stay, positions m..m2-1 (so far
+  // computed from superposed inputs) are recomputed from the draft's own tokens
+  spd::State st;
+  std::memset(&st, 0, sizeof st);
+  st.win_len = m2 < spd::kWin ? m2 : spd::kWin;
+  for (int i = 0; i < k; ++i)
+    for (int j = 0; j < st.win_len; ++j) st.win[i][spd::kWin - st.win_len + j] = ctx->prefix[m2 - st.win_len + j];
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.state, &st, sizeof st, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix + (size_t)m * 4, seq.data(), (size_t)n * 4, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));
+  ctx->prefilled = false;
+  const int32_t *base = ctx->kp.prefix;
+  ctx->kp.prefix = base + m;
+  rc = launch(ctx, spd::kModePrefill, n, m, 0);
+  ctx->kp.prefix = base;
+  if (rc) return rc;
+  int32_t ids[SPD_MAX_K];
+  float gamma[SPD_MAX_K];
+  if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;
+  if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
+  if ((rc = check_device_error(ctx))) return rc;
+  ctx->prefilled = true;
+  ctx->m = m2;
+  ctx->n_gen = 1;
+  for (int i = 0; i < k; ++i) {
     if (out_ids) out_ids[i] = ids[i];
     if (out_gamma) out_gamma[i] = gamma[i];
   }

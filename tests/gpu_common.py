@@ -63,8 +63,14 @@ def _sync_logp(ctx, orc, eps_z):
     orc.set_logP(lp)
 
 
-def compare_first_step(ctx, orc, prefix, stats=None):
-    ids, g = ctx.spd_prefill(prefix)
+def compare_first_step(ctx, orc, prefix, stats=None, reset_draft=None):
+    """First timestep on both sides.  With reset_draft, the restart from that draft (Section 5.3) instead: the
+    device recomputes only the generated positions, the oracle everything."""
+    if reset_draft is None:
+        ids, g = ctx.spd_prefill(prefix)
+    else:
+        prefix = orc.drafts()[reset_draft].tolist()
+        ids, g = ctx.spd_reset(reset_draft)
     following = _follow(ctx, orc, len(prefix))
     ids_o, g_o = orc.prefill(prefix)
     if following:

@@ -207,6 +207,31 @@ def test_self_generated_corpus_gives_hits_end_to_end(tiny_inputs):
     ctx.close()
 
 
+@pytest.mark.parametrize("kv_dtype", ["bf16", "f32"])
+def test_resets_restart_from_a_chosen_draft(tiny_inputs, kv_dtype):
+    """Section 5.3: every few steps one draft is chosen and generation restarts from it.  The device keeps the
+    original prefix's cache and recomputes the generated positions from the draft's tokens; the oracle
+    recomputes everything from prefix + draft."""
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, orc = make_tiny_pair(tiny_inputs, kv_dtype=kv_dtype, max_pos=64)
+    compare_first_step(ctx, orc, prefix)
+    for draft in (1, 0, 2):
+        for _ in range(3):
+            compare_step(ctx, orc)
+        before = orc.drafts()[draft].tolist()
+        compare_first_step(ctx, orc, None, reset_draft=draft)
+        assert orc.drafts()[:, :-1].tolist() == [before] * 3          # the chosen draft is now everyone's prefix
+        toks, lp, g = ctx.spd_generate(1, 2)                          # history restarts after a reset
+        orc.step()
+        assert np.array_equal(toks, orc.drafts()[:, len(before):])
+        compare_first_step(ctx, orc, before)                          # and a plain prefill on the longer prefix agrees too
+    import paper_2405_18400_b200 as P
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_reset(3)
+    assert e.value.status == -3
+    ctx.close()
+
+
 def test_call_order_and_range_errors(tiny_inputs):
     import paper_2405_18400_b200 as P
     wl, weights, tables, prefix = tiny_inputs
