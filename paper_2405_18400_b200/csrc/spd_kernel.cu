@@ -85,7 +85,6 @@ struct Blk {
   volatile int *dead;
   volatile int *quit;  // block-uniform copy of *dead, refreshed inside every grid barrier
   unsigned int bar_target;
-  unsigned int tail_target;
   // consumer ring cursor
   uint32_t c_stage, c_phase;
 };
@@ -1021,7 +1020,6 @@ __global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_co
   b.dead = &s_dead;
   b.quit = &s_quit;
   b.bar_target = 0;
-  b.tail_target = 0;
   b.c_stage = 0;
   b.c_phase = 0;
   if (threadIdx.x == 0) {

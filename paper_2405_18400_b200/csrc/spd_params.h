@@ -34,7 +34,7 @@ struct TableDev {
 // Draft state and the last step's intermediates, in device memory.
 struct State {
   unsigned int bar;         // grid barrier counter (zeroed by the host before every launch)
-  unsigned int tail_bar;    // arrivals of the LM-head phase
+  unsigned int reserved0;
   unsigned int abort_flag;  // set by any thread that gave up a wait
   int32_t err, err_info;
   int32_t win_len;          // valid tokens in each history window

@@ -273,3 +273,35 @@ def test_ring_settings_do_not_change_results(tiny_inputs):
     with pytest.raises(P.SpdError):
         ctx.spd_set_ring(1024, 4)              # a 688-column row (1376 bytes) does not fit
     ctx.close()
+
+
+def test_malformed_table_is_reported_not_hung(tiny_inputs):
+    """A table image without a single empty slot (never produced by spd_ngram_build) makes the probe of an absent
+    key run to its bound: the step returns SPD_ETABLE, nothing hangs, and the context works again afterwards
+    with a sound table."""
+    import paper_2405_18400_b200 as P
+    wl, weights, tables, prefix = tiny_inputs
+    good = P.build_ngram_tables(tables, "cuda:0")
+    slots = 1 << 15
+    img = np.zeros((slots, 4), np.uint32)
+    img[:, 0] = np.arange(slots, dtype=np.uint32) | 0xfff00000          # keys no lookup asks for (token ids >= 4096)
+    img[:, 3] = 1
+    bad = [dict(t) for t in good]
+    bad[0] = {"n": 2, "ngram_slots": slots, "ctx_slots": slots,
+              "ngram": torch.from_numpy(img.view(np.uint8).reshape(-1)).to("cuda:0"),
+              "ctx": torch.from_numpy(img.view(np.uint8).reshape(-1)).to("cuda:0")}
+    packed = P.pack_weights(weights, "cuda:0")
+    ctx = P.SpdContext(wl.shape, packed, bad, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64)
+    ctx.spd_prefill(prefix)                     # the first timestep does not touch the tables
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_step()
+    assert e.value.status == -6
+    with pytest.raises(P.SpdError) as e:        # the failed run invalidated the drafts
+        ctx.spd_step()
+    assert e.value.status == -2
+    ctx.close()
+    ok = P.SpdContext(wl.shape, packed, good, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64)
+    ok.spd_prefill(prefix)
+    ids, par, g = ok.spd_step()
+    assert abs(float(g.sum()) - 1) < 1e-5
+    ok.close()
