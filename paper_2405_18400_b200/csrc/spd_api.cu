@@ -12,6 +12,8 @@
 
 extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size_t dyn_smem, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm);
+extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm);
+extern "C" cudaError_t spd_internal_prefill_launch(const spd::KParams *p, int grid, cudaStream_t stream);
 
 namespace {
 
@@ -35,7 +37,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, total;
+      trace, pf_h, pf_q, pf_o, pf_u, total;
 };
 
 bool valid_config(const spd_config *c) {
@@ -83,6 +85,10 @@ Layout make_layout(const spd_config &c, int grid) {
   L.hist_par = take((size_t)c.max_pos * c.k * 4);
   L.prefix = take((size_t)c.max_pos * 4);
   L.trace = take((size_t)c.n_layers * 2 * c.d_model * 4);
+  L.pf_h = take((size_t)spd::kPfTokens * c.d_model * 4);
+  L.pf_q = take((size_t)spd::kPfTokens * c.d_model * 4);
+  L.pf_o = take((size_t)spd::kPfTokens * c.d_model * 4);
+  L.pf_u = take((size_t)spd::kPfTokens * c.d_ffn * 4);
   L.total = off;
   return L;
 }
@@ -131,17 +137,53 @@ int check_device_error(spd_ctx *ctx) {
   return err[0];
 }
 
-int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0) {
+// Bytes of the state's head that every launch zeroes: with `keep_err` the error words of earlier launches
+// of the same call survive (the first error sticks), else they are cleared too.
+size_t head_bytes(bool keep_err) { return keep_err ? offsetof(spd::State, err) : offsetof(spd::State, win_len); }
+
+int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0, bool keep_err = false) {
   spd::KParams &kp = ctx->kp;
   kp.mode = mode;
   kp.n_iters = n_iters;
   kp.pos0 = pos0;
   kp.step0 = step0;
   // barrier counters, abort flag and error word start from zero at every launch
-  SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, offsetof(spd::State, win_len), ctx->stream));
+  SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(keep_err), ctx->stream));
   SPD_CUDA(spd_internal_launch(&kp, ctx->grid, ctx->dyn_smem, ctx->stream));
   ctx->launches += 1;
   return SPD_OK;
+}
+
+// Runs prefix tokens [first, first + count) (positions alike) through the prefill kernel, kPfTokens at a
+// time: their keys and values enter the cache, nothing else of the state changes.
+int prefill_tokens(spd_ctx *ctx, int first, int count) {
+  spd::KParams &kp = ctx->kp;
+  const int32_t *base = kp.prefix;
+  int rc = SPD_OK;
+  for (int done = 0; done < count && rc == SPD_OK; done += spd::kPfTokens) {
+    const int n = count - done < spd::kPfTokens ? count - done : spd::kPfTokens;
+    kp.mode = spd::kModePrefill;
+    kp.n_iters = n;
+    kp.pos0 = first + done;
+    kp.step0 = 0;
+    kp.prefix = base + first + done;
+    cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(done > 0), ctx->stream);
+    if (e == cudaSuccess) e = spd_internal_prefill_launch(&kp, ctx->grid, ctx->stream);
+    if (e != cudaSuccess) rc = cuda_fail(e, "prefill launch");
+    else ctx->launches += 1;
+  }
+  kp.prefix = base;
+  return rc;
+}
+
+// The last prefix token (position `pos`): the decode kernel's single-token pass, which ends with the
+// first-timestep decision.
+int prefill_last(spd_ctx *ctx, int pos, bool keep_err) {
+  const int32_t *base = ctx->kp.prefix;
+  ctx->kp.prefix = base + pos;
+  const int rc = launch(ctx, spd::kModePrefill, 1, pos, 0, keep_err);
+  ctx->kp.prefix = base;
+  return rc;
 }
 
 int set_device(const spd_ctx *ctx) {
@@ -237,6 +279,9 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   e = spd_internal_prepare(ctx->dyn_smem, &per_sm);
   if (e != cudaSuccess) return fail(cuda_fail(e, "kernel attributes"));
   if (per_sm < 1) return fail(SPD_EINVAL);
+  e = spd_internal_prefill_prepare(&per_sm);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "prefill kernel attributes"));
+  if (per_sm < 1) return fail(SPD_EINVAL);
 
   const int hd = cfg->d_model / cfg->n_heads;
   kp.L = cfg->n_layers; kp.d = cfg->d_model; kp.H = cfg->n_heads; kp.hd = hd; kp.f = cfg->d_ffn; kp.V = cfg->vocab;
@@ -269,6 +314,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.hist_tok = reinterpret_cast<int32_t *>(ws + lay.hist_tok); kp.hist_par = reinterpret_cast<int32_t *>(ws + lay.hist_par);
   kp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
   kp.trace = reinterpret_cast<float *>(ws + lay.trace);
+  kp.pf_h = reinterpret_cast<float *>(ws + lay.pf_h); kp.pf_q = reinterpret_cast<float *>(ws + lay.pf_q);
+  kp.pf_o = reinterpret_cast<float *>(ws + lay.pf_o); kp.pf_u = reinterpret_cast<float *>(ws + lay.pf_u);
 
   // rotary table: cos / sin of pos * theta^(-2i/hd), evaluated in double and rounded once
   std::vector<float2> rope((size_t)cfg->max_pos * (hd / 2));
@@ -336,7 +383,8 @@ int spd_prefill(spd_ctx *ctx, const int32_t *prefix_ids, int32_t m, int32_t *out
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix, prefix_ids, (size_t)m * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));  // st and the caller's ids may go out of scope
   ctx->prefilled = false;
-  if ((rc = launch(ctx, spd::kModePrefill, m, 0, 0))) return rc;
+  if ((rc = prefill_tokens(ctx, 0, m - 1))) return rc;
+  if ((rc = prefill_last(ctx, m - 1, m > 1))) return rc;
   int32_t ids[SPD_MAX_K];
   float gamma[SPD_MAX_K];
   if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;
@@ -384,11 +432,8 @@ int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma) {
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix + (size_t)m * 4, seq.data(), (size_t)n * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));
   ctx->prefilled = false;
-  const int32_t *base = ctx->kp.prefix;
-  ctx->kp.prefix = base + m;
-  rc = launch(ctx, spd::kModePrefill, n, m, 0);
-  ctx->kp.prefix = base;
-  if (rc) return rc;
+  if ((rc = prefill_tokens(ctx, m, n - 1))) return rc;
+  if ((rc = prefill_last(ctx, m2 - 1, n > 1))) return rc;
   int32_t ids[SPD_MAX_K];
   float gamma[SPD_MAX_K];
   if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;

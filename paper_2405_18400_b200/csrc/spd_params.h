@@ -18,6 +18,7 @@ constexpr int kMaxRowsPerChunk = 8;
 constexpr int kMaxStages = 16;
 constexpr int kMaxVec = 4;          // 16-byte column vectors per thread: columns <= 4 * 512 * 8
 constexpr int kMaxSplit = 8;        // attention splits per head
+constexpr int kPfTokens = 16;       // prefix tokens one prefill launch takes
 
 enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2 };
 
@@ -77,6 +78,8 @@ struct KParams {
   int32_t *hist_tok, *hist_par;  // [max_pos][k]
   const int32_t *prefix;     // [max_pos]
   float *trace;              // [L][2][d] or null
+  float *pf_h, *pf_q, *pf_o; // [kPfTokens][d] prefill: residual rows, rotated queries, attention output
+  float *pf_u;               // [kPfTokens][f] prefill: SwiGLU output
   // launch
   int32_t mode, n_iters, pos0, step0;
   int32_t stage_bytes, n_stages;
