@@ -37,7 +37,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, pf_h, pf_q, pf_o, pf_u, total;
+      trace, pf_h, pf_q, pf_xh, pf_xo, pf_xu, total;
 };
 
 bool valid_config(const spd_config *c) {
@@ -56,6 +56,9 @@ bool valid_config(const spd_config *c) {
   if (c->kv_dtype != 0 && c->kv_dtype != 1) return false;
   return true;
 }
+
+// Bytes of a prefill fragment buffer for C columns: per 16 columns, 2 token tiles x 3 terms x 32 lanes x 8 bytes.
+size_t frag_bytes(int C) { return (size_t)((C + 15) / 16) * 2 * 3 * 32 * 8; }
 
 Layout make_layout(const spd_config &c, int grid) {
   Layout L{};
@@ -87,8 +90,9 @@ Layout make_layout(const spd_config &c, int grid) {
   L.trace = take((size_t)c.n_layers * 2 * c.d_model * 4);
   L.pf_h = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_q = take((size_t)spd::kPfTokens * c.d_model * 4);
-  L.pf_o = take((size_t)spd::kPfTokens * c.d_model * 4);
-  L.pf_u = take((size_t)spd::kPfTokens * c.d_ffn * 4);
+  L.pf_xh = take(frag_bytes(c.d_model));
+  L.pf_xo = take(frag_bytes(c.d_model));
+  L.pf_xu = take(frag_bytes(c.d_ffn));
   L.total = off;
   return L;
 }
@@ -315,7 +319,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
   kp.trace = reinterpret_cast<float *>(ws + lay.trace);
   kp.pf_h = reinterpret_cast<float *>(ws + lay.pf_h); kp.pf_q = reinterpret_cast<float *>(ws + lay.pf_q);
-  kp.pf_o = reinterpret_cast<float *>(ws + lay.pf_o); kp.pf_u = reinterpret_cast<float *>(ws + lay.pf_u);
+  kp.pf_xh = reinterpret_cast<uint16_t *>(ws + lay.pf_xh); kp.pf_xo = reinterpret_cast<uint16_t *>(ws + lay.pf_xo);
+  kp.pf_xu = reinterpret_cast<uint16_t *>(ws + lay.pf_xu);
 
   // rotary table: cos / sin of pos * theta^(-2i/hd), evaluated in double and rounded once
   std::vector<float2> rope((size_t)cfg->max_pos * (hd / 2));
@@ -338,6 +343,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   if (e == cudaSuccess) e = cudaMemcpyAsync(ws + lay.layers, layers.data(), layers.size() * sizeof(spd::LayerW), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.state, 0, sizeof(spd::State), s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.trace, 0, (size_t)cfg->n_layers * 2 * cfg->d_model * 4, s);
+  // columns past the row's end inside the last 16-column step of a fragment buffer are never written: zero
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.pf_xh, 0, lay.total - lay.pf_xh, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return fail(cuda_fail(e, "workspace initialisation"));
   *out = ctx;

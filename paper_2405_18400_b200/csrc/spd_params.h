@@ -78,8 +78,10 @@ struct KParams {
   int32_t *hist_tok, *hist_par;  // [max_pos][k]
   const int32_t *prefix;     // [max_pos]
   float *trace;              // [L][2][d] or null
-  float *pf_h, *pf_q, *pf_o; // [kPfTokens][d] prefill: residual rows, rotated queries, attention output
-  float *pf_u;               // [kPfTokens][f] prefill: SwiGLU output
+  float *pf_h, *pf_q;        // [kPfTokens][d] prefill: residual rows, rotated queries
+  // prefill activations as mma fragments, three bf16 terms each: [ceil(C/16)][2][3][32] x 8 bytes
+  uint16_t *pf_xh, *pf_xo;   // gain-scaled residual (C = d), attention output (C = d)
+  uint16_t *pf_xu;           // SwiGLU output (C = f)
   // launch
   int32_t mode, n_iters, pos0, step0;
   int32_t stage_bytes, n_stages;

@@ -3,10 +3,17 @@
 // decision).  With several tokens per weight the products are real matrix-matrix contractions, so they run
 // on tensor cores: mma.sync m16n8k16 with A = 16 weight rows x 16 columns straight from the bf16 rows,
 // B = the tokens' activations split exactly into three bf16 terms (x = hi + mid + lo to float32
-// precision), float32 accumulation.  One persistent cooperative launch per chunk of tokens: a producer
-// warp streams weight tiles (16 rows x 1024 columns) through a shared-memory ring with bulk copies, eight
-// consumer warps share every tile by k-steps, per-warp partial sums are reduced through shared memory once
-// per 16 rows, and the same five phases per layer as in decoding are separated by grid barriers.
+// precision), float32 accumulation.
+//
+// One persistent cooperative launch per chunk of tokens.  Per block: a producer warp streams the block's
+// weight rows (chunks of 32 rows x 512 columns) through a shared-memory ring with bulk copies; eight
+// consumer warps share every chunk by k-steps; per-warp partial sums meet in shared memory once per 16
+// rows.  Activations travel between phases already split and laid out as mma B fragments: the epilogue
+// that produces a value writes its three bf16 terms into a fragment buffer in global memory, and in the next
+// phase a second producer warp pulls 512 columns of all 16 tokens (48 KB) at a time into shared memory with
+// one bulk copy; each consumer warp takes its k-steps' fragments into registers at once, which frees the
+// buffer for the next K block while the current one is multiplied.  No block repeats the conversion.  RMSNorm's gain is applied before the split, its per-token 1/rms after the product
+// (it is a scalar per token).  The five phases per layer are separated by grid barriers as in decoding.
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
@@ -17,28 +24,34 @@ namespace spd {
 
 constexpr int kPfWarps = 8;
 constexpr int kPfThreads = kPfWarps * 32;  // consumer threads
-constexpr int kPfBlock = kPfThreads + 32;  // plus the producer warp
-constexpr int kPfKB = 1024;                // columns per K block
+constexpr int kPfBlock = kPfThreads + 64;  // plus the weight producer warp and the fragment producer warp
+constexpr int kPfKB = 512;                 // columns per K block
 constexpr int kPfKSteps = kPfKB / 16;
-constexpr int kPfTileRows = 16;
-constexpr int kPfMaxTiles = 12;            // row tiles whose accumulators a warp keeps at a time
-constexpr int kPfPitch = kPfKB * 2 + 16;   // bytes between the rows of a tile in a stage (padding: no bank conflicts)
-constexpr int kPfStageBytes = kPfTileRows * kPfPitch;
-constexpr int kPfStages = 3;
-constexpr int kPfXblkBytes = kPfKSteps * 2 * 3 * 32 * 8;  // [k-step][token tile][term][lane] x 8 bytes
+constexpr int kPfTileRows = 16;            // rows of one mma tile
+constexpr int kPfChunkRows = 32;           // rows of one ring stage: two tiles
+constexpr int kPfMaxTiles = 10;            // row tiles whose accumulators a warp keeps at a time
+constexpr int kPfMaxChunks = kPfMaxTiles / 2;
+constexpr int kPfPitch = kPfKB * 2 + 16;   // bytes between the rows of a chunk in a stage (padding: no bank conflicts)
+constexpr int kPfStageBytes = kPfChunkRows * kPfPitch;
+constexpr int kPfStages = 5;
+constexpr int kPfXBufs = 1;                // shared-memory fragment buffers (the consumers empty one into registers at once)
+constexpr int kPfKStepBytes = 2 * 3 * 32 * 8;             // fragments of one k-step: [token tile][term][lane] x 8 bytes
+constexpr int kPfXBytes = kPfKSteps * kPfKStepBytes;      // one K block of fragments
 constexpr int kPfRedBytes = kPfWarps * kPfTileRows * kPfTokens * 4;
 constexpr unsigned long long kPfWaitNs = 1500ull * 1000ull * 1000ull;
 
 struct PfBlk {
   const KParams *p;
   uint8_t *ring;
-  uint2 *xblk;
+  uint8_t *xblk;  // kPfXBufs fragment buffers of kPfXBytes
   float *red;
-  float *rs;  // [16] per-token 1/rms
-  uint64_t *full, *empty;
+  float *rs;      // [16] per-token 1/rms
+  float *am;      // [2][kPfWarps] attention merge: running max, running sum
+  uint64_t *full, *empty, *xfull, *xempty, *xgo;
   volatile int *dead, *quit;
   unsigned int bar_target;
   uint32_t c_stage, c_phase;
+  uint32_t x_n;  // fragment copies consumed so far: copy n sits in buffer n % kPfXBufs and is that buffer's use n / kPfXBufs
 };
 
 __device__ __forceinline__ void pf_give_up(PfBlk &b, int code, int info) {
@@ -48,18 +61,20 @@ __device__ __forceinline__ void pf_give_up(PfBlk &b, int code, int info) {
   *b.dead = 1;
 }
 
-__device__ __forceinline__ void pf_wait(PfBlk &b, uint64_t *bar, uint32_t parity, int info) {
-  if (mbar_try_wait(bar, parity)) return;
-  if (*b.dead) return;
+// Bounded wait on an mbarrier phase; false when the block gave up instead.
+__device__ __forceinline__ bool pf_wait(PfBlk &b, uint64_t *bar, uint32_t parity, int info) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (*b.dead) return false;
   unsigned long long t0 = globaltimer();
   uint32_t n = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++n & 31u) == 0) {
-      if (*b.dead) return;
-      if (ld_relaxed(&b.p->st->abort_flag)) { *b.dead = 1; return; }
-      if (globaltimer() - t0 > kPfWaitNs) { pf_give_up(b, -7, info); return; }
+      if (*b.dead) return false;
+      if (ld_relaxed(&b.p->st->abort_flag)) { *b.dead = 1; return false; }
+      if (globaltimer() - t0 > kPfWaitNs) { pf_give_up(b, -7, info); return false; }
     }
   }
+  return true;
 }
 
 __device__ __forceinline__ bool pf_grid_barrier(PfBlk &b) {
@@ -108,7 +123,7 @@ __device__ __forceinline__ PfPhase pf_phase(const KParams &p, int ph) {
 }
 
 // ---------------------------------------------------------------- producer
-// Chunk order of a phase: per group of up to 12 row tiles, K block by K block, tile by tile.
+// Chunk order of a phase: per group of up to kPfMaxTiles row tiles, K block by K block, chunk (32 rows) by chunk.
 __device__ void pf_producer(PfBlk &b) {
   const KParams &p = *b.p;
   const int lane = threadIdx.x & 31;
@@ -125,8 +140,8 @@ __device__ void pf_producer(PfBlk &b) {
       const int g1 = min(g0 + kPfMaxTiles * kPfTileRows, r1);
       for (int kb = 0; kb < nkb && ok; ++kb) {
         const uint32_t piece = (uint32_t)min(kPfKB, pd.C - kb * kPfKB) * 2u;
-        for (int t0 = g0; t0 < g1 && ok; t0 += kPfTileRows) {
-          const int nrows = min(kPfTileRows, g1 - t0);
+        for (int c0 = g0; c0 < g1 && ok; c0 += kPfChunkRows) {
+          const int nrows = min(kPfChunkRows, g1 - c0);
           int dead = 0;
           if (lane == 0) {
             pf_wait(b, &b.empty[stage], phase ^ 1u, 200);
@@ -137,7 +152,7 @@ __device__ void pf_producer(PfBlk &b) {
           if (dead) { ok = false; break; }
           if (lane < nrows)
             bulk_load(b.ring + (size_t)stage * kPfStageBytes + (size_t)lane * kPfPitch,
-                      W + (size_t)(t0 + lane) * rowbytes + (size_t)kb * kPfKB * 2, piece, &b.full[stage]);
+                      W + (size_t)(c0 + lane) * rowbytes + (size_t)kb * kPfKB * 2, piece, &b.full[stage]);
           if (issued < (uint32_t)kPfStages) ++issued;
           if (++stage == (uint32_t)kPfStages) { stage = 0; phase ^= 1u; }
         }
@@ -145,6 +160,7 @@ __device__ void pf_producer(PfBlk &b) {
     }
   }
   if (!ok && lane == 0) {
+    // giving up: wait (bounded) for the copies already issued, so that none lands after the block has gone
     uint32_t s = stage, ph = phase;
     for (uint32_t i = 0; i < issued; ++i) {
       if (s == 0) { s = (uint32_t)kPfStages; ph ^= 1u; }
@@ -156,7 +172,7 @@ __device__ void pf_producer(PfBlk &b) {
   __syncwarp();
 }
 
-// ---------------------------------------------------------------- consumer helpers
+// ---------------------------------------------------------------- fragments
 __device__ __forceinline__ void pf_mma(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
@@ -165,20 +181,70 @@ __device__ __forceinline__ void pf_mma(float (&d)[4], uint32_t a0, uint32_t a1, 
 __device__ __forceinline__ void pf_ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-__device__ __forceinline__ uint32_t pf_bf16(float v) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v)); }
 
-enum PfSrc { kPfNorm = 0, kPfPlain = 1 };
+// Writes activation v of (token t, column c) into a fragment buffer as three bf16 terms with
+// hi + mid + lo = v exactly: each term takes the leading 8 significant bits of what is left, by truncation,
+// and a float32 has 24.  Layout: [k-step c / 16][token tile t / 8][term][lane (t % 8) * 4 + (c % 8) / 2]
+// x {columns (2q, 2q+1), columns (8 + 2q, 9 + 2q)} bf16, which is what one lane of the mma wants as B.
+__device__ __forceinline__ void pf_put(uint16_t *F, int t, int c, float v) {
+  const uint32_t hi = __float_as_uint(v) & 0xffff0000u;
+  const float r1 = v - __uint_as_float(hi);
+  const uint32_t mid = __float_as_uint(r1) & 0xffff0000u;
+  const float r2 = r1 - __uint_as_float(mid);
+  const uint32_t lo = __float_as_uint(r2);
+  const size_t unit = (size_t)(c >> 4) * 2 + (t >> 3);
+  const size_t e = ((unit * 3) * 32 + (size_t)((t & 7) * 4 + ((c & 7) >> 1))) * 4 + ((c >> 3) & 1) * 2 + (c & 1);
+  F[e] = (uint16_t)(hi >> 16);
+  F[e + 128] = (uint16_t)(mid >> 16);
+  F[e + 256] = (uint16_t)(lo >> 16);
+}
 
-// Per-token 1/rms of the residual rows (every block computes all 16; rows past n_tok count as zero).
-__device__ void pf_token_rms(PfBlk &b, const float *H, int d, int n_tok) {
+// Fragment producer (one thread): copies the K blocks of each phase's fragment buffer into shared memory, in the order the consumers take them.  A phase's fragments are complete once the consumers have
+// passed the grid barrier before it (they say so on `xgo`); a buffer is free again once all consumer warps
+// have taken their fragments of it into registers (`xempty`).
+__device__ void pf_xproducer(PfBlk &b) {
+  const KParams &p = *b.p;
+  uint32_t n = 0;
+  bool ok = true;
+  for (int ph = 0; ph < 4 * p.L && ok; ++ph) {
+    const PfPhase pd = pf_phase(p, ph);
+    int r0, r1;
+    pf_rows(pd.R, pd.gran, r0, r1);
+    const uint8_t *F = reinterpret_cast<const uint8_t *>((ph & 1) == 0 ? p.pf_xh : (ph & 3) == 1 ? p.pf_xo : p.pf_xu);
+    const int nks_total = (pd.C + 15) / 16;
+    const int nkb = (pd.C + kPfKB - 1) / kPfKB;
+    if (!pf_wait(b, b.xgo, (uint32_t)ph & 1u, 320)) break;
+    asm volatile("fence.proxy.async;" ::: "memory");  // the fragments were written with ordinary stores by other blocks
+    for (int g0 = r0; g0 < r1 && ok; g0 += kPfMaxTiles * kPfTileRows)
+      for (int kb = 0; kb < nkb; ++kb) {
+        const int buf = n % kPfXBufs;
+        if (!pf_wait(b, &b.xempty[buf], ((n / kPfXBufs) & 1u) ^ 1u, 330)) { ok = false; break; }
+        const uint32_t bytes = (uint32_t)min(kPfKSteps, nks_total - kb * kPfKSteps) * (uint32_t)kPfKStepBytes;
+        mbar_expect_tx(&b.xfull[buf], bytes);
+        bulk_load(b.xblk + (size_t)buf * kPfXBytes, F + (size_t)kb * kPfXBytes, bytes, &b.xfull[buf]);
+        ++n;
+      }
+  }
+  if (*b.dead) {
+    // giving up: wait (bounded) for the last copy into each buffer, the only ones that can still be in flight
+    for (uint32_t i = 0; i < (uint32_t)kPfXBufs && i < n; ++i) {
+      const uint32_t m = n - 1 - i;
+      unsigned long long t0 = globaltimer();
+      while (!mbar_try_wait(&b.xfull[m % kPfXBufs], (m / kPfXBufs) & 1u) && globaltimer() - t0 < kPfWaitNs) {}
+    }
+  }
+}
+
+// Per-token 1/rms of the residual rows (every block computes all 16; rows past n_tok are zero).
+__device__ void pf_token_rms(PfBlk &b, const float *H, int d) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int t = warp; t < kPfTokens; t += kPfWarps) {
     float ss = 0.f;
-    if (t < n_tok)
-      for (int c = lane * 4; c < d; c += 128) {
-        const float4 v = __ldcg(reinterpret_cast<const float4 *>(H + (size_t)t * d + c));
-        ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
-      }
+#pragma unroll 8
+    for (int c = lane * 4; c < d; c += 128) {
+      const float4 v = __ldcg(reinterpret_cast<const float4 *>(H + (size_t)t * d + c));
+      ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if (lane == 0) b.rs[t] = rsqrtf(ss / (float)d + b.p->eps);
@@ -186,73 +252,38 @@ __device__ void pf_token_rms(PfBlk &b, const float *H, int d, int n_tok) {
   named_sync(1, kPfThreads);
 }
 
-// Stages K block kb of the 16 tokens' activations as B fragments: thread (token t = tid / 16, piece j =
-// tid % 16) handles the 64 columns [kb*1024 + 64 j, +64) of token t = k-steps 4j..4j+3 of the block.
-// Fragment store: xblk[((ks * 2 + token tile) * 3 + term) * 32 + (t % 8) * 4 + q] = {cols (2q, 2q+1), cols (8+2q, 9+2q)}.
-__device__ void pf_stage_x(PfBlk &b, int src, const float *X, const __nv_bfloat16 *gain, int C, int kb, int n_tok) {
-  const int t = threadIdx.x >> 4, j = threadIdx.x & 15;
-  const int nt = t >> 3, g = t & 7;
-  const float rs = src == kPfNorm ? b.rs[t] : 1.f;
+constexpr int kPfOwnSteps = kPfKSteps / kPfWarps;  // k-steps of a K block that one warp multiplies
+
+// One tile against this warp's k-steps of the K block: 16 rows x 16 columns of weights per k-step times the
+// three terms of both token tiles (fragments already in registers).  The two token tiles' accumulators
+// alternate so that consecutive mma do not depend on each other.
+__device__ __forceinline__ void pf_tile(float (&acc)[2][4], uint32_t base, const uint2 (&bb)[kPfOwnSteps][6], int warp) {
 #pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-    const int ks = 4 * j + kk;
-    const int c0 = kb * kPfKB + ks * 16;
-    float x[16];
-#pragma unroll
-    for (int e = 0; e < 16; ++e) x[e] = 0.f;
-    if (t < n_tok) {
-      // columns come in multiples of 8: the last k-step of a row may be half full
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int c = c0 + 8 * half;
-        if (c < C) {
-          const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(X + (size_t)t * C + c));
-          const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(X + (size_t)t * C + c) + 1);
-          float *xh = x + 8 * half;
-          xh[0] = v0.x; xh[1] = v0.y; xh[2] = v0.z; xh[3] = v0.w;
-          xh[4] = v1.x; xh[5] = v1.y; xh[6] = v1.z; xh[7] = v1.w;
-          if (src == kPfNorm) {
-            const uint4 gv = *reinterpret_cast<const uint4 *>(gain + c);
-            const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              xh[2 * e] = xh[2 * e] * rs * __uint_as_float(gw[e] << 16);
-              xh[2 * e + 1] = xh[2 * e + 1] * rs * __uint_as_float(gw[e] & 0xffff0000u);
-            }
-          }
-        }
-      }
-    }
-    uint32_t term[3][16];
-#pragma unroll
-    for (int e = 0; e < 16; ++e) {
-      term[0][e] = pf_bf16(x[e]);
-      float r = x[e] - __uint_as_float(term[0][e] << 16);
-      term[1][e] = pf_bf16(r);
-      r -= __uint_as_float(term[1][e] << 16);
-      term[2][e] = pf_bf16(r);
-    }
+  for (int s = 0; s < kPfOwnSteps; ++s) {
+    uint32_t a0, a1, a2, a3;
+    pf_ldsm_x4(base + (uint32_t)(warp + s * kPfWarps) * 32u, a0, a1, a2, a3);
 #pragma unroll
     for (int k = 0; k < 3; ++k)
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        b.xblk[(size_t)((ks * 2 + nt) * 3 + k) * 32 + g * 4 + q] =
-            make_uint2(term[k][2 * q] | (term[k][2 * q + 1] << 16), term[k][8 + 2 * q] | (term[k][9 + 2 * q] << 16));
+      for (int n = 0; n < 2; ++n) pf_mma(acc[n], a0, a1, a2, a3, bb[s][n * 3 + k].x, bb[s][n * 3 + k].y);
   }
 }
 
 enum PfEpi { kPfQKV = 0, kPfAddH = 1, kPfSwiGLU = 2 };
 
-// One matrix for the 16 tokens: out[t][r] = sum_c W[r][c] x[t][c] for this block's rows, then the
-// phase's epilogue.
-__device__ void pf_gemm(PfBlk &b, const PfPhase &pd, int src, const float *X, const __nv_bfloat16 *gain, int kind, int layer,
-                        int pos0, int n_tok) {
+// One matrix for the 16 tokens: out[t][r] = scale_t * sum_c W[r][c] x[t][c] for this block's rows (x from the
+// phase's fragment buffer; scale_t = 1/rms of token t when `norm`, else 1), then the phase's epilogue.  `gain_next`
+// (kPfAddH): gain of the RMSNorm that reads the new residual next, or null when nothing does.
+__device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const __nv_bfloat16 *gain_next,
+                        int layer, int pos0, int n_tok) {
   const KParams &p = *b.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
   int r0, r1;
   pf_rows(pd.R, pd.gran, r0, r1);
+  const int nks_total = (pd.C + 15) / 16;
   const int nkb = (pd.C + kPfKB - 1) / kPfKB;
-  if (src == kPfNorm) pf_token_rms(b, X, pd.C, n_tok);
+  if (tid == 0) mbar_arrive(b.xgo);  // the grid barrier before this phase is behind us: its fragments are complete
+  if (norm) pf_token_rms(b, p.pf_h, pd.C);
   // ldmatrix addresses of this lane inside a tile: rows 0-7 / 8-15, columns k0 / k0+8
   const uint32_t lane_off = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * kPfPitch + (uint32_t)(lane >> 4) * 16u;
   for (int g0 = r0; g0 < r1; g0 += kPfMaxTiles * kPfTileRows) {
@@ -263,26 +294,31 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, int src, const float *X, co
 #pragma unroll
       for (int n = 0; n < 2; ++n) acc[i][n][0] = acc[i][n][1] = acc[i][n][2] = acc[i][n][3] = 0.f;
     for (int kb = 0; kb < nkb; ++kb) {
-      named_sync(1, kPfThreads);  // everyone is done with the previous K block's fragments
-      pf_stage_x(b, src, X, gain, pd.C, kb, n_tok);
-      named_sync(1, kPfThreads);
-      const int nks = min(kPfKSteps, (pd.C - kb * kPfKB + 15) / 16);
+      const int buf = b.x_n % kPfXBufs;
+      pf_wait(b, &b.xfull[buf], (b.x_n / kPfXBufs) & 1u, 310);
+      b.x_n += 1;
+      // this warp's k-steps of the block: fragments to registers (zeros past the row's end, so that whatever
+      // the ring holds there does not count), then the buffer is free for the K block after the next
+      const uint2 *xb = reinterpret_cast<const uint2 *>(b.xblk + (size_t)buf * kPfXBytes) + lane;
+      const int nks = min(kPfKSteps, nks_total - kb * kPfKSteps);
+      uint2 bb[kPfOwnSteps][6];
 #pragma unroll
-      for (int i = 0; i < kPfMaxTiles; ++i) {
-        if (g0 + i * kPfTileRows < g1) {
+      for (int s = 0; s < kPfOwnSteps; ++s) {
+        const int ks = warp + s * kPfWarps;
+#pragma unroll
+        for (int e = 0; e < 6; ++e) bb[s][e] = ks < nks ? xb[(ks * 6 + e) * 32] : make_uint2(0u, 0u);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&b.xempty[buf]);
+#pragma unroll
+      for (int j = 0; j < kPfMaxChunks; ++j) {
+        if (g0 + j * kPfChunkRows < g1) {
           pf_wait(b, &b.full[b.c_stage], b.c_phase, 300);
-          const uint32_t base = smem_u32(b.ring + (size_t)b.c_stage * kPfStageBytes) + lane_off;
-          for (int ks = warp; ks < nks; ks += kPfWarps) {
-            uint32_t a0, a1, a2, a3;
-            pf_ldsm_x4(base + (uint32_t)ks * 32u, a0, a1, a2, a3);
-            const uint2 *xb = b.xblk + (size_t)(ks * 6) * 32 + lane;
+          const uint32_t cbase = smem_u32(b.ring + (size_t)b.c_stage * kPfStageBytes) + lane_off;
 #pragma unroll
-            for (int n = 0; n < 2; ++n)
-#pragma unroll
-              for (int k = 0; k < 3; ++k) {
-                const uint2 bb = xb[(n * 3 + k) * 32];
-                pf_mma(acc[i][n], a0, a1, a2, a3, bb.x, bb.y);
-              }
+          for (int h = 0; h < 2; ++h) {
+            const int i = 2 * j + h;
+            if (g0 + i * kPfTileRows < g1) pf_tile(acc[i], cbase + (uint32_t)(h * kPfTileRows * kPfPitch), bb, warp);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&b.empty[b.c_stage]);
@@ -310,30 +346,36 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, int src, const float *X, co
         float y = 0.f;
 #pragma unroll
         for (int w = 0; w < kPfWarps; ++w) y += b.red[w * (kPfTileRows * kPfTokens) + row * kPfTokens + t];
+        if (norm) y *= b.rs[t];
         const float other = __shfl_xor_sync(0xffffffffu, y, 16);
         const int r = t0 + row;
-        if (r < g1 && t < n_tok) {
+        if (r < g1) {
+          // tokens past n_tok carry zeros through every phase; only the cache is not touched for them
           const int pos = pos0 + t;
           if (kind == kPfQKV) {
-            const int sec = r / p.d, col = r - sec * p.d;
-            float v = y;
-            if (sec < 2) {
-              const float2 cs = p.rope[(size_t)pos * (p.hd / 2) + (col % p.hd) / 2];
-              v = (row & 1) ? other * cs.y + y * cs.x : y * cs.x - other * cs.y;
-            }
-            const size_t kv = ((size_t)layer * p.max_pos + pos) * p.d + col;
-            if (sec == 0) {
-              p.pf_q[(size_t)t * p.d + col] = v;
-            } else {
-              void *cache = sec == 1 ? p.kcache : p.vcache;
-              if (p.kv_bf16) reinterpret_cast<__nv_bfloat16 *>(cache)[kv] = __float2bfloat16_rn(v);
-              else reinterpret_cast<float *>(cache)[kv] = v;
+            if (t < n_tok) {
+              const int sec = r / p.d, col = r - sec * p.d;
+              float v = y;
+              if (sec < 2) {
+                const float2 cs = p.rope[(size_t)pos * (p.hd / 2) + (col % p.hd) / 2];
+                v = (row & 1) ? other * cs.y + y * cs.x : y * cs.x - other * cs.y;
+              }
+              const size_t kv = ((size_t)layer * p.max_pos + pos) * p.d + col;
+              if (sec == 0) {
+                p.pf_q[(size_t)t * p.d + col] = v;
+              } else {
+                void *cache = sec == 1 ? p.kcache : p.vcache;
+                if (p.kv_bf16) reinterpret_cast<__nv_bfloat16 *>(cache)[kv] = __float2bfloat16_rn(v);
+                else reinterpret_cast<float *>(cache)[kv] = v;
+              }
             }
           } else if (kind == kPfAddH) {
             float *h = p.pf_h + (size_t)t * p.d + r;
-            *h = __ldcg(h) + y;
+            const float hn = __ldcg(h) + y;
+            *h = hn;
+            if (gain_next) pf_put(p.pf_xh, t, r, hn * __bfloat162float(gain_next[r]));
           } else {
-            if (!(row & 1)) p.pf_u[(size_t)t * p.f + (r >> 1)] = y / (1.f + __expf(-y)) * other;
+            if (!(row & 1)) pf_put(p.pf_xu, t, r >> 1, y / (1.f + __expf(-y)) * other);
           }
         }
       }
@@ -342,18 +384,22 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, int src, const float *X, co
 }
 
 // Causal attention of the chunk's tokens over the cache: one (token, head) item per block at a time, a warp
-// per position with an online softmax, the warps merged through shared memory.
+// per position with an online softmax, the warps merged through shared memory.  Items of tokens past n_tok
+// only write zeros.
 __device__ void pf_attention(PfBlk &b, int layer, int pos0, int n_tok) {
   const KParams &p = *b.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int epl = p.hd / 32;
   const float scale = 1.f / sqrtf((float)p.hd);
-  float *s_acc = b.red;                            // [warps][256] (red holds 8 x 256 floats)
-  float *s_m = reinterpret_cast<float *>(b.xblk);  // the fragment area is idle during this phase
-  float *s_l = s_m + kPfWarps;
-  const int items = n_tok * p.H;
+  float *s_acc = b.red;  // [warps][256]
+  float *s_m = b.am, *s_l = b.am + kPfWarps;
+  const int items = kPfTokens * p.H;
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int t = item / p.H, head = item - t * p.H;
+    if (t >= n_tok) {
+      for (int dim = threadIdx.x; dim < p.hd; dim += kPfThreads) pf_put(p.pf_xo, t, head * p.hd + dim, 0.f);
+      continue;
+    }
     const int T = pos0 + t + 1;
     float q[8], acc[8];
 #pragma unroll
@@ -410,7 +456,7 @@ __device__ void pf_attention(PfBlk &b, int layer, int pos0, int n_tok) {
         L = fmaf(s_l[w], wgt, L);
         A = fmaf(s_acc[w * 256 + dim], wgt, A);
       }
-      p.pf_o[(size_t)t * p.d + head * p.hd + dim] = A / L;
+      pf_put(p.pf_xo, t, head * p.hd + dim, A / L);
     }
   }
   named_sync(1, kPfThreads);
@@ -419,23 +465,28 @@ __device__ void pf_attention(PfBlk &b, int layer, int pos0, int n_tok) {
 __device__ void pf_consumer(PfBlk &b) {
   const KParams &p = *b.p;
   const int n_tok = p.n_iters, pos0 = p.pos0;
-  // residual rows start as the tokens' embeddings
-  for (int i = blockIdx.x * kPfThreads + threadIdx.x; i < n_tok * p.d; i += gridDim.x * kPfThreads) {
-    const int t = i / p.d, c = i - t * p.d;
-    p.pf_h[i] = __bfloat162float(p.tok_emb[(size_t)p.prefix[t] * p.d + c]);
+  // residual rows start as the tokens' embeddings (zeros past n_tok)
+  {
+    const __nv_bfloat16 *gain0 = p.layers[0].attn_norm;
+    for (int i = blockIdx.x * kPfThreads + threadIdx.x; i < kPfTokens * p.d; i += gridDim.x * kPfThreads) {
+      const int t = i / p.d, c = i - t * p.d;
+      const float v = t < n_tok ? __bfloat162float(p.tok_emb[(size_t)p.prefix[t] * p.d + c]) : 0.f;
+      p.pf_h[i] = v;
+      pf_put(p.pf_xh, t, c, v * __bfloat162float(gain0[c]));
+    }
   }
   if (pf_grid_barrier(b)) return;
   for (int l = 0; l < p.L; ++l) {
     const LayerW &lw = p.layers[l];
-    pf_gemm(b, pf_phase(p, 4 * l), kPfNorm, p.pf_h, lw.attn_norm, kPfQKV, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l), true, kPfQKV, nullptr, l, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
     pf_attention(b, l, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_gemm(b, pf_phase(p, 4 * l + 1), kPfPlain, p.pf_o, nullptr, kPfAddH, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l + 1), false, kPfAddH, lw.ffn_norm, l, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_gemm(b, pf_phase(p, 4 * l + 2), kPfNorm, p.pf_h, lw.ffn_norm, kPfSwiGLU, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l + 2), true, kPfSwiGLU, nullptr, l, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_gemm(b, pf_phase(p, 4 * l + 3), kPfPlain, p.pf_u, nullptr, kPfAddH, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l + 3), false, kPfAddH, l + 1 < p.L ? p.layers[l + 1].attn_norm : nullptr, l, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
   }
 }
@@ -444,22 +495,27 @@ __device__ void pf_consumer(PfBlk &b) {
 // is what the compiler derives for a block of 384.
 __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_constant__ KParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint64_t s_full[kPfStages], s_empty[kPfStages];
-  __shared__ float s_rs[kPfTokens];
+  __shared__ uint64_t s_full[kPfStages], s_empty[kPfStages], s_xfull[kPfXBufs], s_xempty[kPfXBufs], s_xgo;
+  __shared__ float s_rs[kPfTokens], s_am[2 * kPfWarps];
   __shared__ int s_dead, s_quit;
   PfBlk b;
   b.p = &p;
   b.ring = smem;
-  b.xblk = reinterpret_cast<uint2 *>(smem + (size_t)kPfStages * kPfStageBytes);
-  b.red = reinterpret_cast<float *>(smem + (size_t)kPfStages * kPfStageBytes + kPfXblkBytes);
+  b.xblk = smem + (size_t)kPfStages * kPfStageBytes;
+  b.red = reinterpret_cast<float *>(smem + (size_t)kPfStages * kPfStageBytes + (size_t)kPfXBufs * kPfXBytes);
   b.rs = s_rs;
+  b.am = s_am;
   b.full = s_full;
   b.empty = s_empty;
+  b.xfull = s_xfull;
+  b.xempty = s_xempty;
+  b.xgo = &s_xgo;
   b.dead = &s_dead;
   b.quit = &s_quit;
   b.bar_target = 0;
   b.c_stage = 0;
   b.c_phase = 0;
+  b.x_n = 0;
   if (threadIdx.x == 0) {
     s_dead = 0;
     s_quit = 0;
@@ -467,23 +523,34 @@ __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_consta
       mbar_init(&s_full[s], 1);
       mbar_init(&s_empty[s], kPfWarps);
     }
+    for (int i = 0; i < kPfXBufs; ++i) {
+      mbar_init(&s_xfull[i], 1);
+      mbar_init(&s_xempty[i], kPfWarps);
+    }
+    mbar_init(&s_xgo, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // rows of a last, short tile that no copy writes are still multiplied (into rows nobody reads): the ring
+  // rows of a last, short chunk that no copy writes are still multiplied (into rows nobody reads): the ring
   // starts zeroed so that they hold finite values
   for (size_t i = threadIdx.x; i < (size_t)kPfStages * kPfStageBytes / 16; i += blockDim.x)
     reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0u, 0u, 0u, 0u);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
-  if (threadIdx.x >= kPfThreads) pf_producer(b);
-  else pf_consumer(b);
+  if (threadIdx.x >= kPfThreads + 32) {
+    if (threadIdx.x == kPfThreads + 32) pf_xproducer(b);
+    __syncwarp();
+  } else if (threadIdx.x >= kPfThreads) {
+    pf_producer(b);
+  } else {
+    pf_consumer(b);
+  }
   __syncthreads();
 }
 
 }  // namespace spd
 
 extern "C" size_t spd_internal_prefill_smem(void) {
-  return (size_t)spd::kPfStages * spd::kPfStageBytes + spd::kPfXblkBytes + spd::kPfRedBytes;
+  return (size_t)spd::kPfStages * spd::kPfStageBytes + (size_t)spd::kPfXBufs * spd::kPfXBytes + spd::kPfRedBytes;
 }
 
 extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm) {
