@@ -149,6 +149,22 @@ int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *ou
  */
 int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma);
 
+/*
+ * Nucleus sampling spliced in front of Superposed Decoding (Section 4.5: a nucleus-sampled generation serves
+ * as the prefix of k superposed drafts; Section 2 for the sampler: the smallest set of most probable tokens
+ * whose probability reaches top_p, one token drawn from it in proportion to its probability).  Extends the
+ * prefix by n_new tokens, each drawn from softmax(logits / temperature) restricted to its nucleus - tokens
+ * ordered by probability, equal ones by ascending id; the draw u picks the first token whose running
+ * probability exceeds u times the nucleus' mass - then runs the first timestep (Eq. 1) on the longer prefix:
+ * afterwards the context is as after spd_prefill on prefix + sampled tokens.  The random numbers are the
+ * caller's: uniforms = HOST array of n_new floats in [0, 1).  0 < top_p <= 1, temperature > 0.  HOST outputs,
+ * any may be NULL: out_new [n_new] sampled ids; out_ids / out_gamma [k] as for spd_prefill.  Needs a context
+ * fresh from spd_prefill, spd_reset or spd_sample (no spd_step since), else SPD_ESTATE; SPD_ERANGE when the
+ * prefix would not fit or an argument is out of range.  One launch; synchronises the stream.
+ */
+int spd_sample(spd_ctx *ctx, int32_t n_new, float top_p, float temperature, const float *uniforms, int32_t *out_new,
+               int32_t *out_ids, float *out_gamma);
+
 /* Same as spd_generate but only enqueues the launch: no synchronisation, no outputs.  For callers
  * that time the launch with their own CUDA events; follow with spd_sync. */
 int spd_generate_async(spd_ctx *ctx, int32_t n_steps);
@@ -209,6 +225,13 @@ int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes);
  */
 int spd_debug_score(spd_ctx *ctx, const int32_t *hist, int32_t hist_len, const float *logp, const int32_t *cand_tok,
                     const float *cand_lp);
+
+/*
+ * Test hook for the nucleus sampler alone (the draw that spd_sample makes per token): HOST logits float
+ * [vocab], one uniform number u in [0, 1); *out_token (HOST) receives the drawn id.  No LM pass.  The
+ * context must be prefilled again before decoding continues.
+ */
+int spd_debug_nucleus(spd_ctx *ctx, const float *logits, float top_p, float temperature, float u, int32_t *out_token);
 
 /*
  * The scoring stage of one timestep (what spd_debug_score runs) without any device allocation.  The

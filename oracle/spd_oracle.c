@@ -26,7 +26,9 @@
  * with library matmuls; dense prefill against token-by-token decoding; k = 1 against a greedy
  * loop; the scoring stage against a brute-force enumeration of Eq. 5-7 in the linear domain with
  * dictionary counts; n-gram counts against a naive scan; closed forms for RMSNorm, rotary
- * embedding and single-position attention.  Unpinned against the paper itself (it prints no
+ * embedding and single-position attention; the nucleus sampler against a brute-force search over all
+ * token subsets, closed forms for uniform and two-point distributions, and draw frequencies.
+ * Unpinned against the paper itself (it prints no
  * worked example): delta's value, where tau is applied, the per-draft reading of "no overlap",
  * and the absolute value of P.
  */
@@ -279,6 +281,68 @@ void orc_topk_logprob(const double *z, int vocab, int k, double tau, int32_t *to
   for (int v = 0; v < vocab; ++v) den += exp(z[v] / tau - mx);
   double lse = mx + log(den);
   for (int j = 0; j < k; ++j) lp[j] = z[tok[j]] / tau - lse;
+}
+
+/*
+ * Nucleus sampling (Section 2: the smallest set of tokens whose cumulative probability reaches p, then a
+ * draw from that set in proportion to probability; Section 4.5 uses such generations as prefixes for SPD).
+ * prob = softmax(z / temperature); tokens are taken by descending probability, equal ones by ascending id;
+ * the nucleus is the shortest head of that order whose cumulative probability is >= p; with the uniform
+ * number u in [0, 1) the drawn token is the first whose cumulative probability exceeds u * (mass of the
+ * nucleus).  Returns the token.  info (may be NULL) receives: [0] size of the nucleus, [1] its mass,
+ * [2] distance from p to the nearest cumulative probability next to the cut, [3] distance from u * mass to
+ * the nearer end of the drawn token's interval.
+ */
+typedef struct { double z; int32_t id; } ns_item;
+static int ns_cmp(const void *a, const void *b) {
+  const ns_item *x = (const ns_item *)a, *y = (const ns_item *)b;
+  if (x->z > y->z) return -1;
+  if (x->z < y->z) return 1;
+  return x->id < y->id ? -1 : (x->id > y->id ? 1 : 0);
+}
+int32_t orc_nucleus(const double *z, int vocab, double temperature, double p, double u, double *info) {
+  ns_item *it = (ns_item *)malloc(sizeof(ns_item) * (size_t)vocab);
+  double mx = -INFINITY, den = 0.0;
+  for (int v = 0; v < vocab; ++v)
+    if (z[v] / temperature > mx) mx = z[v] / temperature;
+  for (int v = 0; v < vocab; ++v) den += exp(z[v] / temperature - mx);
+  for (int v = 0; v < vocab; ++v) {
+    it[v].z = z[v];
+    it[v].id = v;
+  }
+  qsort(it, (size_t)vocab, sizeof(ns_item), ns_cmp);
+  /* the cut */
+  double cum = 0.0, before = 0.0;
+  int size = 0;
+  while (size < vocab) {
+    before = cum;
+    cum += exp(it[size].z / temperature - mx) / den;
+    ++size;
+    if (cum >= p) break;
+  }
+  const double mass = cum;
+  const double gap_cut = fmin(fabs(cum - p), fabs(p - before));
+  /* the draw */
+  const double target = u * mass;
+  double run = 0.0, lo = 0.0;
+  int pick = size - 1;
+  for (int i = 0; i < size; ++i) {
+    lo = run;
+    run += exp(it[i].z / temperature - mx) / den;
+    if (run > target) {
+      pick = i;
+      break;
+    }
+  }
+  if (info) {
+    info[0] = (double)size;
+    info[1] = mass;
+    info[2] = gap_cut;
+    info[3] = fmin(target - lo, run - target);
+  }
+  const int32_t tok = it[pick].id;
+  free(it);
+  return tok;
 }
 
 /* gamma_i = p_i / sum_j p_j with p = exp(logP)  (Eq. 4) */

@@ -75,6 +75,8 @@ def lib() -> C.CDLL:
         L.orc_attention_head.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
         L.orc_topk_logprob.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_double, C.c_void_p, C.c_void_p]
         L.orc_gamma.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
+        L.orc_nucleus.restype = C.c_int32
+        L.orc_nucleus.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_double, C.c_void_p]
         L.orc_ngram_counts.argtypes = [C.POINTER(OrcNgram), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.orc_png.restype = C.c_double
         L.orc_png.argtypes = [C.POINTER(OrcConfig), C.POINTER(OrcNgram), C.c_int, C.c_void_p, C.c_int, C.c_int32,
@@ -307,6 +309,14 @@ def topk_logprob(z: np.ndarray, k: int, tau: float):
     lp = np.zeros(k, np.float64)
     lib().orc_topk_logprob(_ptr(z), z.shape[0], k, tau, _ptr(tok), _ptr(lp))
     return tok, lp
+
+
+def nucleus(z: np.ndarray, temperature: float, p: float, u: float):
+    """Nucleus sampling of one token from logits z: (token, {size, mass, gap_cut, gap_draw})."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    info = np.zeros(4, np.float64)
+    tok = lib().orc_nucleus(_ptr(z), z.shape[0], float(temperature), float(p), float(u), _ptr(info))
+    return int(tok), {"size": int(info[0]), "mass": float(info[1]), "gap_cut": float(info[2]), "gap_draw": float(info[3])}
 
 
 def max_threads() -> int:

@@ -65,7 +65,8 @@ _lib: Optional[C.CDLL] = None
 
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
-           "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset"]
+           "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
+           "spd_sample", "spd_debug_nucleus"]
 
 
 def load_library() -> C.CDLL:
@@ -89,6 +90,7 @@ def load_library() -> C.CDLL:
     L.spd_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
     L.spd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_reset.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    L.spd_sample.argtypes = [C.c_void_p, C.c_int32, C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_generate.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_generate_async.argtypes = [C.c_void_p, C.c_int32]
     L.spd_sync.argtypes = [C.c_void_p]
@@ -101,6 +103,7 @@ def load_library() -> C.CDLL:
                                   C.c_void_p]
     L.spd_debug_read.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t]
     L.spd_debug_score.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.spd_debug_nucleus.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_void_p]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
     L.spd_set_ring.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
@@ -234,6 +237,24 @@ class SpdContext:
         g = np.zeros(self.k, np.float32)
         _check(self.lib.spd_reset(self.h, int(draft), ids.ctypes.data, g.ctypes.data), "spd_reset")
         return ids, g
+
+    def spd_debug_nucleus(self, logits, top_p: float, temperature: float, u: float) -> int:
+        z = np.ascontiguousarray(logits, dtype=np.float32)
+        assert z.shape == (self.shape.vocab,)
+        tok = C.c_int32(-1)
+        _check(self.lib.spd_debug_nucleus(self.h, z.ctypes.data, float(top_p), float(temperature), float(u), C.byref(tok)),
+               "spd_debug_nucleus")
+        return int(tok.value)
+
+    def spd_sample(self, uniforms, top_p: float, temperature: float):
+        """Extends the prefix by len(uniforms) nucleus-sampled tokens, then the first timestep: (new ids, ids, gamma)."""
+        u = np.ascontiguousarray(uniforms, dtype=np.float32)
+        new = np.zeros(u.shape[0], np.int32)
+        ids = np.zeros(self.k, np.int32)
+        g = np.zeros(self.k, np.float32)
+        _check(self.lib.spd_sample(self.h, int(u.shape[0]), float(top_p), float(temperature), u.ctypes.data,
+                                   new.ctypes.data, ids.ctypes.data, g.ctypes.data), "spd_sample")
+        return new, ids, g
 
     def spd_step(self):
         ids = np.zeros(self.k, np.int32)

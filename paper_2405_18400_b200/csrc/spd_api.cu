@@ -37,7 +37,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, pf_h, pf_q, pf_xh, pf_xo, pf_xu, total;
+      trace, ns_u, pf_h, pf_q, pf_xh, pf_xo, pf_xu, total;
 };
 
 bool valid_config(const spd_config *c) {
@@ -88,6 +88,7 @@ Layout make_layout(const spd_config &c, int grid) {
   L.hist_par = take((size_t)c.max_pos * c.k * 4);
   L.prefix = take((size_t)c.max_pos * 4);
   L.trace = take((size_t)c.n_layers * 2 * c.d_model * 4);
+  L.ns_u = take((size_t)c.max_pos * 4);
   L.pf_h = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_q = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_xh = take(frag_bytes(c.d_model));
@@ -162,7 +163,7 @@ int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0, bool keep_e
 // time: their keys and values enter the cache, nothing else of the state changes.
 int prefill_tokens(spd_ctx *ctx, int first, int count) {
   spd::KParams &kp = ctx->kp;
-  const int32_t *base = kp.prefix;
+  int32_t *base = kp.prefix;
   int rc = SPD_OK;
   for (int done = 0; done < count && rc == SPD_OK; done += spd::kPfTokens) {
     const int n = count - done < spd::kPfTokens ? count - done : spd::kPfTokens;
@@ -183,7 +184,7 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
 // The last prefix token (position `pos`): the decode kernel's single-token pass, which ends with the
 // first-timestep decision.
 int prefill_last(spd_ctx *ctx, int pos, bool keep_err) {
-  const int32_t *base = ctx->kp.prefix;
+  int32_t *base = ctx->kp.prefix;
   ctx->kp.prefix = base + pos;
   const int rc = launch(ctx, spd::kModePrefill, 1, pos, 0, keep_err);
   ctx->kp.prefix = base;
@@ -316,7 +317,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.pk_ms = reinterpret_cast<float2 *>(ws + lay.pk_ms);
   kp.st = reinterpret_cast<spd::State *>(ws + lay.state);
   kp.hist_tok = reinterpret_cast<int32_t *>(ws + lay.hist_tok); kp.hist_par = reinterpret_cast<int32_t *>(ws + lay.hist_par);
-  kp.prefix = reinterpret_cast<const int32_t *>(ws + lay.prefix);
+  kp.prefix = reinterpret_cast<int32_t *>(ws + lay.prefix);
+  kp.ns_u = reinterpret_cast<const float *>(ws + lay.ns_u);
   kp.trace = reinterpret_cast<float *>(ws + lay.trace);
   kp.pf_h = reinterpret_cast<float *>(ws + lay.pf_h); kp.pf_q = reinterpret_cast<float *>(ws + lay.pf_q);
   kp.pf_xh = reinterpret_cast<uint16_t *>(ws + lay.pf_xh); kp.pf_xo = reinterpret_cast<uint16_t *>(ws + lay.pf_xo);
@@ -450,6 +452,52 @@ int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma) {
   ctx->m = m2;
   ctx->n_gen = 1;
   for (int i = 0; i < k; ++i) {
+    if (out_ids) out_ids[i] = ids[i];
+    if (out_gamma) out_gamma[i] = gamma[i];
+  }
+  return SPD_OK;
+}
+
+int spd_sample(spd_ctx *ctx, int32_t n_new, float top_p, float temperature, const float *uniforms, int32_t *out_new,
+               int32_t *out_ids, float *out_gamma) {
+  if (!ctx || !uniforms) return SPD_EINVAL;
+  if (!ctx->prefilled || ctx->n_gen != 1) return SPD_ESTATE;
+  const spd_config &c = ctx->cfg;
+  const int m = ctx->m;
+  if (n_new < 1 || m + n_new >= c.max_pos) return SPD_ERANGE;
+  if (!(top_p > 0.f) || top_p > 1.f || !(temperature > 0.f)) return SPD_ERANGE;
+  for (int i = 0; i < n_new; ++i)
+    if (!(uniforms[i] >= 0.f) || !(uniforms[i] < 1.f)) return SPD_ERANGE;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.ns_u, uniforms, (size_t)n_new * 4, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));  // the caller's array may go out of scope
+  ctx->prefilled = false;
+  // pass i draws token m + i from the logits of the pass before (the first from those the prefill left),
+  // feeds it at position m + i; the last pass ends with the first-timestep decision
+  spd::KParams &kp = ctx->kp;
+  int32_t *base = kp.prefix;
+  kp.prefix = base + m;
+  kp.ns_p = top_p;
+  kp.ns_inv_temp = 1.0f / temperature;
+  rc = launch(ctx, spd::kModeSample, n_new, m, 0);
+  kp.prefix = base;
+  if (rc) return rc;
+  std::vector<int32_t> fresh(n_new);
+  int32_t ids[SPD_MAX_K];
+  float gamma[SPD_MAX_K];
+  SPD_CUDA(cudaMemcpyAsync(fresh.data(), ctx->ws + ctx->lay.prefix + (size_t)m * 4, (size_t)n_new * 4, cudaMemcpyDeviceToHost,
+                           ctx->stream));
+  if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;
+  if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
+  if ((rc = check_device_error(ctx))) return rc;
+  ctx->prefix.insert(ctx->prefix.end(), fresh.begin(), fresh.end());
+  ctx->prefilled = true;
+  ctx->m = m + n_new;
+  ctx->n_gen = 1;
+  for (int i = 0; i < n_new; ++i)
+    if (out_new) out_new[i] = fresh[i];
+  for (int i = 0; i < c.k; ++i) {
     if (out_ids) out_ids[i] = ids[i];
     if (out_gamma) out_gamma[i] = gamma[i];
   }
@@ -608,6 +656,22 @@ int spd_debug_score(spd_ctx *ctx, const int32_t *hist, int32_t hist_len, const f
   ctx->prefilled = false;  // the draft state no longer belongs to a decoding run
   // launch() zeroes the head of the state only; the fields set above lie behind it
   if ((rc = launch(ctx, spd::kModeScoreOnly, 0, 0, 0))) return rc;
+  return spd_sync(ctx);
+}
+
+int spd_debug_nucleus(spd_ctx *ctx, const float *logits, float top_p, float temperature, float u, int32_t *out_token) {
+  if (!ctx || !logits || !out_token) return SPD_EINVAL;
+  if (!(top_p > 0.f) || top_p > 1.f || !(temperature > 0.f) || !(u >= 0.f) || !(u < 1.f)) return SPD_ERANGE;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.logits, logits, (size_t)ctx->cfg.vocab * 4, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.ns_u, &u, 4, cudaMemcpyHostToDevice, ctx->stream));
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));
+  ctx->prefilled = false;  // the logits no longer belong to a decoding run
+  ctx->kp.ns_p = top_p;
+  ctx->kp.ns_inv_temp = 1.0f / temperature;
+  if ((rc = launch(ctx, spd::kModeNucleusOnly, 0, 0, 0))) return rc;
+  if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), out_token, 4))) return rc;
   return spd_sync(ctx);
 }
 

@@ -20,6 +20,7 @@
 
 #include "spd_params.h"
 #include "spd_ptx.cuh"
+#include "spd_nucleus.cuh"
 
 namespace spd {
 
@@ -126,6 +127,7 @@ __device__ __forceinline__ void produce_matrix(Blk &b, Producer &pr, const __nv_
   }
 }
 
+template <bool kSampler>
 __device__ void producer_main(Blk &b) {
   const KParams &p = *b.p;
   Producer pr{0u, 0u, 0u};
@@ -137,7 +139,8 @@ __device__ void producer_main(Blk &b) {
       produce_matrix(b, pr, lw.wgate_up, 2 * p.f, p.d, 2);
       produce_matrix(b, pr, lw.wdown, p.d, p.f, 1);
     }
-    if (p.mode == kModeDecode || it == p.n_iters - 1) produce_matrix(b, pr, p.lm_head, p.V, p.d, 1);
+    const bool head = kSampler ? p.mode != kModePrefill : p.mode == kModeDecode;
+    if (head || it == p.n_iters - 1) produce_matrix(b, pr, p.lm_head, p.V, p.d, 1);
   }
   if (*b.dead) {
     // Giving up: nothing more is issued; wait (bounded) until every copy already issued has landed,
@@ -894,10 +897,12 @@ __device__ void tail_score_select(Blk &b, bool first, int step) {
   named_sync(1, kConsumerThreads);
 }
 
-// Next LM input (block 0): the token embedding in prefill, the superposed embedding of Eq. 3 in decode.
+// Next LM input (block 0): the token embedding in prefill and sampling, the superposed embedding of Eq. 3 in
+// decode.
+template <bool kSampler>
 __device__ void embed_input(const KParams &p, int it) {
   const State *st = p.st;
-  if (p.mode == kModePrefill) {
+  if (p.mode == kModePrefill || (kSampler && p.mode == kModeSample)) {
     const int tok = p.prefix[it];
     for (int c = threadIdx.x; c < p.d; c += kConsumerThreads) p.h[c] = __bfloat162float(p.tok_emb[(size_t)tok * p.d + c]);
   } else {
@@ -910,13 +915,35 @@ __device__ void embed_input(const KParams &p, int it) {
   }
 }
 
+// After the last sampled token's pass: every draft's history window is the end of the lengthened prefix
+// (p.prefix[it] is its last token, at position pos0 + it), as the host sets it up before a prefill.
+__device__ void sample_windows(const KParams &p, int it) {
+  State *st = p.st;
+  const int len = min(p.pos0 + it + 1, kWin);
+  if ((int)threadIdx.x < p.k)
+    for (int j = 0; j < len; ++j) st->win[threadIdx.x][kWin - len + j] = p.prefix[it - len + 1 + j];
+  if (threadIdx.x == 0) {
+    st->win_len = len;
+    st->n_gen = 0;
+  }
+}
+
 // ---------------------------------------------------------------- consumer main loop
+template <bool kSampler>
 __device__ void consumer_main(Blk &b) {
   const KParams &p = *b.p;
   float xr[kMaxVec][8];
   for (int it = 0; it < p.n_iters; ++it) {
     const int pos = p.pos0 + it;
-    if (blockIdx.x == 0) embed_input(p, it);
+    if (blockIdx.x == 0) {
+      if (kSampler && p.mode == kModeSample) {
+        // the next token is drawn from the logits of the pass before (Section 4.5: a nucleus-sampled prefix)
+        const int tok = ns_sample(p.logits, p.V, p.ns_inv_temp, p.ns_p, p.ns_u[it], reinterpret_cast<uint8_t *>(b.part));
+        if (threadIdx.x == 0) p.prefix[it] = tok;
+        named_sync(1, kConsumerThreads);
+      }
+      embed_input<kSampler>(p, it);
+    }
     if (grid_barrier(b)) return;
     for (int l = 0; l < p.L; ++l) {
       const LayerW lw = p.layers[l];
@@ -938,7 +965,8 @@ __device__ void consumer_main(Blk &b) {
       if (grid_barrier(b)) return;
     }
     const bool last = it == p.n_iters - 1;
-    if (p.mode == kModeDecode || last) {
+    const bool head = kSampler ? p.mode != kModePrefill : p.mode == kModeDecode;
+    if (head || last) {
       EpiArgs ea{0, pos, 0};
       prologue_norm(b, p.h, p.final_norm, p.d, xr);
       consume_matrix(b, p.V, p.d, 1, xr, kEpiLogits, ea);
@@ -947,16 +975,18 @@ __device__ void consumer_main(Blk &b) {
       cta_rows(p.V, 1, r0, r1);
       if (threadIdx.x < 32) block_topk(p, r0, r1);
       if (grid_barrier(b)) return;
-      if (blockIdx.x == 0) {
+      if (blockIdx.x == 0 && (!kSampler || p.mode != kModeSample || last)) {
         if (threadIdx.x < 32) tail_keep_topk(p);
-        const bool first = p.mode == kModePrefill;
+        const bool first = p.mode != kModeDecode;
+        if (kSampler && p.mode == kModeSample) sample_windows(p, it);
         tail_score_select(b, first, first ? 0 : p.step0 + it);
       }
     }
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) {
+template <bool kSampler>
+__device__ __forceinline__ void kernel_body(const KParams &p) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages];
   __shared__ float s_red[64];
@@ -987,29 +1017,51 @@ __global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_co
     if (blockIdx.x == 0 && threadIdx.x < kConsumerThreads) tail_score_select(b, false, p.step0);
     return;
   }
+  if (kSampler && p.mode == kModeNucleusOnly) {
+    if (blockIdx.x == 0 && threadIdx.x < kConsumerThreads) {
+      const int tok = ns_sample(p.logits, p.V, p.ns_inv_temp, p.ns_p, p.ns_u[0], reinterpret_cast<uint8_t *>(b.part));
+      if (threadIdx.x == 0) p.st->cand_tok[0] = tok;
+    }
+    return;
+  }
   if (threadIdx.x >= kConsumerThreads) {
-    if (threadIdx.x == kConsumerThreads) producer_main(b);
+    if (threadIdx.x == kConsumerThreads) producer_main<kSampler>(b);
   } else {
-    consumer_main(b);
+    consumer_main<kSampler>(b);
   }
   __syncthreads();
 }
 
+// The decoding kernel, and its twin that also carries the nucleus sampler (kModeSample, kModeNucleusOnly): two
+// entry points so that the sampler's code does not weigh on the register allocation of the decode loop.
+__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) { kernel_body<false>(p); }
+__global__ void __launch_bounds__(kThreads, 1) spd_sample_kernel(const __grid_constant__ KParams p) { kernel_body<true>(p); }
+
 }  // namespace spd
 
 // Host-side launcher used by the API file.
+static const void *kernel_for(int mode) {
+  return mode == spd::kModeSample || mode == spd::kModeNucleusOnly ? reinterpret_cast<const void *>(&spd::spd_sample_kernel)
+                                                                  : reinterpret_cast<const void *>(&spd::spd_decode_kernel);
+}
+
 extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size_t dyn_smem, cudaStream_t stream) {
   void *args[] = {const_cast<spd::KParams *>(p)};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&spd::spd_decode_kernel), dim3(grid), dim3(spd::kThreads),
-                                     args, dyn_smem, stream);
+  return cudaLaunchCooperativeKernel(kernel_for(p->mode), dim3(grid), dim3(spd::kThreads), args, dyn_smem, stream);
 }
 
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm) {
-  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_decode_kernel),
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
-  if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void *>(&spd::spd_decode_kernel),
-                                                       spd::kThreads, dyn_smem);
+  int least = 1 << 30;
+  for (int mode : {(int)spd::kModeDecode, (int)spd::kModeSample}) {
+    cudaError_t e = cudaFuncSetAttribute(kernel_for(mode), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
+    if (e != cudaSuccess) return e;
+    int n = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel_for(mode), spd::kThreads, dyn_smem);
+    if (e != cudaSuccess) return e;
+    if (n < least) least = n;
+  }
+  *blocks_per_sm = least;
+  return cudaSuccess;
 }
 
 // ---------------------------------------------------------------- scoring stage without any allocation

@@ -20,7 +20,7 @@ constexpr int kMaxVec = 4;          // 16-byte column vectors per thread: column
 constexpr int kMaxSplit = 8;        // attention splits per head
 constexpr int kPfTokens = 16;       // prefix tokens one prefill launch takes
 
-enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2 };
+enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2, kModeSample = 3, kModeNucleusOnly = 4 };
 
 struct LayerW {
   const __nv_bfloat16 *attn_norm, *wqkv, *wo, *ffn_norm, *wgate_up, *wdown;
@@ -76,12 +76,15 @@ struct KParams {
   float2 *pk_ms;             // [grid] (max of z/tau, sum of exp(z/tau - max))
   State *st;
   int32_t *hist_tok, *hist_par;  // [max_pos][k]
-  const int32_t *prefix;     // [max_pos]
+  int32_t *prefix;           // [max_pos]; kModeSample appends the sampled tokens
   float *trace;              // [L][2][d] or null
   float *pf_h, *pf_q;        // [kPfTokens][d] prefill: residual rows, rotated queries
   // prefill activations as mma fragments, three bf16 terms each: [ceil(C/16)][2][3][32] x 8 bytes
   uint16_t *pf_xh, *pf_xo;   // gain-scaled residual (C = d), attention output (C = d)
   uint16_t *pf_xu;           // SwiGLU output (C = f)
+  // nucleus sampling (kModeSample): one uniform number per sampled token
+  const float *ns_u;         // [max_pos]
+  float ns_p, ns_inv_temp;
   // launch
   int32_t mode, n_iters, pos0, step0;
   int32_t stage_bytes, n_stages;

@@ -63,10 +63,13 @@ def _sync_logp(ctx, orc, eps_z):
     orc.set_logP(lp)
 
 
-def compare_first_step(ctx, orc, prefix, stats=None, reset_draft=None):
+def compare_first_step(ctx, orc, prefix, stats=None, reset_draft=None, device=None):
     """First timestep on both sides.  With reset_draft, the restart from that draft (Section 5.3) instead: the
-    device recomputes only the generated positions, the oracle everything."""
-    if reset_draft is None:
+    device recomputes only the generated positions, the oracle everything.  With device = (ids, gamma), the
+    device has already taken its first timestep on `prefix` (after sampling its tail, Section 4.5)."""
+    if device is not None:
+        ids, g = device
+    elif reset_draft is None:
         ids, g = ctx.spd_prefill(prefix)
     else:
         prefix = orc.drafts()[reset_draft].tolist()
