@@ -244,6 +244,20 @@ def run_ours(args, wl):
         one = e0.elapsed_time(e1)
         kpass = {"ms_per_step_single_draft": one / K, "ms_per_step_k_passes": k * one / K, "ms_per_step_spd": ms / K,
                  "saving": k * one / ms, "note": "k sequential batch-1 passes (k=1 contexts, own KV cache) vs one superposed pass"}
+        if e2e_s:
+            # the paper's latency comparison (Section 4.3): k nucleus-sampled generations against one SPD request
+            u = np.linspace(0.05, 0.95, gen - 1).astype(np.float32)
+            ns_t = []
+            for _ in range(2):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                c1.spd_prefill(prefix)
+                c1.spd_sample(u, 0.9, 1.0)
+                ns_t.append(time.perf_counter() - t0)
+            kpass.update({"nucleus_ms_per_request": min(ns_t) * 1e3, "nucleus_k_requests_ms": k * min(ns_t) * 1e3,
+                          "spd_ms_per_request": e2e_s * 1e3, "request_saving": k * min(ns_t) / e2e_s,
+                          "nucleus_note": "prefill + %d nucleus-sampled passes (top-p 0.9, T 1) through spd_sample, host to "
+                                          "host; the draw of the last token (no pass) is not run" % (gen - 1)})
         c1.close()
 
     out = {

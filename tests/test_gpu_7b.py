@@ -93,3 +93,31 @@ def test_7b_tables_scoring_stage_with_hits(big):
         if np.min(-np.diff(srt)) > 1e-3:
             assert ctx.spd_debug_read("SEL").tolist() == want["sel"].tolist()
     assert hits >= 8
+
+
+def test_7b_nucleus_splice(big):
+    """Nucleus sampling at the full vocabulary (V = 32000) on the 7B-shape decoder's own, nearly flat, logits and
+    on colder ones, drawn one call at a time so that every draw is checked against the oracle's sampler; then
+    one launch of the same draws gives the same tokens, and the first timestep on prefix + sample agrees with
+    the oracle's dense prefill."""
+    from tests.test_gpu_nucleus import accepted, uniforms
+
+    wl, ctx, orc, tables, prefix = big
+    us = uniforms(6, 21)
+    for top_p, temperature in ((0.9, 1.0), (0.95, 0.02)):
+        ctx.spd_prefill(prefix)
+        seq, exact = list(prefix), 0
+        for u in us:
+            z = ctx.spd_debug_read("LOGITS")
+            new, ids, g = ctx.spd_sample([u], top_p, temperature)
+            want, ok = accepted(z, temperature, top_p, float(u))
+            assert int(new[0]) in ok
+            exact += int(new[0]) == want
+            seq.append(int(new[0]))
+        assert exact >= 4
+        z_last = ctx.spd_debug_read("LOGITS")
+        ctx.spd_prefill(prefix)
+        new_all, ids2, g2 = ctx.spd_sample(us, top_p, temperature)
+        assert new_all.tolist() == seq[len(prefix):] and ids2.tolist() == ids.tolist() and np.array_equal(g, g2)
+        assert np.array_equal(ctx.spd_debug_read("LOGITS"), z_last)
+    compare_first_step(ctx, orc, seq, None, device=(ids2, g2))
