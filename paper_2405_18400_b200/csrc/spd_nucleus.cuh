@@ -19,11 +19,14 @@
 namespace spd {
 
 constexpr int kNsBins = 64;
-constexpr float kNsOne = 1099511627776.f;  // 2^40
+constexpr int kNsBatch = 8;  // logits a thread loads before it looks at them
 
 struct NsShared {
-  unsigned long long bins[kConsumerWarps][kNsBins];
+  // per warp and digit: mass as two 20-bit halves (32-bit shared-memory atomics are native, 64-bit ones are
+  // not; a warp adds at most 2016 values below 2^20 to a cell) and count
+  unsigned int hi[kConsumerWarps][kNsBins], lo[kConsumerWarps][kNsBins];
   unsigned int cnts[kConsumerWarps][kNsBins];
+  unsigned long long park[3];   // values carried from the first search to the second
   unsigned long long tot[kNsBins];
   unsigned int ctot[kNsBins];
   // search state and results (thread 0 writes, everyone reads after a barrier)
@@ -43,8 +46,13 @@ __device__ __forceinline__ uint32_t ns_key(float z) {
   const uint32_t u = __float_as_uint(z + 0.f);  // -0 and +0 are one value
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
-__device__ __forceinline__ unsigned long long ns_mass(float z, float inv_t, float m) {
-  return __float2ull_rd(__expf(fmaf(z, inv_t, -m)) * kNsOne);
+// e = exp(z / T - max) in 2^-40 units, rounded down, as two 20-bit halves (e * 2^20 and the remainder * 2^20 are
+// exact in float32, so the halves are exact)
+__device__ __forceinline__ void ns_mass(float z, float inv_t, float m, unsigned int &hi, unsigned int &lo) {
+  const float e20 = __expf(fmaf(z, inv_t, -m)) * 1048576.f;
+  const float fh = floorf(e20);
+  hi = (unsigned int)fh;
+  lo = (unsigned int)((e20 - fh) * 1048576.f);
 }
 
 // Locates the first token (in the order above) whose running sum reaches s.target (>= 1): leaves its key in
@@ -57,34 +65,48 @@ __device__ void ns_search(NsShared &s, const float *logits, int V, float inv_t, 
   for (int pass = 0; pass < 6; ++pass) {
     const int width = pass < 5 ? 6 : 2, shift = 32 - decided - width;
     for (int i = tid; i < kConsumerWarps * kNsBins; i += kConsumerThreads) {
-      (&s.bins[0][0])[i] = 0ull;
+      (&s.hi[0][0])[i] = 0u;
+      (&s.lo[0][0])[i] = 0u;
       (&s.cnts[0][0])[i] = 0u;
     }
     named_sync(1, kConsumerThreads);
     const uint32_t prefix = s.prefix;
-    int cur = -1;
-    unsigned long long cur_q = 0ull;
-    unsigned int cur_c = 0u;
-    for (int r = tid; r < V; r += kConsumerThreads) {
-      const float z = __ldcg(logits + r);
-      const uint32_t key = ns_key(z);
-      if (decided == 0 || (key >> (32 - decided)) == prefix) {
-        const int d = (int)((key >> shift) & ((1u << width) - 1u));
-        if (d != cur) {
-          if (cur >= 0) {
-            atomicAdd(&s.bins[warp][cur], cur_q);
-            atomicAdd(&s.cnts[warp][cur], cur_c);
+    int cur = -1;  // a run of logits with one digit is summed in registers: at most 63 values of at most 2^20
+    unsigned int cur_hi = 0u, cur_lo = 0u, cur_c = 0u;
+    for (int r0 = tid; r0 < V; r0 += kNsBatch * kConsumerThreads) {
+      float zb[kNsBatch];  // a batch of loads in flight: the logits come from L2
+#pragma unroll
+      for (int e = 0; e < kNsBatch; ++e) {
+        const int r = r0 + e * kConsumerThreads;
+        zb[e] = r < V ? __ldcg(logits + r) : 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < kNsBatch; ++e) {
+        if (r0 + e * kConsumerThreads >= V) break;
+        const float z = zb[e];
+        const uint32_t key = ns_key(z);
+        if (decided == 0 || (key >> (32 - decided)) == prefix) {
+          const int d = (int)((key >> shift) & ((1u << width) - 1u));
+          if (d != cur) {
+            if (cur >= 0) {
+              atomicAdd(&s.hi[warp][cur], cur_hi + (cur_lo >> 20));
+              atomicAdd(&s.lo[warp][cur], cur_lo & 0xfffffu);
+              atomicAdd(&s.cnts[warp][cur], cur_c);
+            }
+            cur = d;
+            cur_hi = cur_lo = cur_c = 0u;
           }
-          cur = d;
-          cur_q = 0ull;
-          cur_c = 0u;
+          unsigned int h, l;
+          ns_mass(z, inv_t, m, h, l);
+          cur_hi += h;
+          cur_lo += l;
+          cur_c += 1u;
         }
-        cur_q += ns_mass(z, inv_t, m);
-        cur_c += 1u;
       }
     }
     if (cur >= 0) {
-      atomicAdd(&s.bins[warp][cur], cur_q);
+      atomicAdd(&s.hi[warp][cur], cur_hi + (cur_lo >> 20));
+      atomicAdd(&s.lo[warp][cur], cur_lo & 0xfffffu);
       atomicAdd(&s.cnts[warp][cur], cur_c);
     }
     named_sync(1, kConsumerThreads);
@@ -92,7 +114,7 @@ __device__ void ns_search(NsShared &s, const float *logits, int V, float inv_t, 
       unsigned long long q = 0ull;
       unsigned int c = 0u;
       for (int w = 0; w < kConsumerWarps; ++w) {
-        q += s.bins[w][tid];
+        q += ((unsigned long long)s.hi[w][tid] << 20) + s.lo[w][tid];
         c += s.cnts[w][tid];
       }
       s.tot[tid] = q;
@@ -143,7 +165,13 @@ __device__ __noinline__ int ns_sample(const float *logits, int V, float inv_t, f
   named_sync(1, kConsumerThreads);
   // largest logit
   float zm = -3.402823466e38f;
-  for (int r = tid; r < V; r += kConsumerThreads) zm = fmaxf(zm, __ldcg(logits + r));
+  for (int r0 = tid; r0 < V; r0 += kNsBatch * kConsumerThreads) {
+#pragma unroll
+    for (int e = 0; e < kNsBatch; ++e) {
+      const int r = r0 + e * kConsumerThreads;
+      if (r < V) zm = fmaxf(zm, __ldcg(logits + r));
+    }
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) zm = fmaxf(zm, __shfl_xor_sync(0xffffffffu, zm, o));
   float *wmax = reinterpret_cast<float *>(&s.tot[0]);
@@ -175,17 +203,16 @@ __device__ __noinline__ int ns_sample(const float *logits, int V, float inv_t, f
     unsigned long long t = mass ? __double2ull_rd((double)u * (double)mass) : 0ull;
     if (mass && t >= mass) t = mass - 1ull;
     // second search: first token whose running sum exceeds t
-    s.bins[0][0] = t;  // parked here across the search set-up below
-    s.tot[0] = take;
-    s.tot[1] = (unsigned long long)cut_key;
+    s.park[0] = t;
+    s.park[1] = take;
+    s.park[2] = (unsigned long long)cut_key;
     s.above = 0ull;
     s.prefix = 0u;
     s.target = t + 1ull;
   }
   named_sync(1, kConsumerThreads);
-  const unsigned long long t = s.bins[0][0], take = s.tot[0];
-  const uint32_t cut_key = (uint32_t)s.tot[1];
-  named_sync(1, kConsumerThreads);
+  const unsigned long long t = s.park[0], take = s.park[1];
+  const uint32_t cut_key = (uint32_t)s.park[2];
   ns_search(s, logits, V, inv_t, m, 0.f);
   // which of the logits equal to the located one: the j-th by ascending id
   const uint32_t hit_key = s.prefix;
@@ -199,7 +226,11 @@ __device__ __noinline__ int ns_sample(const float *logits, int V, float inv_t, f
   const int seg = (V + kConsumerThreads - 1) / kConsumerThreads;
   const int lo = tid * seg, hi = min(V, lo + seg);
   int mine = 0;
-  for (int r = lo; r < hi; ++r) mine += ns_key(__ldcg(logits + r)) == hit_key ? 1 : 0;
+  for (int r0 = lo; r0 < hi; r0 += kNsBatch) {
+#pragma unroll
+    for (int e = 0; e < kNsBatch; ++e)
+      if (r0 + e < hi) mine += ns_key(__ldcg(logits + r0 + e)) == hit_key ? 1 : 0;
+  }
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {

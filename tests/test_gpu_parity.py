@@ -76,6 +76,19 @@ def test_long_context_uses_split_attention(tiny_inputs):
     ctx.close()
 
 
+@pytest.mark.parametrize("m", [1, 2, 16, 17, 18, 33, 49])
+def test_prefill_chunk_boundaries(tiny_inputs, m):
+    """The batched prefill takes 16 prefix tokens per launch and leaves the last token to the decode kernel:
+    prefix lengths around those boundaries (none, one, a full launch, a launch of one token, several)."""
+    wl, _, _, _ = tiny_inputs
+    prefix = si.make_prefix("zipf", m, wl.shape.vocab, 1.1, seed=30 + m)
+    ctx, orc = make_tiny_pair(tiny_inputs)
+    compare_first_step(ctx, orc, prefix)
+    assert ctx.spd_launch_count() == 1 + (m - 1 + 15) // 16
+    compare_step(ctx, orc)
+    ctx.close()
+
+
 def test_odd_shape_model():
     """head_dim 96, d_ffn not a multiple of the thread count, vocabulary not divisible by the grid."""
     shape = si.ModelShape("odd", 1, 192, 2, 200, 1000)
