@@ -225,7 +225,7 @@ def run_ours(args, wl):
         e2e_s = max_over_ranks(e2e_s, dev, world)
     e2e = {"value": world * k * gen / e2e_s if e2e_s else None, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len / gen,
            "d2h_bytes_per_step": 12.0 * k, "what": "spd_prefill(host ids) + %d spd_step calls returning ids, parents and gamma "
-           "to the host, per request of %d tokens per draft; prefill = batched kernel over 16 tokens per launch + one decode-kernel pass for the last prefix token" % (gen - 1, gen),
+           "to the host, per request of %d tokens per draft; prefill = one launch of the batched kernel per 16 prefix tokens, the last one ending with the LM head and the first timestep" % (gen - 1, gen),
            "ms_per_request": e2e_s * 1e3 if e2e_s else None}
 
     # ---- the same number of drafts from k separate single-draft passes through the same kernels

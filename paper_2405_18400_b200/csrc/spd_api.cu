@@ -142,25 +142,26 @@ int check_device_error(spd_ctx *ctx) {
   return err[0];
 }
 
-// Bytes of the state's head that every launch zeroes: with `keep_err` the error words of earlier launches
-// of the same call survive (the first error sticks), else they are cleared too.
+// Bytes of the state's head that every launch zeroes: with `keep_err` (later launches of a multi-launch call)
+// the error words of the earlier launches survive (the first error sticks), else they are cleared too.
 size_t head_bytes(bool keep_err) { return keep_err ? offsetof(spd::State, err) : offsetof(spd::State, win_len); }
 
-int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0, bool keep_err = false) {
+int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0) {
   spd::KParams &kp = ctx->kp;
   kp.mode = mode;
   kp.n_iters = n_iters;
   kp.pos0 = pos0;
   kp.step0 = step0;
   // barrier counters, abort flag and error word start from zero at every launch
-  SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(keep_err), ctx->stream));
+  SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream));
   SPD_CUDA(spd_internal_launch(&kp, ctx->grid, ctx->dyn_smem, ctx->stream));
   ctx->launches += 1;
   return SPD_OK;
 }
 
-// Runs prefix tokens [first, first + count) (positions alike) through the prefill kernel, kPfTokens at a
-// time: their keys and values enter the cache, nothing else of the state changes.
+// Runs prefix tokens [first, first + count) (positions alike), the last of which ends the prefix, through the
+// prefill kernel, kPfTokens at a time: their keys and values enter the cache, and the last launch goes on to
+// the LM head on the prefix's last token and the first timestep (Eq. 1).
 int prefill_tokens(spd_ctx *ctx, int first, int count) {
   spd::KParams &kp = ctx->kp;
   int32_t *base = kp.prefix;
@@ -171,6 +172,7 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
     kp.n_iters = n;
     kp.pos0 = first + done;
     kp.step0 = 0;
+    kp.pf_head = done + n == count ? 1 : 0;
     kp.prefix = base + first + done;
     cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(done > 0), ctx->stream);
     if (e == cudaSuccess) e = spd_internal_prefill_launch(&kp, ctx->grid, ctx->stream);
@@ -178,16 +180,7 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
     else ctx->launches += 1;
   }
   kp.prefix = base;
-  return rc;
-}
-
-// The last prefix token (position `pos`): the decode kernel's single-token pass, which ends with the
-// first-timestep decision.
-int prefill_last(spd_ctx *ctx, int pos, bool keep_err) {
-  int32_t *base = ctx->kp.prefix;
-  ctx->kp.prefix = base + pos;
-  const int rc = launch(ctx, spd::kModePrefill, 1, pos, 0, keep_err);
-  ctx->kp.prefix = base;
+  kp.pf_head = 0;
   return rc;
 }
 
@@ -392,8 +385,7 @@ int spd_prefill(spd_ctx *ctx, const int32_t *prefix_ids, int32_t m, int32_t *out
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix, prefix_ids, (size_t)m * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));  // st and the caller's ids may go out of scope
   ctx->prefilled = false;
-  if ((rc = prefill_tokens(ctx, 0, m - 1))) return rc;
-  if ((rc = prefill_last(ctx, m - 1, m > 1))) return rc;
+  if ((rc = prefill_tokens(ctx, 0, m))) return rc;
   int32_t ids[SPD_MAX_K];
   float gamma[SPD_MAX_K];
   if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;
@@ -441,8 +433,7 @@ int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma) {
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix + (size_t)m * 4, seq.data(), (size_t)n * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));
   ctx->prefilled = false;
-  if ((rc = prefill_tokens(ctx, m, n - 1))) return rc;
-  if ((rc = prefill_last(ctx, m2 - 1, n > 1))) return rc;
+  if ((rc = prefill_tokens(ctx, m, n))) return rc;
   int32_t ids[SPD_MAX_K];
   float gamma[SPD_MAX_K];
   if ((rc = read_state(ctx, offsetof(spd::State, cand_tok), ids, sizeof ids))) return rc;

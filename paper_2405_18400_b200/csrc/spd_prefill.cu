@@ -19,6 +19,7 @@
 
 #include "spd_params.h"
 #include "spd_ptx.cuh"
+#include "spd_tail.cuh"
 
 namespace spd {
 
@@ -110,9 +111,14 @@ struct PfPhase {
   const __nv_bfloat16 *W;
   int R, C, gran;
 };
+__device__ __forceinline__ int pf_phases(const KParams &p) { return 4 * p.L + (p.pf_head ? 1 : 0); }
 __device__ __forceinline__ PfPhase pf_phase(const KParams &p, int ph) {
-  const LayerW &lw = p.layers[ph >> 2];
   PfPhase d;
+  if (ph == 4 * p.L) {  // the LM head, after the last layer
+    d.W = p.lm_head; d.R = p.V; d.C = p.d; d.gran = 1;
+    return d;
+  }
+  const LayerW &lw = p.layers[ph >> 2];
   switch (ph & 3) {
     case 0: d.W = lw.wqkv; d.R = 3 * p.d; d.C = p.d; d.gran = 2; break;
     case 1: d.W = lw.wo; d.R = p.d; d.C = p.d; d.gran = 1; break;
@@ -129,7 +135,7 @@ __device__ void pf_producer(PfBlk &b) {
   const int lane = threadIdx.x & 31;
   uint32_t stage = 0, phase = 0, issued = 0;
   bool ok = true;
-  for (int ph = 0; ph < 4 * p.L && ok; ++ph) {
+  for (int ph = 0; ph < pf_phases(p) && ok; ++ph) {
     const PfPhase pd = pf_phase(p, ph);
     int r0, r1;
     pf_rows(pd.R, pd.gran, r0, r1);
@@ -206,7 +212,7 @@ __device__ void pf_xproducer(PfBlk &b) {
   const KParams &p = *b.p;
   uint32_t n = 0;
   bool ok = true;
-  for (int ph = 0; ph < 4 * p.L && ok; ++ph) {
+  for (int ph = 0; ph < pf_phases(p) && ok; ++ph) {
     const PfPhase pd = pf_phase(p, ph);
     int r0, r1;
     pf_rows(pd.R, pd.gran, r0, r1);
@@ -269,13 +275,13 @@ __device__ __forceinline__ void pf_tile(float (&acc)[2][4], uint32_t base, const
   }
 }
 
-enum PfEpi { kPfQKV = 0, kPfAddH = 1, kPfSwiGLU = 2 };
+enum PfEpi { kPfQKV = 0, kPfAddH = 1, kPfSwiGLU = 2, kPfLogits = 3 };
 
 // One matrix for the 16 tokens: out[t][r] = scale_t * sum_c W[r][c] x[t][c] for this block's rows (x from the
 // phase's fragment buffer; scale_t = 1/rms of token t when `norm`, else 1), then the phase's epilogue.  `gain_next`
 // (kPfAddH): gain of the RMSNorm that reads the new residual next, or null when nothing does.
 __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const __nv_bfloat16 *gain_next,
-                        int layer, int pos0, int n_tok) {
+                        int layer, int which, int pos0, int n_tok) {
   const KParams &p = *b.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
   int r0, r1;
@@ -374,6 +380,12 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
             const float hn = __ldcg(h) + y;
             *h = hn;
             if (gain_next) pf_put(p.pf_xh, t, r, hn * __bfloat162float(gain_next[r]));
+            if (p.pf_head && t == n_tok - 1) {  // the prefix's last token: what the decode kernel would leave behind
+              if (p.trace) p.trace[((size_t)layer * 2 + which) * p.d + r] = hn;
+              if (layer == p.L - 1 && which == 1) p.h[r] = hn;
+            }
+          } else if (kind == kPfLogits) {
+            if (t == n_tok - 1) p.logits[r] = y;
           } else {
             if (!(row & 1)) pf_put(p.pf_xu, t, r >> 1, y / (1.f + __expf(-y)) * other);
           }
@@ -478,16 +490,32 @@ __device__ void pf_consumer(PfBlk &b) {
   if (pf_grid_barrier(b)) return;
   for (int l = 0; l < p.L; ++l) {
     const LayerW &lw = p.layers[l];
-    pf_gemm(b, pf_phase(p, 4 * l), true, kPfQKV, nullptr, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l), true, kPfQKV, nullptr, l, 0, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
     pf_attention(b, l, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_gemm(b, pf_phase(p, 4 * l + 1), false, kPfAddH, lw.ffn_norm, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l + 1), false, kPfAddH, lw.ffn_norm, l, 0, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_gemm(b, pf_phase(p, 4 * l + 2), true, kPfSwiGLU, nullptr, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l + 2), true, kPfSwiGLU, nullptr, l, 0, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_gemm(b, pf_phase(p, 4 * l + 3), false, kPfAddH, l + 1 < p.L ? p.layers[l + 1].attn_norm : nullptr, l, pos0, n_tok);
+    pf_gemm(b, pf_phase(p, 4 * l + 3), false, kPfAddH,
+            l + 1 < p.L ? p.layers[l + 1].attn_norm : (p.pf_head ? p.final_norm : nullptr), l, 1, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
+  }
+  if (p.pf_head) {
+    // the prefix ends here: logits of its last token, then the first timestep (Eq. 1) as in the decode kernel
+    pf_gemm(b, pf_phase(p, 4 * p.L), true, kPfLogits, nullptr, 0, 0, pos0, n_tok);
+    named_sync(1, kPfThreads);
+    int r0, r1;
+    pf_rows(p.V, 1, r0, r1);
+    if (threadIdx.x < 32) block_topk(p, r0, r1);
+    if (pf_grid_barrier(b)) return;
+    if (blockIdx.x == 0 && threadIdx.x < 32) {
+      tail_keep_topk(p);
+      tail_first(p, threadIdx.x, 0);
+      __syncwarp();
+      tail_gamma(p, threadIdx.x);
+    }
   }
 }
 

@@ -56,7 +56,7 @@ def test_one_launch_generate_equals_single_steps(tiny_inputs):
     assert toks.tolist() == hist
     assert np.array_equal(g, g2) and np.array_equal(lp, a.spd_debug_read("LOGP"))       # bit-identical
     assert np.array_equal(a.spd_debug_read("LOGITS"), b.spd_debug_read("LOGITS"))
-    pre = 1 + (len(prefix) - 1 + 15) // 16          # prefill: 16 tokens per launch, the last token on its own
+    pre = (len(prefix) + 15) // 16                  # prefill: 16 tokens per launch
     assert a.spd_launch_count() == pre + 6 and b.spd_launch_count() == pre + 1
     # and again from the start on the same context: prefill restarts it
     b.spd_prefill(prefix)
@@ -78,13 +78,13 @@ def test_long_context_uses_split_attention(tiny_inputs):
 
 @pytest.mark.parametrize("m", [1, 2, 16, 17, 18, 33, 49])
 def test_prefill_chunk_boundaries(tiny_inputs, m):
-    """The batched prefill takes 16 prefix tokens per launch and leaves the last token to the decode kernel:
-    prefix lengths around those boundaries (none, one, a full launch, a launch of one token, several)."""
+    """The batched prefill takes 16 prefix tokens per launch, the last launch ending with the LM head and the
+    first timestep: prefix lengths around those boundaries (one token, a full launch, one token over, several)."""
     wl, _, _, _ = tiny_inputs
     prefix = si.make_prefix("zipf", m, wl.shape.vocab, 1.1, seed=30 + m)
     ctx, orc = make_tiny_pair(tiny_inputs)
     compare_first_step(ctx, orc, prefix)
-    assert ctx.spd_launch_count() == 1 + (m - 1 + 15) // 16
+    assert ctx.spd_launch_count() == (m + 15) // 16
     compare_step(ctx, orc)
     ctx.close()
 
