@@ -37,7 +37,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, ns_u, pf_h, pf_q, pf_xh, pf_xo, pf_xu, total;
+      trace, ns_u, pf_h, pf_q, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, total;
 };
 
 bool valid_config(const spd_config *c) {
@@ -91,6 +91,9 @@ Layout make_layout(const spd_config &c, int grid) {
   L.ns_u = take((size_t)c.max_pos * 4);
   L.pf_h = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_q = take((size_t)spd::kPfTokens * c.d_model * 4);
+  L.pf_part = take((size_t)c.n_heads * 8 * spd::kPfTokens * hd * 4);
+  L.pf_ml = take((size_t)c.n_heads * 8 * spd::kPfTokens * sizeof(float2));
+  L.pf_cnt = take((size_t)c.n_heads * 2 * 4);
   L.pf_xh = take(frag_bytes(c.d_model));
   L.pf_xo = take(frag_bytes(c.d_model));
   L.pf_xu = take(frag_bytes(c.d_ffn));
@@ -316,6 +319,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.pf_h = reinterpret_cast<float *>(ws + lay.pf_h); kp.pf_q = reinterpret_cast<float *>(ws + lay.pf_q);
   kp.pf_xh = reinterpret_cast<uint16_t *>(ws + lay.pf_xh); kp.pf_xo = reinterpret_cast<uint16_t *>(ws + lay.pf_xo);
   kp.pf_xu = reinterpret_cast<uint16_t *>(ws + lay.pf_xu);
+  kp.pf_part = reinterpret_cast<float *>(ws + lay.pf_part); kp.pf_ml = reinterpret_cast<float2 *>(ws + lay.pf_ml);
+  kp.pf_cnt = reinterpret_cast<unsigned int *>(ws + lay.pf_cnt);
 
   // rotary table: cos / sin of pos * theta^(-2i/hd), evaluated in double and rounded once
   std::vector<float2> rope((size_t)cfg->max_pos * (hd / 2));
@@ -339,7 +344,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.state, 0, sizeof(spd::State), s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.trace, 0, (size_t)cfg->n_layers * 2 * cfg->d_model * 4, s);
   // columns past the row's end inside the last 16-column step of a fragment buffer are never written: zero
-  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.pf_xh, 0, lay.total - lay.pf_xh, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.pf_cnt, 0, lay.total - lay.pf_cnt, s);  // also the arrival counters
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return fail(cuda_fail(e, "workspace initialisation"));
   *out = ctx;

@@ -82,6 +82,11 @@ struct KParams {
   // prefill activations as mma fragments, three bf16 terms each: [ceil(C/16)][2][3][32] x 8 bytes
   uint16_t *pf_xh, *pf_xo;   // gain-scaled residual (C = d), attention output (C = d)
   uint16_t *pf_xu;           // SwiGLU output (C = f)
+  // prefill attention split over position ranges: per (head, token half, range) unnormalised sums and (max, sum),
+  // arrivals per (head, token half)
+  float *pf_part;            // [H * 2 * 8][8][hd]
+  float2 *pf_ml;             // [H * 2 * 8][8]
+  unsigned int *pf_cnt;      // [H * 2], zero between phases
   // nucleus sampling (kModeSample): one uniform number per sampled token
   const float *ns_u;         // [max_pos]
   float ns_p, ns_inv_temp;

@@ -39,6 +39,8 @@ constexpr int kPfXBufs = 1;                // shared-memory fragment buffers (th
 constexpr int kPfKStepBytes = 2 * 3 * 32 * 8;             // fragments of one k-step: [token tile][term][lane] x 8 bytes
 constexpr int kPfXBytes = kPfKSteps * kPfKStepBytes;      // one K block of fragments
 constexpr int kPfRedBytes = kPfWarps * kPfTileRows * kPfTokens * 4;
+constexpr int kPfMaxSplit = 8;              // attention: position ranges a head is split into
+constexpr int kPfAmFloats = 3 * kPfWarps * 8 + 2 * 8;  // attention item of 8 tokens: (max, sum, factor) per warp and token, merged (max, sum)
 constexpr unsigned long long kPfWaitNs = 1500ull * 1000ull * 1000ull;
 
 struct PfBlk {
@@ -47,9 +49,10 @@ struct PfBlk {
   uint8_t *xblk;  // kPfXBufs fragment buffers of kPfXBytes
   float *red;
   float *rs;      // [16] per-token 1/rms
-  float *am;      // [2][kPfWarps] attention merge: running max, running sum
+  float *am;      // attention merge scratch: kPfAmFloats floats
   uint64_t *full, *empty, *xfull, *xempty, *xgo;
   volatile int *dead, *quit;
+  int *last;      // attention: whether this block merges a head's splits
   unsigned int bar_target;
   uint32_t c_stage, c_phase;
   uint32_t x_n;  // fragment copies consumed so far: copy n sits in buffer n % kPfXBufs and is that buffer's use n / kPfXBufs
@@ -404,7 +407,7 @@ __device__ void pf_attention(PfBlk &b, int layer, int pos0, int n_tok) {
   const int epl = p.hd / 32;
   const float scale = 1.f / sqrtf((float)p.hd);
   float *s_acc = b.red;  // [warps][256]
-  float *s_m = b.am, *s_l = b.am + kPfWarps;
+  float *s_m = b.am, *s_l = b.am + kPfWarps;  // generic path: one (max, sum) per warp
   const int items = kPfTokens * p.H;
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int t = item / p.H, head = item - t * p.H;
@@ -474,6 +477,240 @@ __device__ void pf_attention(PfBlk &b, int layer, int pos0, int n_tok) {
   named_sync(1, kPfThreads);
 }
 
+// ---------------------------------------------------------------- attention, bf16 cache, head_dim <= 128
+// Item = (head, range of cached positions); all tokens of the chunk share every key / value row that is loaded.
+// A warp takes one position at a time: lane = EPL dims of the row; the 8 tokens of a sweep have their partial
+// dot products folded across the lanes so that lanes 4j..4j+3 end up with token j's score, keep its online
+// softmax state there, and hand the weights back to every lane for the weighted sum of values.
+template <int EPL>
+__device__ __forceinline__ void pf_load_row(const __nv_bfloat16 *src, float (&x)[EPL]) {
+  if (EPL == 4) {
+    const uint2 v = __ldcg(reinterpret_cast<const uint2 *>(src));
+    x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+    x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+  } else if (EPL == 2) {
+    const unsigned int v = __ldcg(reinterpret_cast<const unsigned int *>(src));
+    x[0] = __uint_as_float(v << 16); x[1] = __uint_as_float(v & 0xffff0000u);
+  } else {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e)
+      x[e] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short *>(src) + e) << 16);
+  }
+}
+
+// One warp, tokens t0..t0+7, positions lo + warp, lo + warp + 8, ... < hi.  Leaves (max, sum) of this lane's
+// token (lanes 4j..4j+3: token t0 + j) and the unnormalised weighted value sums of all 8 tokens for this lane's
+// dims.
+template <int EPL>
+__device__ __forceinline__ void pf_attn_sweep(const KParams &p, const __nv_bfloat16 *kbase, const __nv_bfloat16 *vbase, int lo,
+                                              int hi, int t0, int pos0, int n_tok, int head, float &m, float &l,
+                                              float (&acc)[8][EPL]) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float scale = 1.f / sqrtf((float)p.hd);
+  float q[8][EPL];
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      q[j][e] = t0 + j < n_tok ? __ldcg(p.pf_q + (size_t)(t0 + j) * p.d + head * p.hd + lane * EPL + e) * scale : 0.f;
+      acc[j][e] = 0.f;
+    }
+  const int mine = t0 + ((lane >> 2) & 7);
+  const int limit = mine < n_tok ? pos0 + mine : -1;  // last position this lane's token may look at
+  m = -CUDART_INF_F;
+  l = 0.f;
+  int tp = lo + warp;
+  float kn[EPL], vn[EPL];
+  if (tp < hi) {
+    pf_load_row<EPL>(kbase + (size_t)tp * p.d, kn);
+    pf_load_row<EPL>(vbase + (size_t)tp * p.d, vn);
+  }
+  for (; tp < hi; tp += kPfWarps) {
+    float kx[EPL], vx[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      kx[e] = kn[e];
+      vx[e] = vn[e];
+    }
+    if (tp + kPfWarps < hi) {  // next row's loads fly while this one is used
+      pf_load_row<EPL>(kbase + (size_t)(tp + kPfWarps) * p.d, kn);
+      pf_load_row<EPL>(vbase + (size_t)(tp + kPfWarps) * p.d, vn);
+    }
+    float d8[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      d8[j] = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) d8[j] = fmaf(q[j][e], kx[e], d8[j]);
+    }
+    // fold: 8 partial sums over 32 lanes -> lane holds the full sum of token (lane / 4) % 8
+    float d4[4], d2[2], sc;
+    {
+      const bool up = lane & 16;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float send = up ? d8[j] : d8[j + 4], keep = up ? d8[j + 4] : d8[j];
+        d4[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+      }
+    }
+    {
+      const bool up = lane & 8;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const float send = up ? d4[j] : d4[j + 2], keep = up ? d4[j + 2] : d4[j];
+        d2[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+      }
+    }
+    {
+      const bool up = lane & 4;
+      const float send = up ? d2[0] : d2[1], keep = up ? d2[1] : d2[0];
+      sc = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    sc += __shfl_xor_sync(0xffffffffu, sc, 2);
+    sc += __shfl_xor_sync(0xffffffffu, sc, 1);
+    const bool visible = tp <= limit;
+    const float mn = visible ? fmaxf(m, sc) : m;
+    const float c = mn == m ? 1.f : __expf(m - mn);
+    const float pw = visible ? __expf(sc - mn) : 0.f;
+    l = fmaf(l, c, pw);
+    m = mn;
+    if (__any_sync(0xffffffffu, c != 1.f)) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float cj = __shfl_sync(0xffffffffu, c, 4 * j);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[j][e] *= cj;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float pj = __shfl_sync(0xffffffffu, pw, 4 * j);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[j][e] = fmaf(pj, vx[e], acc[j][e]);
+    }
+  }
+}
+
+// Item = (head, 8 of the chunk's 16 tokens, range of positions).  Short contexts are not split by position
+// (the ranges' merge is not worth it); long ones are split as far as the grid has blocks for.
+template <int EPL>
+__device__ __forceinline__ void pf_attention_rows(const KParams *pp, float *am, float *red, int *last, int layer, int pos0,
+                                                  int n_tok) {
+  const KParams &p = *pp;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int T = pos0 + n_tok;  // positions in the cache after this chunk
+  int S = 1;
+  if (T >= 256) S = max(1, min(kPfMaxSplit, (int)gridDim.x / (2 * p.H)));
+  float *s_m = am, *s_l = am + kPfWarps * 8, *s_f = am + 2 * kPfWarps * 8;  // [warp][token]
+  float *s_M = am + 3 * kPfWarps * 8, *s_L = s_M + 8;                      // [token]
+  float *sum = red;                                                        // [8 tokens][hd] merged value sums
+  const int items = p.H * 2 * S;
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int head = item / (2 * S), half = (item / S) & 1, sp = item % S;
+    const int t0 = half * 8;
+    if (t0 >= n_tok) {  // no such tokens in this chunk: their attention output is zero
+      if (sp == 0)
+        for (int i = tid; i < 8 * p.hd; i += kPfThreads) pf_put(p.pf_xo, t0 + i / p.hd, head * p.hd + i % p.hd, 0.f);
+      continue;
+    }
+    const int lo = (int)((long long)T * sp / S), hi = (int)((long long)T * (sp + 1) / S);
+    const __nv_bfloat16 *kbase = reinterpret_cast<const __nv_bfloat16 *>(p.kcache) + (size_t)layer * p.max_pos * p.d + head * p.hd + lane * EPL;
+    const __nv_bfloat16 *vbase = reinterpret_cast<const __nv_bfloat16 *>(p.vcache) + (size_t)layer * p.max_pos * p.d + head * p.hd + lane * EPL;
+    float m, l, acc[8][EPL];
+    pf_attn_sweep<EPL>(p, kbase, vbase, lo, hi, t0, pos0, n_tok, head, m, l, acc);
+    named_sync(1, kPfThreads);  // scratch of the item before is no longer read
+    if ((lane & 3) == 0) {
+      s_m[warp * 8 + (lane >> 2)] = m;
+      s_l[warp * 8 + (lane >> 2)] = l;
+    }
+    named_sync(1, kPfThreads);
+    if (tid < kPfWarps * 8) {  // (warp w, token j): this warp's factor towards the block's maximum
+      const int j = tid & 7;
+      float M = -CUDART_INF_F;
+#pragma unroll
+      for (int w = 0; w < kPfWarps; ++w) M = fmaxf(M, s_m[w * 8 + j]);
+      s_f[tid] = s_m[tid] == -CUDART_INF_F ? 0.f : __expf(s_m[tid] - M);
+      if (tid < 8) {
+        float L = 0.f;
+#pragma unroll
+        for (int w = 0; w < kPfWarps; ++w) L = fmaf(s_l[w * 8 + j], s_m[w * 8 + j] == -CUDART_INF_F ? 0.f : __expf(s_m[w * 8 + j] - M), L);
+        s_M[j] = M;
+        s_L[j] = L;
+      }
+    }
+    named_sync(1, kPfThreads);
+    // the warps add their value sums one after the other: a fixed order
+    for (int w = 0; w < kPfWarps; ++w) {
+      if (warp == w) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float f = s_f[w * 8 + j];
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) {
+            float *dst = sum + (size_t)j * p.hd + lane * EPL + e;
+            *dst = (w == 0 ? 0.f : *dst) + acc[j][e] * f;
+          }
+        }
+      }
+      named_sync(1, kPfThreads);
+    }
+    if (S == 1) {
+      for (int i = tid; i < 8 * p.hd; i += kPfThreads) {
+        const int j = i / p.hd;
+        const float L = s_L[j];
+        pf_put(p.pf_xo, t0 + j, head * p.hd + i - j * p.hd, L > 0.f ? sum[i] / L : 0.f);
+      }
+    } else {
+      // partial result of this range to global memory; the block that completes the group merges its ranges
+      const int group = item / S;  // (head, half)
+      float *part = p.pf_part + (size_t)item * 8 * p.hd;
+      float2 *ml = p.pf_ml + (size_t)item * 8;
+      for (int i = tid; i < 8 * p.hd; i += kPfThreads) part[i] = sum[i];
+      if (tid < 8) ml[tid] = make_float2(s_M[tid], s_L[tid]);
+      __threadfence();
+      named_sync(1, kPfThreads);
+      if (tid == 0) {
+        const unsigned int seen = atomicAdd(p.pf_cnt + group, 1u);
+        *last = seen == (unsigned int)(S - 1);
+        if (*last) {
+          p.pf_cnt[group] = 0u;  // all ranges of this group have arrived: ready for the next layer
+          __threadfence();
+        }
+      }
+      named_sync(1, kPfThreads);
+      if (*last) {
+        const float *part0 = p.pf_part + (size_t)group * S * 8 * p.hd;
+        const float2 *ml0 = p.pf_ml + (size_t)group * S * 8;
+        for (int i = tid; i < 8 * p.hd; i += kPfThreads) {
+          const int j = i / p.hd;
+          float M = -CUDART_INF_F;
+          for (int r = 0; r < S; ++r) M = fmaxf(M, __ldcg(&ml0[(size_t)r * 8 + j]).x);
+          float L = 0.f, A = 0.f;
+          for (int r = 0; r < S; ++r) {
+            const float2 v = __ldcg(&ml0[(size_t)r * 8 + j]);
+            const float f = v.x == -CUDART_INF_F ? 0.f : __expf(v.x - M);
+            L = fmaf(v.y, f, L);
+            A = fmaf(__ldcg(&part0[(size_t)r * 8 * p.hd + i]), f, A);
+          }
+          pf_put(p.pf_xo, t0 + j, head * p.hd + i - j * p.hd, L > 0.f ? A / L : 0.f);
+        }
+      }
+    }
+    named_sync(1, kPfThreads);
+  }
+}
+
+// One dispatch on the head dimension.
+__device__ __forceinline__ void pf_attention_bf16(const KParams *pp, float *am, float *red, int *last, int layer, int pos0,
+                                               int n_tok) {
+  switch (pp->hd / 32) {
+    case 1: pf_attention_rows<1>(pp, am, red, last, layer, pos0, n_tok); break;
+    case 2: pf_attention_rows<2>(pp, am, red, last, layer, pos0, n_tok); break;
+    case 3: pf_attention_rows<3>(pp, am, red, last, layer, pos0, n_tok); break;
+    default: pf_attention_rows<4>(pp, am, red, last, layer, pos0, n_tok); break;
+  }
+}
+
 __device__ void pf_consumer(PfBlk &b) {
   const KParams &p = *b.p;
   const int n_tok = p.n_iters, pos0 = p.pos0;
@@ -492,7 +729,11 @@ __device__ void pf_consumer(PfBlk &b) {
     const LayerW &lw = p.layers[l];
     pf_gemm(b, pf_phase(p, 4 * l), true, kPfQKV, nullptr, l, 0, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
-    pf_attention(b, l, pos0, n_tok);
+    if (p.kv_bf16 && p.hd <= 128) {
+      pf_attention_bf16(b.p, b.am, b.red, b.last, l, pos0, n_tok);
+    } else {
+      pf_attention(b, l, pos0, n_tok);
+    }
     if (pf_grid_barrier(b)) return;
     pf_gemm(b, pf_phase(p, 4 * l + 1), false, kPfAddH, lw.ffn_norm, l, 0, pos0, n_tok);
     if (pf_grid_barrier(b)) return;
@@ -524,7 +765,8 @@ __device__ void pf_consumer(PfBlk &b) {
 __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_constant__ KParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t s_full[kPfStages], s_empty[kPfStages], s_xfull[kPfXBufs], s_xempty[kPfXBufs], s_xgo;
-  __shared__ float s_rs[kPfTokens], s_am[2 * kPfWarps];
+  __shared__ float s_rs[kPfTokens], s_am[kPfAmFloats];
+  __shared__ int s_last;
   __shared__ int s_dead, s_quit;
   PfBlk b;
   b.p = &p;
@@ -533,6 +775,7 @@ __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_consta
   b.red = reinterpret_cast<float *>(smem + (size_t)kPfStages * kPfStageBytes + (size_t)kPfXBufs * kPfXBytes);
   b.rs = s_rs;
   b.am = s_am;
+  b.last = &s_last;
   b.full = s_full;
   b.empty = s_empty;
   b.xfull = s_xfull;

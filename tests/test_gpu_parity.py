@@ -105,13 +105,14 @@ def test_odd_shape_model():
 
 def test_head_dim_128_long_context():
     """head_dim 128 with a bf16 cache takes the attention fast path (half a warp per position, eight positions
-    in flight per warp); a 300-token prefix spreads every head over several blocks and rounds."""
+    in flight per warp); a 300-token prefix spreads every head over several blocks and rounds, in the decode
+    kernel and in the prefill kernel (position ranges merged by the last block to arrive)."""
     shape = si.ModelShape("hd128", 2, 256, 2, 512, 1000)
     weights = si.make_weights(shape, seed=11)
     tables = si.make_ngram_tables(shape.vocab, 1.1, 50_000, (2, 3), 5000, seed=12)
     lam = [0.3, 0.2] + [0.0] * 6
     ctx, orc = make_pair(shape, weights, tables, 3, (2, 3), lam, 0.4, 0.2, 0.05, 512, "bf16")
-    for n in (1, 7, 300):
+    for n in (1, 7, 260, 300):     # 260 = 16 launches of 16 tokens + one of 4: a split prefill attention with an empty token half
         prefix = si.make_prefix("zipf", n, shape.vocab, 1.1, seed=13 + n)
         compare_first_step(ctx, orc, prefix)
         for _ in range(4):
