@@ -1,4 +1,5 @@
 // Host side of the C ABI declared in include/spd.h: argument checks, workspace layout, launches.
+#include <cuda.h>  // tensor-map types and the encoder's signature only; the entry point comes from the runtime
 #include <cuda_runtime.h>
 
 #include <cmath>
@@ -37,7 +38,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, ns_u, pf_h, pf_q, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, total;
+      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, total;
 };
 
 bool valid_config(const spd_config *c) {
@@ -89,6 +90,7 @@ Layout make_layout(const spd_config &c, int grid) {
   L.prefix = take((size_t)c.max_pos * 4);
   L.trace = take((size_t)c.n_layers * 2 * c.d_model * 4);
   L.ns_u = take((size_t)c.max_pos * 4);
+  L.pf_tmaps = take((size_t)(4 * c.n_layers + 1) * sizeof(CUtensorMap));
   L.pf_h = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_q = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_part = take((size_t)c.n_heads * 8 * spd::kPfTokens * hd * 4);
@@ -99,6 +101,22 @@ Layout make_layout(const spd_config &c, int grid) {
   L.pf_xu = take(frag_bytes(c.d_ffn));
   L.total = off;
   return L;
+}
+
+// Tensor map of a bf16 matrix [rows][cols] for the prefill kernel's tiled copies: boxes of 64 columns x 32 rows
+// (128 bytes per row), 128-byte shared-memory swizzle, zeros outside the matrix.
+using TensorMapEncode = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                     const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                     CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool weight_map(TensorMapEncode encode, const void *w, int rows, int cols, CUtensorMap *out) {
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64, 32};
+  const cuuint32_t step[2] = {1, 1};
+  return encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(w), dims, strides, box, step,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 constexpr int kLayoutGrid = 1024;  // workspace is sized for up to this many blocks
@@ -319,6 +337,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.pf_h = reinterpret_cast<float *>(ws + lay.pf_h); kp.pf_q = reinterpret_cast<float *>(ws + lay.pf_q);
   kp.pf_xh = reinterpret_cast<uint16_t *>(ws + lay.pf_xh); kp.pf_xo = reinterpret_cast<uint16_t *>(ws + lay.pf_xo);
   kp.pf_xu = reinterpret_cast<uint16_t *>(ws + lay.pf_xu);
+  kp.pf_tmaps = ws + lay.pf_tmaps;
   kp.pf_part = reinterpret_cast<float *>(ws + lay.pf_part); kp.pf_ml = reinterpret_cast<float2 *>(ws + lay.pf_ml);
   kp.pf_cnt = reinterpret_cast<unsigned int *>(ws + lay.pf_cnt);
 
@@ -338,8 +357,27 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
     layers[l].wgate_up = static_cast<const __nv_bfloat16 *>(w->wgate_up[l]);
     layers[l].wdown = static_cast<const __nv_bfloat16 *>(w->wdown[l]);
   }
+  // tensor maps of the matrices in the order the prefill kernel walks them
+  std::vector<CUtensorMap> tmaps((size_t)4 * cfg->n_layers + 1);
+  {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &found);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)"));
+    if (found != cudaDriverEntryPointSuccess || !fn) return fail(SPD_EINVAL);
+    const TensorMapEncode encode = reinterpret_cast<TensorMapEncode>(fn);
+    const int d = cfg->d_model, f = cfg->d_ffn;
+    bool ok = true;
+    for (int l = 0; l < cfg->n_layers && ok; ++l) {
+      ok = weight_map(encode, w->wqkv[l], 3 * d, d, &tmaps[4 * l]) && weight_map(encode, w->wo[l], d, d, &tmaps[4 * l + 1]) &&
+           weight_map(encode, w->wgate_up[l], 2 * f, d, &tmaps[4 * l + 2]) && weight_map(encode, w->wdown[l], d, f, &tmaps[4 * l + 3]);
+    }
+    ok = ok && weight_map(encode, w->lm_head, cfg->vocab, d, &tmaps[(size_t)4 * cfg->n_layers]);
+    if (!ok) return fail(SPD_EINVAL);
+  }
   cudaStream_t s = ctx->stream;
-  e = cudaMemcpyAsync(ws + lay.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s);
+  e = cudaMemcpyAsync(ws + lay.pf_tmaps, tmaps.data(), tmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + lay.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(ws + lay.layers, layers.data(), layers.size() * sizeof(spd::LayerW), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.state, 0, sizeof(spd::State), s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.trace, 0, (size_t)cfg->n_layers * 2 * cfg->d_model * 4, s);

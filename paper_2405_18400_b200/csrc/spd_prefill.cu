@@ -32,13 +32,16 @@ constexpr int kPfTileRows = 16;            // rows of one mma tile
 constexpr int kPfChunkRows = 32;           // rows of one ring stage: two tiles
 constexpr int kPfMaxTiles = 10;            // row tiles whose accumulators a warp keeps at a time
 constexpr int kPfMaxChunks = kPfMaxTiles / 2;
-constexpr int kPfPitch = kPfKB * 2 + 16;   // bytes between the rows of a chunk in a stage (padding: no bank conflicts)
-constexpr int kPfStageBytes = kPfChunkRows * kPfPitch;
+static_assert(kPfMaxTiles % 2 == 0, "a full group must end on the second partial-sum buffer");
+constexpr int kPfBoxCols = 64;             // one tensor-copy box: 32 rows x 64 columns = 32 x 128 bytes, 128-byte swizzle
+constexpr int kPfBoxBytes = kPfChunkRows * kPfBoxCols * 2;
+constexpr int kPfBoxes = kPfKB / kPfBoxCols;
+constexpr int kPfStageBytes = kPfBoxes * kPfBoxBytes;
 constexpr int kPfStages = 5;
 constexpr int kPfXBufs = 1;                // shared-memory fragment buffers (the consumers empty one into registers at once)
 constexpr int kPfKStepBytes = 2 * 3 * 32 * 8;             // fragments of one k-step: [token tile][term][lane] x 8 bytes
 constexpr int kPfXBytes = kPfKSteps * kPfKStepBytes;      // one K block of fragments
-constexpr int kPfRedBytes = kPfWarps * kPfTileRows * kPfTokens * 4;
+constexpr int kPfRedBytes = kPfWarps * kPfTileRows * kPfTokens * 4;  // one buffer of partial sums; there are two
 constexpr int kPfMaxSplit = 8;              // attention: position ranges a head is split into
 constexpr int kPfAmFloats = 3 * kPfWarps * 8 + 2 * 8;  // attention item of 8 tokens: (max, sum, factor) per warp and token, merged (max, sum)
 constexpr unsigned long long kPfWaitNs = 1500ull * 1000ull * 1000ull;
@@ -132,7 +135,19 @@ __device__ __forceinline__ PfPhase pf_phase(const KParams &p, int ph) {
 }
 
 // ---------------------------------------------------------------- producer
+// Tiled bulk copy of one box (64 columns x 32 rows at column x, row y of the matrix the tensor map describes)
+// into shared memory; rows and columns past the matrix arrive as zeros; completion is counted on `bar` in bytes.
+__device__ __forceinline__ void pf_box_load(void *dst, const void *tmap, int x, int y, uint64_t *bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                   smem_u32(dst)),
+               "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
+               : "memory");
+}
+
 // Chunk order of a phase: per group of up to kPfMaxTiles row tiles, K block by K block, chunk (32 rows) by chunk.
+// A chunk is 8 boxes, one per lane 0..7, in the 128-byte-swizzled layout that ldmatrix reads without bank
+// conflicts: box j of a stage holds columns 64 j .. 64 j + 63, row r of it lies at r * 128, and its 16-byte
+// unit u sits at unit u ^ (r % 8).
 __device__ void pf_producer(PfBlk &b) {
   const KParams &p = *b.p;
   const int lane = threadIdx.x & 31;
@@ -142,26 +157,24 @@ __device__ void pf_producer(PfBlk &b) {
     const PfPhase pd = pf_phase(p, ph);
     int r0, r1;
     pf_rows(pd.R, pd.gran, r0, r1);
-    const uint8_t *W = reinterpret_cast<const uint8_t *>(pd.W);
-    const size_t rowbytes = (size_t)pd.C * 2;
+    const uint8_t *tmap = reinterpret_cast<const uint8_t *>(p.pf_tmaps) + (size_t)ph * 128;
     const int nkb = (pd.C + kPfKB - 1) / kPfKB;
     for (int g0 = r0; g0 < r1 && ok; g0 += kPfMaxTiles * kPfTileRows) {
       const int g1 = min(g0 + kPfMaxTiles * kPfTileRows, r1);
       for (int kb = 0; kb < nkb && ok; ++kb) {
-        const uint32_t piece = (uint32_t)min(kPfKB, pd.C - kb * kPfKB) * 2u;
+        const int nbox = min(kPfBoxes, (pd.C - kb * kPfKB + kPfBoxCols - 1) / kPfBoxCols);  // boxes that touch the matrix
         for (int c0 = g0; c0 < g1 && ok; c0 += kPfChunkRows) {
-          const int nrows = min(kPfChunkRows, g1 - c0);
           int dead = 0;
           if (lane == 0) {
             pf_wait(b, &b.empty[stage], phase ^ 1u, 200);
             dead = *b.dead;
-            if (!dead) mbar_expect_tx(&b.full[stage], piece * (uint32_t)nrows);
+            if (!dead) mbar_expect_tx(&b.full[stage], (uint32_t)(nbox * kPfBoxBytes));
           }
           dead = __shfl_sync(0xffffffffu, dead, 0);
           if (dead) { ok = false; break; }
-          if (lane < nrows)
-            bulk_load(b.ring + (size_t)stage * kPfStageBytes + (size_t)lane * kPfPitch,
-                      W + (size_t)(c0 + lane) * rowbytes + (size_t)kb * kPfKB * 2, piece, &b.full[stage]);
+          if (lane < nbox)
+            pf_box_load(b.ring + (size_t)stage * kPfStageBytes + (size_t)lane * kPfBoxBytes, tmap, kb * kPfKB + lane * kPfBoxCols, c0,
+                        &b.full[stage]);
           if (issued < (uint32_t)kPfStages) ++issued;
           if (++stage == (uint32_t)kPfStages) { stage = 0; phase ^= 1u; }
         }
@@ -266,11 +279,11 @@ constexpr int kPfOwnSteps = kPfKSteps / kPfWarps;  // k-steps of a K block that 
 // One tile against this warp's k-steps of the K block: 16 rows x 16 columns of weights per k-step times the
 // three terms of both token tiles (fragments already in registers).  The two token tiles' accumulators
 // alternate so that consecutive mma do not depend on each other.
-__device__ __forceinline__ void pf_tile(float (&acc)[2][4], uint32_t base, const uint2 (&bb)[kPfOwnSteps][6], int warp) {
+__device__ __forceinline__ void pf_tile(float (&acc)[2][4], uint32_t base, const uint2 (&bb)[kPfOwnSteps][6]) {
 #pragma unroll
   for (int s = 0; s < kPfOwnSteps; ++s) {
     uint32_t a0, a1, a2, a3;
-    pf_ldsm_x4(base + (uint32_t)(warp + s * kPfWarps) * 32u, a0, a1, a2, a3);
+    pf_ldsm_x4(base + (uint32_t)s * (uint32_t)(kPfWarps / 4 * kPfBoxBytes), a0, a1, a2, a3);  // k-step warp + 8 s: two boxes on
 #pragma unroll
     for (int k = 0; k < 3; ++k)
 #pragma unroll
@@ -293,8 +306,10 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
   const int nkb = (pd.C + kPfKB - 1) / kPfKB;
   if (tid == 0) mbar_arrive(b.xgo);  // the grid barrier before this phase is behind us: its fragments are complete
   if (norm) pf_token_rms(b, p.pf_h, pd.C);
-  // ldmatrix addresses of this lane inside a tile: rows 0-7 / 8-15, columns k0 / k0+8
-  const uint32_t lane_off = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * kPfPitch + (uint32_t)(lane >> 4) * 16u;
+  // ldmatrix address of this lane for the warp's first k-step (k-step = warp) of a chunk's first tile: row
+  // (lane % 8) + 8 for the lower half of the tile, 16-byte unit 2 (k-step % 4) + (columns 8-15 ? 1 : 0), swizzled
+  const uint32_t l_row = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8);
+  const uint32_t lane_off = (uint32_t)(warp >> 2) * kPfBoxBytes + l_row * 128u + (((uint32_t)((warp & 3) * 2 + (lane >> 4)) ^ (l_row & 7u)) << 4);
   for (int g0 = r0; g0 < r1; g0 += kPfMaxTiles * kPfTileRows) {
     const int g1 = min(g0 + kPfMaxTiles * kPfTileRows, r1);
     float acc[kPfMaxTiles][2][4];
@@ -327,7 +342,7 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             const int i = 2 * j + h;
-            if (g0 + i * kPfTileRows < g1) pf_tile(acc[i], cbase + (uint32_t)(h * kPfTileRows * kPfPitch), bb, warp);
+            if (g0 + i * kPfTileRows < g1) pf_tile(acc[i], cbase + (uint32_t)(h * kPfTileRows * 128), bb);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&b.empty[b.c_stage]);
@@ -340,8 +355,9 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
     for (int i = 0; i < kPfMaxTiles; ++i) {
       if (g0 + i * kPfTileRows < g1) {
         const int t0 = g0 + i * kPfTileRows;
-        named_sync(1, kPfThreads);  // red[] free again
-        float *mine = b.red + warp * (kPfTileRows * kPfTokens);
+        // two buffers alternate: the barrier of the tile in between separates a buffer's readers from its next writers
+        float *red = b.red + (i & 1) * (kPfRedBytes / 4);
+        float *mine = red + warp * (kPfTileRows * kPfTokens);
         const int gr = lane >> 2, q = lane & 3;
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
@@ -354,7 +370,7 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
         const int row = tid >> 4, t = tid & 15;  // one thread per (row, token); rows r and r^1 sit 16 lanes apart
         float y = 0.f;
 #pragma unroll
-        for (int w = 0; w < kPfWarps; ++w) y += b.red[w * (kPfTileRows * kPfTokens) + row * kPfTokens + t];
+        for (int w = 0; w < kPfWarps; ++w) y += red[w * (kPfTileRows * kPfTokens) + row * kPfTokens + t];
         if (norm) y *= b.rs[t];
         const float other = __shfl_xor_sync(0xffffffffu, y, 16);
         const int r = t0 + row;
@@ -763,7 +779,9 @@ __device__ void pf_consumer(PfBlk &b) {
 // Nine warps leave one scheduler with three of them: 16384 registers / (3 x 32) caps a thread at 168, which
 // is what the compiler derives for a block of 384.
 __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_constant__ KParams p) {
-  extern __shared__ __align__(128) uint8_t smem[];
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  // the swizzle pattern of the tiled copies repeats every 1024 bytes of shared-memory address
+  uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   __shared__ uint64_t s_full[kPfStages], s_empty[kPfStages], s_xfull[kPfXBufs], s_xempty[kPfXBufs], s_xgo;
   __shared__ float s_rs[kPfTokens], s_am[kPfAmFloats];
   __shared__ int s_last;
@@ -801,8 +819,8 @@ __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_consta
     mbar_init(&s_xgo, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // rows of a last, short chunk that no copy writes are still multiplied (into rows nobody reads): the ring
-  // starts zeroed so that they hold finite values
+  // boxes wholly past a matrix's last column are never copied, yet every warp multiplies all its k-steps
+  // (against zero fragments there): the ring starts zeroed so that such boxes hold finite values
   for (size_t i = threadIdx.x; i < (size_t)kPfStages * kPfStageBytes / 16; i += blockDim.x)
     reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0u, 0u, 0u, 0u);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -821,7 +839,7 @@ __global__ void __launch_bounds__(384, 1) spd_prefill_kernel(const __grid_consta
 }  // namespace spd
 
 extern "C" size_t spd_internal_prefill_smem(void) {
-  return (size_t)spd::kPfStages * spd::kPfStageBytes + (size_t)spd::kPfXBufs * spd::kPfXBytes + spd::kPfRedBytes;
+  return (size_t)spd::kPfStages * spd::kPfStageBytes + (size_t)spd::kPfXBufs * spd::kPfXBytes + 2 * spd::kPfRedBytes + 1024;  // + alignment slack
 }
 
 extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm) {
