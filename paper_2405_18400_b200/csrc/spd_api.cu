@@ -38,7 +38,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, total;
+      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, total;
 };
 
 bool valid_config(const spd_config *c) {
@@ -93,6 +93,7 @@ Layout make_layout(const spd_config &c, int grid) {
   L.pf_tmaps = take((size_t)(4 * c.n_layers + 1) * sizeof(CUtensorMap));
   L.pf_h = take((size_t)spd::kPfTokens * c.d_model * 4);
   L.pf_q = take((size_t)spd::kPfTokens * c.d_model * 4);
+  L.pf_ss = take((size_t)grid * spd::kPfTokens * 4);
   L.pf_part = take((size_t)c.n_heads * 8 * spd::kPfTokens * hd * 4);
   L.pf_ml = take((size_t)c.n_heads * 8 * spd::kPfTokens * sizeof(float2));
   L.pf_cnt = take((size_t)c.n_heads * 2 * 4);
@@ -338,6 +339,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.pf_xh = reinterpret_cast<uint16_t *>(ws + lay.pf_xh); kp.pf_xo = reinterpret_cast<uint16_t *>(ws + lay.pf_xo);
   kp.pf_xu = reinterpret_cast<uint16_t *>(ws + lay.pf_xu);
   kp.pf_tmaps = ws + lay.pf_tmaps;
+  kp.pf_ss = reinterpret_cast<float *>(ws + lay.pf_ss);
   kp.pf_part = reinterpret_cast<float *>(ws + lay.pf_part); kp.pf_ml = reinterpret_cast<float2 *>(ws + lay.pf_ml);
   kp.pf_cnt = reinterpret_cast<unsigned int *>(ws + lay.pf_cnt);
 

@@ -79,6 +79,7 @@ struct KParams {
   int32_t *prefix;           // [max_pos]; kModeSample appends the sampled tokens
   float *trace;              // [L][2][d] or null
   float *pf_h, *pf_q;        // [kPfTokens][d] prefill: residual rows, rotated queries
+  float *pf_ss;              // [grid][kPfTokens] per block: sums of squares of the residual values it produced
   const void *pf_tmaps;      // [4 L + 1] tensor maps (128 bytes each) of the layers' matrices and the LM head, for the prefill's tiled copies
   // prefill activations as mma fragments, three bf16 terms each: [ceil(C/16)][2][3][32] x 8 bytes
   uint16_t *pf_xh, *pf_xo;   // gain-scaled residual (C = d), attention output (C = d)

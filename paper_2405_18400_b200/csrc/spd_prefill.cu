@@ -257,21 +257,33 @@ __device__ void pf_xproducer(PfBlk &b) {
   }
 }
 
-// Per-token 1/rms of the residual rows (every block computes all 16; rows past n_tok are zero).
-__device__ void pf_token_rms(PfBlk &b, const float *H, int d) {
+// Per-token 1/rms of the residual rows from the blocks' partial sums of squares (each block publishes the sums
+// over the rows or columns it produced; added here in a fixed order).
+__device__ void pf_token_rms(PfBlk &b, int d) {
+  const KParams &p = *b.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int t = warp; t < kPfTokens; t += kPfWarps) {
     float ss = 0.f;
-#pragma unroll 8
-    for (int c = lane * 4; c < d; c += 128) {
-      const float4 v = __ldcg(reinterpret_cast<const float4 *>(H + (size_t)t * d + c));
-      ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
-    }
+    for (int blk = lane; blk < (int)gridDim.x; blk += 32) ss += __ldcg(p.pf_ss + (size_t)blk * kPfTokens + t);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    if (lane == 0) b.rs[t] = rsqrtf(ss / (float)d + b.p->eps);
+    if (lane == 0) b.rs[t] = rsqrtf(ss / (float)d + p.eps);
   }
   named_sync(1, kPfThreads);
+}
+
+// Publishes this block's sums of squares: thread (slot = tid / 16, token = tid % 16) brings the sum over the
+// residual values of its token that it produced.
+__device__ void pf_publish_ss(PfBlk &b, float ssq) {
+  named_sync(1, kPfThreads);  // the scratch is no longer read
+  b.red[threadIdx.x] = ssq;
+  named_sync(1, kPfThreads);
+  if (threadIdx.x < kPfTokens) {
+    float s = 0.f;
+#pragma unroll
+    for (int r = 0; r < kPfThreads / kPfTokens; ++r) s += b.red[r * kPfTokens + threadIdx.x];
+    b.p->pf_ss[(size_t)blockIdx.x * kPfTokens + threadIdx.x] = s;
+  }
 }
 
 constexpr int kPfOwnSteps = kPfKSteps / kPfWarps;  // k-steps of a K block that one warp multiplies
@@ -305,7 +317,8 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
   const int nks_total = (pd.C + 15) / 16;
   const int nkb = (pd.C + kPfKB - 1) / kPfKB;
   if (tid == 0) mbar_arrive(b.xgo);  // the grid barrier before this phase is behind us: its fragments are complete
-  if (norm) pf_token_rms(b, p.pf_h, pd.C);
+  if (norm) pf_token_rms(b, pd.C);
+  float ssq = 0.f;  // kPfAddH: sum of squares of the residual values this thread produces (its token = tid % 16)
   // ldmatrix address of this lane for the warp's first k-step (k-step = warp) of a chunk's first tile: row
   // (lane % 8) + 8 for the lower half of the tile, 16-byte unit 2 (k-step % 4) + (columns 8-15 ? 1 : 0), swizzled
   const uint32_t l_row = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8);
@@ -398,6 +411,7 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
             float *h = p.pf_h + (size_t)t * p.d + r;
             const float hn = __ldcg(h) + y;
             *h = hn;
+            ssq = fmaf(hn, hn, ssq);
             if (gain_next) pf_put(p.pf_xh, t, r, hn * __bfloat162float(gain_next[r]));
             if (p.pf_head && t == n_tok - 1) {  // the prefix's last token: what the decode kernel would leave behind
               if (p.trace) p.trace[((size_t)layer * 2 + which) * p.d + r] = hn;
@@ -412,6 +426,7 @@ __device__ void pf_gemm(PfBlk &b, const PfPhase &pd, bool norm, int kind, const 
       }
     }
   }
+  if (kind == kPfAddH) pf_publish_ss(b, ssq);
 }
 
 // Causal attention of the chunk's tokens over the cache: one (token, head) item per block at a time, a warp
@@ -730,15 +745,19 @@ __device__ __forceinline__ void pf_attention_bf16(const KParams *pp, float *am, 
 __device__ void pf_consumer(PfBlk &b) {
   const KParams &p = *b.p;
   const int n_tok = p.n_iters, pos0 = p.pos0;
-  // residual rows start as the tokens' embeddings (zeros past n_tok)
+  // residual rows start as the tokens' embeddings (zeros past n_tok); a block takes a range of columns
   {
     const __nv_bfloat16 *gain0 = p.layers[0].attn_norm;
-    for (int i = blockIdx.x * kPfThreads + threadIdx.x; i < kPfTokens * p.d; i += gridDim.x * kPfThreads) {
-      const int t = i / p.d, c = i - t * p.d;
+    const int c0 = (int)((long long)p.d * blockIdx.x / gridDim.x), c1 = (int)((long long)p.d * (blockIdx.x + 1) / gridDim.x);
+    const int t = threadIdx.x & 15;
+    float ssq = 0.f;
+    for (int c = c0 + (threadIdx.x >> 4); c < c1; c += kPfThreads / kPfTokens) {
       const float v = t < n_tok ? __bfloat162float(p.tok_emb[(size_t)p.prefix[t] * p.d + c]) : 0.f;
-      p.pf_h[i] = v;
+      p.pf_h[(size_t)t * p.d + c] = v;
       pf_put(p.pf_xh, t, c, v * __bfloat162float(gain0[c]));
+      ssq = fmaf(v, v, ssq);
     }
+    pf_publish_ss(b, ssq);
   }
   if (pf_grid_barrier(b)) return;
   for (int l = 0; l < p.L; ++l) {

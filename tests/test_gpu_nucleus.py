@@ -140,3 +140,47 @@ def test_one_launch_equals_single_draws(tiny_inputs):
     ta, _, _ = a.spd_generate(5, 6)
     tb, _, _ = b.spd_generate(5, 6)
     assert ta.tolist() == tb.tolist()
+
+
+def test_n_sampled_prefixes_times_k_drafts(tiny_inputs):
+    """NS_SPDk (Section 4.5): n nucleus-sampled continuations of one prefix, each extended by k superposed
+    drafts, from n contexts over the same weights and tables.  Interleaving the contexts' calls changes nothing:
+    each gives what it gives alone, and different random numbers give different continuations."""
+    import paper_2405_18400_b200 as P
+
+    wl, weights, tables, prefix = tiny_inputs
+    packed = P.pack_weights(weights, "cuda:0")
+    dtabs = P.build_ngram_tables(tables, "cuda:0")
+    n, k, n_new, steps = 3, wl.k, 5, 4
+
+    def make():
+        return P.SpdContext(wl.shape, packed, dtabs, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, wl.max_pos, "bf16")
+
+    us = [uniforms(n_new, 100 + i) for i in range(n)]
+    alone = []
+    for i in range(n):
+        c = make()
+        c.spd_prefill(prefix)
+        new, _, _ = c.spd_sample(us[i], 0.9, 0.3)
+        toks, lp, g = c.spd_generate(steps, steps + 1)
+        alone.append((new.tolist(), toks.tolist(), lp.tolist()))
+        c.close()
+    ctxs = [make() for _ in range(n)]
+    for c in ctxs:
+        c.spd_prefill(prefix)
+    news, hist = [], []
+    for i, c in enumerate(ctxs):
+        new, ids, _ = c.spd_sample(us[i], 0.9, 0.3)
+        news.append(new.tolist())
+        hist.append([[int(t)] for t in ids])
+    for _ in range(steps):                      # one step of every context in turn
+        for i, c in enumerate(ctxs):
+            ids, par, _ = c.spd_step()
+            hist[i] = [hist[i][int(par[r])] + [int(ids[r])] for r in range(k)]
+    for i, c in enumerate(ctxs):
+        assert news[i] == alone[i][0] and hist[i] == alone[i][1]
+        assert c.spd_debug_read("LOGP").tolist() == alone[i][2]
+        c.close()
+    assert len({tuple(a[0]) for a in alone}) > 1
+    drafts = {tuple(row) for a in alone for row in a[1]}
+    assert len(drafts) >= n * k - 1             # n k drafts, (nearly) all distinct
