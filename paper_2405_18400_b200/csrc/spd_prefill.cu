@@ -1,19 +1,21 @@
-// Prefill kernel: the decoder over up to 16 prefix tokens at once (first timestep, Eq. 1, all but the last
-// prefix token; the last one goes through the decode kernel, which also takes the first-timestep
-// decision).  With several tokens per weight the products are real matrix-matrix contractions, so they run
-// on tensor cores: mma.sync m16n8k16 with A = 16 weight rows x 16 columns straight from the bf16 rows,
-// B = the tokens' activations split exactly into three bf16 terms (x = hi + mid + lo to float32
-// precision), float32 accumulation.
+// Prefill kernel: the decoder over up to 16 prefix tokens at once, and, in the launch that holds the prefix's
+// last token, the LM head on that token and the first timestep (Eq. 1).  With several tokens per weight the
+// products are real matrix-matrix contractions, so they run on tensor cores: mma.sync m16n8k16 with A = 16
+// weight rows x 16 columns straight from the bf16 rows, B = the tokens' activations split exactly into three
+// bf16 terms (x = hi + mid + lo to float32 precision), float32 accumulation.
 //
 // One persistent cooperative launch per chunk of tokens.  Per block: a producer warp streams the block's
-// weight rows (chunks of 32 rows x 512 columns) through a shared-memory ring with bulk copies; eight
-// consumer warps share every chunk by k-steps; per-warp partial sums meet in shared memory once per 16
-// rows.  Activations travel between phases already split and laid out as mma B fragments: the epilogue
-// that produces a value writes its three bf16 terms into a fragment buffer in global memory, and in the next
-// phase a second producer warp pulls 512 columns of all 16 tokens (48 KB) at a time into shared memory with
-// one bulk copy; each consumer warp takes its k-steps' fragments into registers at once, which frees the
-// buffer for the next K block while the current one is multiplied.  No block repeats the conversion.  RMSNorm's gain is applied before the split, its per-token 1/rms after the product
-// (it is a scalar per token).  The five phases per layer are separated by grid barriers as in decoding.
+// weight rows (chunks of 32 rows x 512 columns = 8 tiled TMA copies in the 128-byte-swizzled layout that
+// ldmatrix reads without bank conflicts) through a shared-memory ring; eight consumer warps share every chunk
+// by k-steps and keep the accumulators of up to 10 row tiles in registers, so that a block's rows of a matrix
+// are streamed once; per-warp partial sums meet in shared memory once per 16 rows.  Activations travel
+// between phases already split and laid out as mma B fragments: the epilogue that produces a value writes its
+// three bf16 terms into a fragment buffer in global memory, and in the next phase a second producer warp pulls
+// 512 columns of all 16 tokens (48 KB) at a time into shared memory with one bulk copy; each consumer warp
+// takes its k-steps' fragments into registers at once, which frees the buffer for the next K block while the
+// current one is multiplied.  No block repeats the conversion.  RMSNorm's gain is applied before the split,
+// its per-token 1/rms (from per-block partial sums of squares) after the product: it is a scalar per token.
+// The five phases per layer are separated by grid barriers as in decoding; every wait is bounded.
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
