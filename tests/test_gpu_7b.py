@@ -39,6 +39,9 @@ def test_7b_steps_match_oracle(big):
     compare_first_step(ctx, orc, prefix, stats)
     for _ in range(4):
         compare_step(ctx, orc, stats)
+    # restart from the second draft (Section 5.3): the batched prefill recomputes the five generated positions
+    compare_first_step(ctx, orc, None, stats, reset_draft=1)
+    compare_step(ctx, orc, stats)
     errs = [s for s in stats if "eps_z" in s]
     assert max(s["eps_z"] for s in errs) < 2e-3
     flips = sum(s.get("cache_flips", 0) for s in stats)
