@@ -259,6 +259,14 @@ int spd_score_static(const spd_config *cfg, const spd_ngram_table *tables, int32
                      int32_t hist_len, const float *logp, const int32_t *cand_tok, const float *cand_lp,
                      int32_t *out_sel, float *out_logp, float *out_gamma, float *out_score);
 
+/*
+ * Test hook for the bounded device waits: launches the prefill kernel on one token with one block withholding
+ * its arrival at the first grid barrier, so that the other blocks' waits (1.5 s) run out.  The kernel then
+ * ends by itself (every block gives up, drains its copies in flight and returns) and the call returns what the
+ * device recorded, which must be SPD_ETIMEOUT.  The context stays usable: prefill it again.
+ */
+int spd_debug_expire(spd_ctx *ctx);
+
 /* Number of kernel launches this context has enqueued so far. */
 int64_t spd_launch_count(const spd_ctx *ctx);
 

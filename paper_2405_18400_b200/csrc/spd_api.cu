@@ -711,4 +711,25 @@ int spd_debug_nucleus(spd_ctx *ctx, const float *logits, float top_p, float temp
   return spd_sync(ctx);
 }
 
+int spd_debug_expire(spd_ctx *ctx) {
+  if (!ctx) return SPD_EINVAL;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  ctx->prefilled = false;
+  SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.prefix, 0, 4, ctx->stream));  // token 0 at position 0
+  ctx->kp.pf_stall = 1;
+  spd::KParams &kp = ctx->kp;
+  kp.mode = spd::kModePrefill;
+  kp.n_iters = 1;
+  kp.pos0 = 0;
+  kp.step0 = 0;
+  kp.pf_head = 0;
+  cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream);
+  if (e == cudaSuccess) e = spd_internal_prefill_launch(&kp, ctx->grid, ctx->stream);
+  kp.pf_stall = 0;
+  if (e != cudaSuccess) return cuda_fail(e, "prefill launch");
+  ctx->launches += 1;
+  return check_device_error(ctx);
+}
+
 }  // extern "C"

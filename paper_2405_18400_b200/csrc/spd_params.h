@@ -94,6 +94,7 @@ struct KParams {
   float ns_p, ns_inv_temp;
   // launch
   int32_t mode, n_iters, pos0, step0;
+  int32_t pf_stall;          // prefill kernel, test hook: block 0 withholds its arrival at the grid barriers
   int32_t pf_head;           // prefill kernel: the launch ends the prefix: LM head on its last token and first timestep
   int32_t stage_bytes, n_stages;
 };

@@ -93,7 +93,7 @@ __device__ __forceinline__ bool pf_grid_barrier(PfBlk &b) {
     if (!*b.dead) {
       unsigned int *bar = &b.p->st->bar;
       __threadfence();
-      atomicAdd(bar, 1u);
+      if (!(b.p->pf_stall && blockIdx.x == 0)) atomicAdd(bar, 1u);  // the test hook's missing arrival: every wait runs out
       unsigned long long t0 = globaltimer();
       uint32_t n = 0;
       while ((int)(ld_acquire(bar) - b.bar_target) < 0) {

@@ -320,3 +320,29 @@ def test_malformed_table_is_reported_not_hung(tiny_inputs):
     ids, par, g = ok.spd_step()
     assert abs(float(g.sum()) - 1) < 1e-5
     ok.close()
+
+
+def test_expired_wait_is_reported_and_the_context_stays_usable(tiny_inputs):
+    """One block withholds its arrival at a grid barrier of the prefill kernel: every other block's bounded wait
+    runs out, the kernel ends by itself, the host reads SPD_ETIMEOUT, and the same context then decodes as a fresh
+    one does."""
+    import time
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, _ = make_tiny_pair(tiny_inputs)
+    ref, _ = make_tiny_pair(tiny_inputs)
+    ids0, g0 = ref.spd_prefill(prefix)
+    t0 = time.perf_counter()
+    status = ctx.spd_debug_expire()
+    dt = time.perf_counter() - t0
+    assert status == -7
+    assert 1.0 < dt < 10.0
+    import paper_2405_18400_b200 as P
+    with pytest.raises(P.SpdError) as e:            # no drafts to continue
+        ctx.spd_step()
+    assert e.value.status == -2
+    ids, g = ctx.spd_prefill(prefix)
+    assert ids.tolist() == ids0.tolist() and np.array_equal(g, g0)
+    a, _, _ = ctx.spd_generate(4, 5)
+    b, _, _ = ref.spd_generate(4, 5)
+    assert a.tolist() == b.tolist()
+    ctx.close(); ref.close()
