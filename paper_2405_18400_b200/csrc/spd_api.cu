@@ -120,6 +120,8 @@ bool weight_map(TensorMapEncode encode, const void *w, int rows, int cols, CUten
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+static_assert(sizeof(CUtensorMap) == spd::kTensorMapBytes, "the prefill kernel steps through the tensor maps by this size");
+
 constexpr int kLayoutGrid = 1024;  // workspace is sized for up to this many blocks
 
 }  // namespace

@@ -18,6 +18,7 @@ constexpr int kMaxRowsPerChunk = 8;
 constexpr int kMaxStages = 16;
 constexpr int kMaxVec = 4;          // 16-byte column vectors per thread: columns <= 4 * 512 * 8
 constexpr int kMaxSplit = 8;        // attention splits per head
+constexpr int kTensorMapBytes = 128; // size of one tensor map object (CUtensorMap)
 constexpr int kPfTokens = 16;       // prefix tokens one prefill launch takes
 
 enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2, kModeSample = 3, kModeNucleusOnly = 4 };

@@ -159,7 +159,7 @@ __device__ void pf_producer(PfBlk &b) {
     const PfPhase pd = pf_phase(p, ph);
     int r0, r1;
     pf_rows(pd.R, pd.gran, r0, r1);
-    const uint8_t *tmap = reinterpret_cast<const uint8_t *>(p.pf_tmaps) + (size_t)ph * 128;
+    const uint8_t *tmap = reinterpret_cast<const uint8_t *>(p.pf_tmaps) + (size_t)ph * kTensorMapBytes;
     const int nkb = (pd.C + kPfKB - 1) / kPfKB;
     for (int g0 = r0; g0 < r1 && ok; g0 += kPfMaxTiles * kPfTileRows) {
       const int g1 = min(g0 + kPfMaxTiles * kPfTileRows, r1);
