@@ -259,7 +259,8 @@ def run_ours(args, wl):
             kpass.update({"nucleus_ms_per_request": min(ns_t) * 1e3, "nucleus_k_requests_ms": k * min(ns_t) * 1e3,
                           "spd_ms_per_request": e2e_s * 1e3, "request_saving": k * min(ns_t) / e2e_s,
                           "nucleus_note": "prefill + %d nucleus-sampled passes (top-p 0.9, T 1) through spd_sample, host to "
-                                          "host; the draw of the last token (no pass) is not run" % (gen - 1)})
+                                          "host; the draw of the last token (no pass) is not run; a sampled pass costs about 8 %% more than a "
+                                          "decode step of one draft (the draw runs on one block while the others wait)" % (gen - 1)})
         c1.close()
 
     out = {
