@@ -80,7 +80,6 @@ struct KParams {
   int32_t *prefix;           // [max_pos]; kModeSample appends the sampled tokens
   float *trace;              // [L][2][d] or null
   float *pf_h, *pf_q;        // [kPfTokens][d] prefill: residual rows, rotated queries
-  float *pf_ss;              // [grid][kPfTokens] per block: sums of squares of the residual values it produced
   const void *pf_tmaps;      // [4 L + 1] tensor maps (128 bytes each) of the layers' matrices and the LM head, for the prefill's tiled copies
   // prefill activations as mma fragments, three bf16 terms each: [ceil(C/16)][2][3][32] x 8 bytes
   uint16_t *pf_xh, *pf_xo;   // gain-scaled residual (C = d), attention output (C = d)
@@ -95,9 +94,11 @@ struct KParams {
   float ns_p, ns_inv_temp;
   // launch
   int32_t mode, n_iters, pos0, step0;
-  int32_t pf_stall;          // prefill kernel, test hook: block 0 withholds its arrival at the grid barriers
   int32_t pf_head;           // prefill kernel: the launch ends the prefix: LM head on its last token and first timestep
   int32_t stage_bytes, n_stages;
+  // prefill kernel only (kept behind the fields the decode kernel reads: its code is sensitive to their offsets)
+  float *pf_ss;              // [grid][kPfTokens] per block: sums of squares of the residual values it produced
+  int32_t pf_stall;          // prefill kernel, test hook: block 0 withholds its arrival at the grid barriers
 };
 
 }  // namespace spd
