@@ -10,6 +10,7 @@
 
 #include "spd.h"
 #include "spd_params.h"
+#include "spd_prefill_tc.h"
 
 extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size_t dyn_smem, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm);
@@ -38,8 +39,17 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, total;
+      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, tc_tmaps, tc_h, tc_q, tc_y, tc_x, total;
 };
+
+// Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 128 tokens send
+// all but their last 1..128 tokens through the tensor-core path, 128 at a time.
+int tc_rows(const spd_config &c) {
+  const int hd = c.d_model / c.n_heads;
+  if (hd % 64) return 0;  // its attention kernel reads 8 dimensions at a time per lane, 8 lanes per head
+  const int full = (c.max_pos - 2) / spd::kTcTile * spd::kTcTile;
+  return full < spd::kTcMaxTokens ? full : spd::kTcMaxTokens;
+}
 
 bool valid_config(const spd_config *c) {
   if (!c) return false;
@@ -100,6 +110,13 @@ Layout make_layout(const spd_config &c, int grid) {
   L.pf_xh = take(frag_bytes(c.d_model));
   L.pf_xo = take(frag_bytes(c.d_model));
   L.pf_xu = take(frag_bytes(c.d_ffn));
+  const size_t tcr = (size_t)tc_rows(c);
+  const size_t wide = (size_t)(3 * c.d_model > 2 * c.d_ffn ? 3 * c.d_model : 2 * c.d_ffn);
+  L.tc_tmaps = take(2 * sizeof(CUtensorMap));
+  L.tc_h = take(tcr * c.d_model * 4);
+  L.tc_q = take(tcr * c.d_model * 4);
+  L.tc_y = take(tcr * wide * 4);
+  L.tc_x = take(3 * tcr * (size_t)(c.d_model > c.d_ffn ? c.d_model : c.d_ffn) * 2);
   L.total = off;
   return L;
 }
@@ -116,6 +133,18 @@ bool weight_map(TensorMapEncode encode, const void *w, int rows, int cols, CUten
   const cuuint32_t box[2] = {64, 32};
   const cuuint32_t step[2] = {1, 1};
   return encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(w), dims, strides, box, step,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor map of the term buffer of the long-prefix path seen as a bf16 matrix [rows][cols]: boxes of 64 columns x
+// 128 rows, 128-byte swizzle, zeros outside.
+bool term_map(TensorMapEncode encode, const void *x, int rows, int cols, CUtensorMap *out) {
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)spd::kTcTile};
+  const cuuint32_t step[2] = {1, 1};
+  return encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(x), dims, strides, box, step,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -138,6 +167,8 @@ struct spd_ctx {
   bool prefilled;
   int32_t m;       // prefix length
   std::vector<int32_t> prefix;  // host copy of the prefix (spd_reset extends it)
+  std::vector<spd::LayerW> layers_host;  // the layer table, for the long-prefix path's launches
+  int tc_rows;     // tokens one long-prefix job takes (0: path unused)
   int32_t n_gen;   // tokens generated per draft
   int64_t launches;
 };
@@ -190,6 +221,39 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
   spd::KParams &kp = ctx->kp;
   int32_t *base = kp.prefix;
   int rc = SPD_OK;
+  // Long run of tokens: all but the last 1..128 go through the tensor-core path, whole tiles of 128 at a time.
+  int tc_done = 0;
+  if (ctx->tc_rows > 0 && count > spd::kTcTile) {
+    const int tc_total = (count - 1) / spd::kTcTile * spd::kTcTile;
+    SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream));
+    spd::TcJob job;
+    job.L = kp.L; job.d = kp.d; job.H = kp.H; job.hd = kp.hd; job.f = kp.f; job.max_pos = kp.max_pos; job.kv_bf16 = kp.kv_bf16;
+    job.eps = kp.eps;
+    job.layers = ctx->layers_host.data();
+    job.tok_emb = kp.tok_emb;
+    job.w_tmaps = ctx->ws + ctx->lay.pf_tmaps;
+    job.x_tmaps = ctx->ws + ctx->lay.tc_tmaps;
+    job.kcache = kp.kcache; job.vcache = kp.vcache; job.rope = kp.rope;
+    job.h = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_h);
+    job.y = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_y);
+    job.q = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_q);
+    job.x = reinterpret_cast<uint16_t *>(ctx->ws + ctx->lay.tc_x);
+    job.x_term_rows = ctx->tc_rows;
+    job.st = kp.st;
+    while (tc_done < tc_total) {
+      const int n = tc_total - tc_done < ctx->tc_rows ? tc_total - tc_done : ctx->tc_rows;
+      job.ids = base + first + tc_done;
+      job.pos0 = first + tc_done;
+      job.n_tok = n;
+      int launched = 0;
+      const cudaError_t e = spd_internal_tc_prefill(&job, ctx->stream, &launched);
+      ctx->launches += launched;
+      if (e != cudaSuccess) return cuda_fail(e, "long-prefix launch");
+      tc_done += n;
+    }
+    first += tc_done;
+    count -= tc_done;
+  }
   for (int done = 0; done < count && rc == SPD_OK; done += spd::kPfTokens) {
     const int n = count - done < spd::kPfTokens ? count - done : spd::kPfTokens;
     kp.mode = spd::kModePrefill;
@@ -198,7 +262,7 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
     kp.step0 = 0;
     kp.pf_head = done + n == count ? 1 : 0;
     kp.prefix = base + first + done;
-    cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(done > 0), ctx->stream);
+    cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(done > 0 || tc_done > 0), ctx->stream);
     if (e == cudaSuccess) e = spd_internal_prefill_launch(&kp, ctx->grid, ctx->stream);
     if (e != cudaSuccess) rc = cuda_fail(e, "prefill launch");
     else ctx->launches += 1;
@@ -304,6 +368,11 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   e = spd_internal_prefill_prepare(&per_sm);
   if (e != cudaSuccess) return fail(cuda_fail(e, "prefill kernel attributes"));
   if (per_sm < 1) return fail(SPD_EINVAL);
+  ctx->tc_rows = tc_rows(*cfg);
+  if (ctx->tc_rows > 0) {
+    e = spd_internal_tc_prepare();
+    if (e != cudaSuccess) return fail(cuda_fail(e, "long-prefix kernel attributes"));
+  }
 
   const int hd = cfg->d_model / cfg->n_heads;
   kp.L = cfg->n_layers; kp.d = cfg->d_model; kp.H = cfg->n_heads; kp.hd = hd; kp.f = cfg->d_ffn; kp.V = cfg->vocab;
@@ -363,6 +432,9 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   }
   // tensor maps of the matrices in the order the prefill kernel walks them
   std::vector<CUtensorMap> tmaps((size_t)4 * cfg->n_layers + 1);
+  CUtensorMap xmaps[2];
+  std::memset(xmaps, 0, sizeof xmaps);
+  ctx->layers_host = layers;
   {
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
@@ -377,6 +449,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
            weight_map(encode, w->wgate_up[l], 2 * f, d, &tmaps[4 * l + 2]) && weight_map(encode, w->wdown[l], d, f, &tmaps[4 * l + 3]);
     }
     ok = ok && weight_map(encode, w->lm_head, cfg->vocab, d, &tmaps[(size_t)4 * cfg->n_layers]);
+    if (ok && ctx->tc_rows > 0)
+      ok = term_map(encode, ws + lay.tc_x, 3 * ctx->tc_rows, d, &xmaps[0]) && term_map(encode, ws + lay.tc_x, 3 * ctx->tc_rows, f, &xmaps[1]);
     if (!ok) return fail(SPD_EINVAL);
   }
   cudaStream_t s = ctx->stream;
@@ -386,7 +460,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.state, 0, sizeof(spd::State), s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.trace, 0, (size_t)cfg->n_layers * 2 * cfg->d_model * 4, s);
   // columns past the row's end inside the last 16-column step of a fragment buffer are never written: zero
-  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.pf_cnt, 0, lay.total - lay.pf_cnt, s);  // also the arrival counters
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + lay.pf_cnt, 0, lay.tc_tmaps - lay.pf_cnt, s);  // also the arrival counters
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + lay.tc_tmaps, xmaps, sizeof xmaps, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return fail(cuda_fail(e, "workspace initialisation"));
   *out = ctx;

@@ -1,0 +1,30 @@
+// Host-side description of one long-prefix prefill job (see spd_prefill_tc.cu).
+#pragma once
+#include "spd_params.h"
+
+namespace spd {
+
+constexpr int kTcTile = 128;      // tokens per tile of the tensor-core products
+constexpr int kTcMaxTokens = 512; // tokens one job takes at most
+
+struct TcJob {
+  int32_t L, d, H, hd, f, max_pos, kv_bf16;
+  float eps;
+  const LayerW *layers;              // HOST copy of the layer table [L]
+  const __nv_bfloat16 *tok_emb;
+  const uint8_t *w_tmaps;            // device: tensor maps of the layers' matrices, four per layer
+  const uint8_t *x_tmaps;            // device: tensor maps of the term buffer seen as [3 * x_term_rows][d] and [..][f]
+  void *kcache, *vcache;
+  const float2 *rope;
+  float *h, *y, *q;                  // [x_term_rows][d], [x_term_rows][max(3d, 2f)], [x_term_rows][d]
+  uint16_t *x;                       // [3][x_term_rows][max(d, f)] bf16 terms
+  int32_t x_term_rows;
+  const int32_t *ids;                // device: the job's token ids
+  int32_t pos0, n_tok;               // first position; tokens (a multiple of kTcTile, <= x_term_rows)
+  State *st;
+};
+
+}  // namespace spd
+
+extern "C" cudaError_t spd_internal_tc_prepare(void);
+extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);

@@ -1,0 +1,66 @@
+"""Prefixes of more than 128 tokens: all but the last 1..128 tokens go through the tensor-core path (tcgen05
+products over tiles of 128 tokens, up to 512 tokens per job), the rest through the 16-token prefill kernel,
+which ends with the first timestep (Eq. 1).  Both fill the same cache; the first timestep and the steps after
+it are compared with the oracle as for short prefixes."""
+import numpy as np
+import pytest
+
+import spd_inputs as si
+from tests.gpu_common import compare_first_step, compare_step, make_pair, make_tiny_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def _expected_launches(m, layers, job_tokens):
+    tc = (m - 1) // 128 * 128 if m > 128 else 0
+    jobs = -(-tc // job_tokens) if tc else 0
+    return jobs * 9 * layers + (m - tc + 15) // 16
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("m", [129, 293, 700])
+def test_long_prefix_tiny(tiny_inputs, m, kv_dtype):
+    """Tiny shape: d_ffn = 688 leaves a ragged last 64-column stage and 2 d_ffn = 1376 a ragged last row tile;
+    129 = one tile and one token, 293 = one job of two tiles, 700 = a job of 512 tokens and one of 128."""
+    wl, _, _, _ = tiny_inputs
+    prefix = si.make_prefix("zipf", m, wl.shape.vocab, 1.1, seed=500 + m)
+    ctx, orc = make_tiny_pair(tiny_inputs, max_pos=1024, kv_dtype=kv_dtype)
+    compare_first_step(ctx, orc, prefix)
+    assert ctx.spd_launch_count() == _expected_launches(m, wl.shape.n_layers, 512)
+    for _ in range(3):
+        compare_step(ctx, orc)
+    # and once more on the same context (the term buffers and the cache are reused)
+    prefix2 = si.make_prefix("zipf", 257, wl.shape.vocab, 1.1, seed=900 + m)
+    compare_first_step(ctx, orc, prefix2)
+    compare_step(ctx, orc)
+    ctx.close()
+
+
+def test_long_prefix_head_dim_128():
+    """head_dim 128 (the 7B shapes' attention layout), bf16 cache; max_pos 300 caps a job at 256 tokens."""
+    shape = si.ModelShape("hd128", 2, 256, 2, 512, 1000)
+    weights = si.make_weights(shape, seed=11)
+    tables = si.make_ngram_tables(shape.vocab, 1.1, 50_000, (2, 3), 5000, seed=12)
+    lam = [0.3, 0.2] + [0.0] * 6
+    for max_pos, m in ((300, 290), (1024, 1000)):
+        ctx, orc = make_pair(shape, weights, tables, 3, (2, 3), lam, 0.4, 0.2, 0.05, max_pos, "bf16")
+        prefix = si.make_prefix("zipf", m, shape.vocab, 1.1, seed=77 + m)
+        compare_first_step(ctx, orc, prefix)
+        assert ctx.spd_launch_count() == _expected_launches(m, 2, 256 if max_pos == 300 else 512)
+        for _ in range(3):
+            compare_step(ctx, orc)
+        ctx.close()
+
+
+def test_reset_after_long_prefix(tiny_inputs):
+    """A restart from a draft (Section 5.3) recomputes only the generated positions on top of a cache that the
+    long-prefix path filled."""
+    wl, _, _, _ = tiny_inputs
+    prefix = si.make_prefix("zipf", 300, wl.shape.vocab, 1.1, seed=321)
+    ctx, orc = make_tiny_pair(tiny_inputs, max_pos=512)
+    compare_first_step(ctx, orc, prefix)
+    for _ in range(4):
+        compare_step(ctx, orc)
+    compare_first_step(ctx, orc, None, reset_draft=1)
+    compare_step(ctx, orc)
+    ctx.close()
