@@ -43,10 +43,10 @@ struct Layout {
 };
 
 // Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 128 tokens send
-// all but their last 1..128 tokens through the tensor-core path, 128 at a time.
+// all but their last 1..16 tokens through the tensor-core path.
 int tc_rows(const spd_config &c) {
   const int hd = c.d_model / c.n_heads;
-  if (hd % 64) return 0;  // its attention kernel reads 8 dimensions at a time per lane, 8 lanes per head
+  if (hd != 64 && hd != 128) return 0;  // the head sizes its attention kernel is built for
   const int full = (c.max_pos - 2) / spd::kTcTile * spd::kTcTile;
   return full < spd::kTcMaxTokens ? full : spd::kTcMaxTokens;
 }
@@ -221,10 +221,10 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
   spd::KParams &kp = ctx->kp;
   int32_t *base = kp.prefix;
   int rc = SPD_OK;
-  // Long run of tokens: all but the last 1..128 go through the tensor-core path, whole tiles of 128 at a time.
+  // Long run of tokens: all but the last 1..16 go through the tensor-core path, in jobs of up to tc_rows tokens.
   int tc_done = 0;
   if (ctx->tc_rows > 0 && count > spd::kTcTile) {
-    const int tc_total = (count - 1) / spd::kTcTile * spd::kTcTile;
+    const int tc_total = count - ((count - 1) % spd::kPfTokens + 1);
     SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream));
     spd::TcJob job;
     job.L = kp.L; job.d = kp.d; job.H = kp.H; job.hd = kp.hd; job.f = kp.f; job.max_pos = kp.max_pos; job.kv_bf16 = kp.kv_bf16;

@@ -295,113 +295,314 @@ __global__ void __launch_bounds__(256) spd_tc_swiglu_kernel(const float *Y, uint
   }
 }
 
-// Causal attention of the block's tokens over the cache.  Block = (8 consecutive tokens, one head), a warp per
-// token; the warp's lanes form 4 groups of 8: a group takes every fourth cached position, each of its lanes
-// PER = head_dim / 8 dimensions of it; online softmax per group, the groups merged by shuffles at the end.
-// The eight warps read the same cache rows at about the same time.  Output as three bf16 terms.
-template <int PER, bool BF16>
-__global__ void __launch_bounds__(256) spd_tc_attn_kernel(const float *Q, const void *kcache, const void *vcache, uint16_t *X,
-                                                          size_t term_stride, int d, int hd, int max_pos, int layer, int pos0) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t = blockIdx.x * 8 + warp, head = blockIdx.y;
-  const int g = lane >> 3, s = lane & 7;
-  const int per = PER > 0 ? PER : hd / 8;
-  constexpr int kMax = PER > 0 ? PER : 32;
-  const int T = pos0 + t + 1;
-  const float scale = 1.f / sqrtf((float)hd);
-  const int col = head * hd + s * per;
-  float q[kMax], acc[kMax];
-#pragma unroll
-  for (int e = 0; e < kMax; ++e) {
-    q[e] = e < per ? Q[(size_t)t * d + col + e] * scale : 0.f;
-    acc[e] = 0.f;
+// Causal attention over a float32 cache (a bf16 cache takes spd_tc_attn_mma_kernel below): 16 consecutive tokens
+// of one head.  The block brings 32 cached positions at
+// a time into shared memory as float32 (keys with padded rows, so that a lane per position reads its row without
+// bank conflicts); a warp owns two tokens: scores with a lane per position, the tile's softmax weights by warp
+// reductions (online softmax across tiles), weighted value sums with HD / 32 dimensions per lane and the weights
+// passed round by shuffles.  Every cache row is read once per 16 tokens.  Output as three bf16 terms.
+template <int HD>
+__global__ void __launch_bounds__(256) spd_tc_attn_kernel(const float *Q, const float *kcache, const float *vcache, uint16_t *X,
+                                                          size_t term_stride, int d, int max_pos, int layer, int pos0, int n_tok) {
+  constexpr int kTok = 16, kPos = 32;
+  constexpr int KS = HD + 4;    // key row stride in floats: 16-byte aligned, rows 4 banks apart
+  constexpr int DPL = HD / 32;  // value dimensions per lane
+  __shared__ __align__(16) float sq[kTok * HD];
+  __shared__ __align__(16) float sk[kPos * KS];
+  __shared__ __align__(16) float sv[kPos * HD];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int head = blockIdx.y, t0 = blockIdx.x * kTok;
+  const float scale = 1.f / sqrtf((float)HD);
+  for (int i = tid; i < kTok * HD; i += 256) {
+    const int tt = i / HD, c = i - tt * HD;
+    sq[i] = t0 + tt < n_tok ? Q[(size_t)(t0 + tt) * d + head * HD + c] * scale : 0.f;
   }
-  float m = -CUDART_INF_F, l = 0.f;
-  for (int tp0 = 0; tp0 < T; tp0 += 4) {
-    const int tp = tp0 + g;
-    const bool visible = tp < T;
-    const size_t base = ((size_t)layer * max_pos + (visible ? tp : 0)) * d + col;
-    float kv[kMax], vv[kMax];
-    if (BF16) {
-      const uint4 *kp = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(kcache) + base);
-      const uint4 *vp = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(vcache) + base);
+  const int last_pos = pos0 + min(t0 + kTok - 1, n_tok - 1);  // the last position a token of this block sees
+  const int ta = t0 + 2 * warp, tb = ta + 1;
+  const int pa = pos0 + ta, pb = pos0 + tb;
+  float ma = -CUDART_INF_F, mb = -CUDART_INF_F, la = 0.f, lb = 0.f;
+  float acca[DPL], accb[DPL];
 #pragma unroll
-      for (int e = 0; e < kMax; e += 8) {
-        if (e < per) {
-          const uint4 a = kp[e >> 3], b = vp[e >> 3];
-          const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+  for (int e = 0; e < DPL; ++e) acca[e] = accb[e] = 0.f;
+  for (int tile0 = 0; tile0 <= last_pos; tile0 += kPos) {
+    __syncthreads();  // the previous tile has been used (first round: nothing)
+    for (int i = tid; i < kPos * HD / 8; i += 256) {
+      const int r = i / (HD / 8), c8 = (i - r * (HD / 8)) * 8;
+      const int pos = tile0 + r;
+      float kf[8], vf[8];
+      if (pos <= last_pos) {
+        const size_t at = ((size_t)layer * max_pos + pos) * d + head * HD + c8;
+        const float4 *kp = reinterpret_cast<const float4 *>(kcache + at), *vp = reinterpret_cast<const float4 *>(vcache + at);
+        const float4 k0 = kp[0], k1 = kp[1], v0 = vp[0], v1 = vp[1];
+        kf[0] = k0.x; kf[1] = k0.y; kf[2] = k0.z; kf[3] = k0.w; kf[4] = k1.x; kf[5] = k1.y; kf[6] = k1.z; kf[7] = k1.w;
+        vf[0] = v0.x; vf[1] = v0.y; vf[2] = v0.z; vf[3] = v0.w; vf[4] = v1.x; vf[5] = v1.y; vf[6] = v1.z; vf[7] = v1.w;
+      } else {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            kv[e + 2 * j] = __uint_as_float(aw[j] << 16);
-            kv[e + 2 * j + 1] = __uint_as_float(aw[j] & 0xffff0000u);
-            vv[e + 2 * j] = __uint_as_float(bw[j] << 16);
-            vv[e + 2 * j + 1] = __uint_as_float(bw[j] & 0xffff0000u);
-          }
+        for (int j = 0; j < 8; ++j) kf[j] = vf[j] = 0.f;
+      }
+      float4 *kd = reinterpret_cast<float4 *>(sk + r * KS + c8), *vd = reinterpret_cast<float4 *>(sv + r * HD + c8);
+      kd[0] = make_float4(kf[0], kf[1], kf[2], kf[3]);
+      kd[1] = make_float4(kf[4], kf[5], kf[6], kf[7]);
+      vd[0] = make_float4(vf[0], vf[1], vf[2], vf[3]);
+      vd[1] = make_float4(vf[4], vf[5], vf[6], vf[7]);
+    }
+    __syncthreads();
+    // scores of position tile0 + lane for the warp's two tokens
+    float sa = 0.f, sb = 0.f;
+    {
+      const float4 *kr = reinterpret_cast<const float4 *>(sk + lane * KS);
+      const float4 *qa = reinterpret_cast<const float4 *>(sq + (2 * warp) * HD), *qb = qa + HD / 4;
+#pragma unroll 8
+      for (int c = 0; c < HD / 4; ++c) {
+        const float4 k4 = kr[c], a4 = qa[c], b4 = qb[c];
+        sa = fmaf(a4.x, k4.x, sa); sa = fmaf(a4.y, k4.y, sa); sa = fmaf(a4.z, k4.z, sa); sa = fmaf(a4.w, k4.w, sa);
+        sb = fmaf(b4.x, k4.x, sb); sb = fmaf(b4.y, k4.y, sb); sb = fmaf(b4.z, k4.z, sb); sb = fmaf(b4.w, k4.w, sb);
+      }
+    }
+    const int pos = tile0 + lane;
+    sa = pos <= pa ? sa : -CUDART_INF_F;
+    sb = pos <= pb ? sb : -CUDART_INF_F;
+    float xa = sa, xb = sb;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      xa = fmaxf(xa, __shfl_xor_sync(0xffffffffu, xa, o));
+      xb = fmaxf(xb, __shfl_xor_sync(0xffffffffu, xb, o));
+    }
+    // position 0 is visible to every token, so the running maxima are finite from the first tile on
+    const float mna = fmaxf(ma, xa), mnb = fmaxf(mb, xb);
+    const float ca = __expf(ma - mna), cb = __expf(mb - mnb);
+    const float wa = __expf(sa - mna), wb = __expf(sb - mnb);
+    float ua = wa, ub = wb;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ua += __shfl_xor_sync(0xffffffffu, ua, o);
+      ub += __shfl_xor_sync(0xffffffffu, ub, o);
+    }
+    la = fmaf(la, ca, ua);
+    lb = fmaf(lb, cb, ub);
+    ma = mna;
+    mb = mnb;
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) {
+      acca[e] *= ca;
+      accb[e] *= cb;
+    }
+#pragma unroll
+    for (int j = 0; j < kPos; ++j) {
+      const float ja = __shfl_sync(0xffffffffu, wa, j), jb = __shfl_sync(0xffffffffu, wb, j);
+      const float *vr = sv + j * HD + lane * DPL;
+      float v[DPL];
+      if (DPL == 4) {
+        const float4 v4 = *reinterpret_cast<const float4 *>(vr);
+        v[0] = v4.x; v[1] = v4.y; v[DPL - 2] = v4.z; v[DPL - 1] = v4.w;
+      } else {
+        const float2 v2 = *reinterpret_cast<const float2 *>(vr);
+        v[0] = v2.x; v[1] = v2.y;
+      }
+#pragma unroll
+      for (int e = 0; e < DPL; ++e) {
+        acca[e] = fmaf(ja, v[e], acca[e]);
+        accb[e] = fmaf(jb, v[e], accb[e]);
+      }
+    }
+  }
+  const float ia = 1.f / la, ib = 1.f / lb;
+#pragma unroll
+  for (int e = 0; e < DPL; ++e) {
+    if (ta < n_tok) tc_put3(X, term_stride, (size_t)ta * d + head * HD + lane * DPL + e, acca[e] * ia);
+    if (tb < n_tok) tc_put3(X, term_stride, (size_t)tb * d + head * HD + lane * DPL + e, accb[e] * ib);
+  }
+}
+
+// ---------------------------------------------------------------- attention over a bf16 cache on tensor cores
+__device__ __forceinline__ void tc_mma_sync(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void tc_ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void tc_ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+// The three bf16 terms of v (v = hi + mid + lo exactly), each in the upper half of a word.
+__device__ __forceinline__ void tc_split3(float v, uint32_t &hi, uint32_t &mid, uint32_t &lo) {
+  hi = __float_as_uint(v) & 0xffff0000u;
+  const float r1 = v - __uint_as_float(hi);
+  mid = __float_as_uint(r1) & 0xffff0000u;
+  lo = __float_as_uint(r1 - __uint_as_float(mid)) & 0xffff0000u;
+}
+
+// Causal attention of 64 consecutive tokens of one head over a bf16 cache, on tensor cores (mma.sync m16n8k16:
+// the attention's share of the arithmetic is small, so the warp-level instructions serve).  Keys and values
+// are bf16 already and therefore exact operands; the scaled queries and the softmax weights are float32 and go
+// in as three bf16 terms each, as the activations of the products do.  A warp owns 16 tokens: scores of a tile of
+// 64 cached positions (tokens x positions, keys read from padded shared-memory rows), online softmax on the
+// accumulator fragments, the weights' terms repacked in registers as the next product's left operand, values
+// through transposing matrix loads.  Rows of every shared-memory tile are 16 bytes longer than their data: eight
+// consecutive rows then start in different bank groups.
+template <int HD>
+__global__ void __launch_bounds__(128) spd_tc_attn_mma_kernel(const float *Q, const uint16_t *kcache, const uint16_t *vcache, uint16_t *X,
+                                                              size_t term_stride, int d, int max_pos, int layer, int pos0, int n_tok) {
+  constexpr int kTok = 64, kPos = 64;
+  constexpr int RS = HD * 2 + 16;  // bytes per tile row
+  constexpr int KS = HD / 16;      // k-steps over the head's dimensions
+  constexpr int DT = HD / 8;       // output tiles of 8 dimensions
+  extern __shared__ __align__(16) uint8_t at_smem[];
+  uint8_t *sq = at_smem;                // [3 terms][64 tokens][RS]
+  uint8_t *sk = sq + 3 * kTok * RS;     // [64 positions][RS]
+  uint8_t *sv = sk + kPos * RS;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, q = lane & 3;
+  const int head = blockIdx.y, t0 = blockIdx.x * kTok;
+  const float scale = 1.f / sqrtf((float)HD);
+  for (int i = tid; i < kTok * HD; i += 128) {
+    const int tt = i / HD, c = i - tt * HD;
+    const float v = t0 + tt < n_tok ? Q[(size_t)(t0 + tt) * d + head * HD + c] * scale : 0.f;
+    uint32_t hi, mid, lo;
+    tc_split3(v, hi, mid, lo);
+    uint16_t *dst = reinterpret_cast<uint16_t *>(sq + tt * RS) + c;
+    dst[0] = (uint16_t)(hi >> 16);
+    dst[kTok * RS / 2] = (uint16_t)(mid >> 16);
+    dst[2 * kTok * RS / 2] = (uint16_t)(lo >> 16);
+  }
+  const int last_pos = pos0 + min(t0 + kTok - 1, n_tok - 1);  // the last position a token of this block sees
+  const int tw = t0 + warp * 16;
+  const int p_lo = pos0 + tw + g, p_hi = p_lo + 8, warp_last = pos0 + tw + 15;
+  float m[2] = {-CUDART_INF_F, -CUDART_INF_F}, l[2] = {0.f, 0.f};
+  float o[DT][4];
+#pragma unroll
+  for (int i = 0; i < DT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  const uint32_t sq_u = smem_u32(sq), sk_u = smem_u32(sk), sv_u = smem_u32(sv);
+  // per-lane offsets: left operand (tokens x dimensions), keys (32-bit words), values (transposed matrices)
+  const uint32_t a_off = (uint32_t)((warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * RS + (lane >> 4) * 16);
+  const uint32_t k_off = (uint32_t)(g * RS + q * 4);
+  const uint32_t v_off = (uint32_t)((((lane >> 3) & 1) * 8 + (lane & 7)) * RS + (lane >> 4) * 16);
+  for (int tile0 = 0; tile0 <= last_pos; tile0 += kPos) {
+    __syncthreads();  // the previous tile has been used; first round: the queries are in place after the next barrier
+    for (int i = tid; i < kPos * HD / 8; i += 128) {
+      const int r = i / (HD / 8), c8 = i - r * (HD / 8);
+      const int pos = tile0 + r;
+      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+      if (pos <= last_pos) {
+        const size_t at = ((size_t)layer * max_pos + pos) * d + head * HD + c8 * 8;
+        a = *reinterpret_cast<const uint4 *>(kcache + at);
+        b = *reinterpret_cast<const uint4 *>(vcache + at);
+      }
+      *reinterpret_cast<uint4 *>(sk + r * RS + c8 * 16) = a;
+      *reinterpret_cast<uint4 *>(sv + r * RS + c8 * 16) = b;
+    }
+    __syncthreads();
+    if (tile0 > warp_last) continue;  // nothing of this tile is visible to the warp's tokens (the barriers are above)
+    float s[kPos / 8][4];
+#pragma unroll
+    for (int i = 0; i < kPos / 8; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      uint32_t a[3][4];
+#pragma unroll
+      for (int j = 0; j < 3; ++j) tc_ldsm_x4(sq_u + (uint32_t)(j * kTok * RS) + a_off + (uint32_t)(ks * 32), a[j]);
+#pragma unroll
+      for (int nt = 0; nt < kPos / 8; ++nt) {
+        uint32_t b0, b1;
+        const uint32_t addr = sk_u + k_off + (uint32_t)(nt * 8 * RS + ks * 32);
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(b0) : "r"(addr));
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(b1) : "r"(addr + 16));
+#pragma unroll
+        for (int j = 0; j < 3; ++j) tc_mma_sync(s[nt], a[j], b0, b1);
+      }
+    }
+    // causal mask, row maxima (rows g and g + 8 of the warp's 16 tokens; a row lives in the four lanes of a quad)
+    float mx[2] = {-CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+    for (int nt = 0; nt < kPos / 8; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int pos = tile0 + nt * 8 + 2 * q + (e & 1);
+        if (pos > (e < 2 ? p_lo : p_hi)) s[nt][e] = -CUDART_INF_F;
+        mx[e >> 1] = fmaxf(mx[e >> 1], s[nt][e]);
+      }
+    float c[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+      const float mn = fmaxf(m[r], mx[r]);  // finite: position 0 is visible to every token in the first tile
+      c[r] = __expf(m[r] - mn);
+      m[r] = mn;
+      l[r] *= c[r];
+    }
+#pragma unroll
+    for (int i = 0; i < DT; ++i) {
+      o[i][0] *= c[0]; o[i][1] *= c[0]; o[i][2] *= c[1]; o[i][3] *= c[1];
+    }
+    // the weights and their terms, repacked as left operands: positions 16 kk .. 16 kk + 15 are score tiles 2 kk, 2 kk + 1
+    uint32_t pt[kPos / 16][3][4];
+#pragma unroll
+    for (int nt = 0; nt < kPos / 8; ++nt) {
+      float pw[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) pw[e] = __expf(s[nt][e] - m[e >> 1]);
+      l[0] += pw[0] + pw[1];
+      l[1] += pw[2] + pw[3];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        uint32_t h0, m0, l0, h1, m1, l1;
+        tc_split3(pw[2 * r], h0, m0, l0);
+        tc_split3(pw[2 * r + 1], h1, m1, l1);
+        const int reg = (nt & 1) * 2 + r;
+        pt[nt >> 1][0][reg] = h1 | (h0 >> 16);
+        pt[nt >> 1][1][reg] = m1 | (m0 >> 16);
+        pt[nt >> 1][2][reg] = l1 | (l0 >> 16);
+      }
+    }
+#pragma unroll
+    for (int kk = 0; kk < kPos / 16; ++kk)
+#pragma unroll
+      for (int dp = 0; dp < DT / 2; ++dp) {
+        uint32_t b[4];
+        tc_ldsm_x4_trans(sv_u + v_off + (uint32_t)(kk * 16 * RS + dp * 32), b);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+          tc_mma_sync(o[2 * dp], pt[kk][j], b[0], b[1]);
+          tc_mma_sync(o[2 * dp + 1], pt[kk][j], b[2], b[3]);
         }
       }
-    } else {
-      const float4 *kp = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(kcache) + base);
-      const float4 *vp = reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(vcache) + base);
-#pragma unroll
-      for (int e = 0; e < kMax; e += 4) {
-        if (e < per) {
-          const float4 a = kp[e >> 2], b = vp[e >> 2];
-          kv[e] = a.x; kv[e + 1] = a.y; kv[e + 2] = a.z; kv[e + 3] = a.w;
-          vv[e] = b.x; vv[e + 1] = b.y; vv[e + 2] = b.z; vv[e + 3] = b.w;
-        }
-      }
-    }
-    float dot = 0.f;
-#pragma unroll
-    for (int e = 0; e < kMax; ++e)
-      if (e < per) dot = fmaf(q[e], kv[e], dot);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-    if (visible) {
-      const float mn = fmaxf(m, dot);
-      const float c = __expf(m - mn), pw = __expf(dot - mn);  // m = -inf at first: c = 0
-      l = fmaf(l, c, pw);
-#pragma unroll
-      for (int e = 0; e < kMax; ++e)
-        if (e < per) acc[e] = fmaf(acc[e], c, pw * vv[e]);
-      m = mn;
-    }
   }
-  // the four groups' states
 #pragma unroll
-  for (int off = 8; off <= 16; off <<= 1) {
-    const float mo = __shfl_xor_sync(0xffffffffu, m, off), lo = __shfl_xor_sync(0xffffffffu, l, off);
-    const float M = fmaxf(m, mo);
-    const float cs = m == -CUDART_INF_F ? 0.f : __expf(m - M), co = mo == -CUDART_INF_F ? 0.f : __expf(mo - M);
-    l = l * cs + lo * co;
+  for (int r = 0; r < 2; ++r) {
+    l[r] += __shfl_xor_sync(0xffffffffu, l[r], 1);
+    l[r] += __shfl_xor_sync(0xffffffffu, l[r], 2);
+  }
+  const float inv[2] = {1.f / l[0], 1.f / l[1]};
 #pragma unroll
-    for (int e = 0; e < kMax; ++e) {
-      const float ao = __shfl_xor_sync(0xffffffffu, acc[e], off);
-      if (e < per) acc[e] = (g & (off >> 3)) ? ao * co + acc[e] * cs : acc[e] * cs + ao * co;
+  for (int i = 0; i < DT; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int t = tw + g + (e >> 1) * 8;
+      if (t < n_tok) tc_put3(X, term_stride, (size_t)t * d + head * HD + i * 8 + 2 * q + (e & 1), o[i][e] * inv[e >> 1]);
     }
-    m = M;
-  }
-  if (g == 0) {
-    const float inv = 1.f / l;
-#pragma unroll
-    for (int e = 0; e < kMax; ++e)
-      if (e < per) tc_put3(X, term_stride, (size_t)t * d + col + e, acc[e] * inv);
-  }
 }
 
 }  // namespace spd
 
 namespace {
 
-template <int PER>
+template <int HD>
+constexpr size_t attn_mma_smem() { return (size_t)5 * 64 * (HD * 2 + 16); }  // three query terms, keys, values: 64 padded rows each
+
+template <int HD>
 cudaError_t launch_attn(const spd::TcJob &j, int layer, int n_tok, cudaStream_t s) {
-  const dim3 grid(n_tok / 8, j.H);
   const size_t ts = (size_t)j.x_term_rows * j.d;
   if (j.kv_bf16)
-    spd::spd_tc_attn_kernel<PER, true><<<grid, 256, 0, s>>>(j.q, j.kcache, j.vcache, j.x, ts, j.d, j.hd, j.max_pos, layer, j.pos0);
+    spd::spd_tc_attn_mma_kernel<HD><<<dim3((n_tok + 63) / 64, j.H), 128, attn_mma_smem<HD>(), s>>>(
+        j.q, static_cast<const uint16_t *>(j.kcache), static_cast<const uint16_t *>(j.vcache), j.x, ts, j.d, j.max_pos, layer, j.pos0, n_tok);
   else
-    spd::spd_tc_attn_kernel<PER, false><<<grid, 256, 0, s>>>(j.q, j.kcache, j.vcache, j.x, ts, j.d, j.hd, j.max_pos, layer, j.pos0);
+    spd::spd_tc_attn_kernel<HD><<<dim3((n_tok + 15) / 16, j.H), 256, 0, s>>>(j.q, static_cast<const float *>(j.kcache),
+                                                                           static_cast<const float *>(j.vcache), j.x, ts, j.d, j.max_pos,
+                                                                           layer, j.pos0, n_tok);
   return cudaGetLastError();
 }
 
@@ -410,12 +611,21 @@ size_t tc_gemm_smem() { return (size_t)spd::kTcStages * spd::kTcStageBytes + 102
 }  // namespace
 
 extern "C" cudaError_t spd_internal_tc_prepare(void) {
-  return cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_tc_gemm_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)tc_gemm_smem());
+  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_tc_gemm_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)tc_gemm_smem());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_tc_attn_mma_kernel<64>), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_mma_smem<64>());
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_tc_attn_mma_kernel<128>), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_mma_smem<128>());
+  return e;
 }
 
-// Enqueues the decoder over j.n_tok tokens (a multiple of 128, at most j.x_term_rows) at positions j.pos0 ..:
-// their keys and values enter the cache.  *launches receives the number of kernels enqueued.
+// Enqueues the decoder over j.n_tok tokens (at most j.x_term_rows) at positions j.pos0 ..: their keys and values
+// enter the cache.  The products run over whole tiles of 128 tokens: the rows past n_tok of the last tile hold
+// whatever an earlier job left, give rows of Y that nothing reads (a row of Y depends on its own token only).
+// *launches receives the number of kernels enqueued.
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t s, int *launches) {
   const spd::TcJob &j = *job;
   const int n = j.n_tok, d = j.d, f = j.f;
@@ -425,7 +635,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
   cudaError_t e = cudaSuccess;
   auto gemm = [&](const uint8_t *xmap, int which, int N, int C) {
     if (e != cudaSuccess) return;
-    const dim3 grid((N + spd::kTcN - 1) / spd::kTcN, n / spd::kTcM);
+    const dim3 grid((N + spd::kTcN - 1) / spd::kTcN, (n + spd::kTcM - 1) / spd::kTcM);
     spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, j.w_tmaps + (size_t)which * spd::kTensorMapBytes, j.y, N, C,
                                                                          j.x_term_rows, j.st);
     e = cudaGetLastError();
@@ -443,7 +653,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
     if (e != cudaSuccess) break;
     spd::spd_tc_rope_cache_kernel<<<n, 256, 0, s>>>(j.y, j.q, j.kcache, j.vcache, j.rope, d, j.hd, j.max_pos, l, j.pos0, j.kv_bf16);
     if ((e = cudaGetLastError()) != cudaSuccess) break;
-    e = j.hd == 128 ? launch_attn<16>(j, l, n, s) : j.hd == 64 ? launch_attn<8>(j, l, n, s) : launch_attn<0>(j, l, n, s);
+    e = j.hd == 128 ? launch_attn<128>(j, l, n, s) : launch_attn<64>(j, l, n, s);  // other head sizes never get here
     count += 2;
     gemm(xmap_d, 4 * l + 1, d, d);
     resid(j.y, nullptr, j.layers[l].ffn_norm);

@@ -20,7 +20,7 @@ struct TcJob {
   uint16_t *x;                       // [3][x_term_rows][max(d, f)] bf16 terms
   int32_t x_term_rows;
   const int32_t *ids;                // device: the job's token ids
-  int32_t pos0, n_tok;               // first position; tokens (a multiple of kTcTile, <= x_term_rows)
+  int32_t pos0, n_tok;               // first position; tokens (<= x_term_rows)
   State *st;
 };
 
