@@ -10,8 +10,8 @@
 // computes a tile of 128 tokens x 128 rows: a producer thread fills a ring of stages (three term tiles of
 // 128 tokens x 64 columns and one weight tile of 128 rows x 64 columns, all in the 128-byte-swizzled K-major
 // layout the tensor cores read), one thread issues the 12 instructions of a stage (3 terms x 4 k-steps of 16
-// columns) and hands the stage back with tcgen05.commit, four warps move the finished accumulator from
-// tensor memory to global memory.  Every wait is bounded; a wait that runs out records SPD_ETIMEOUT in the
+// columns) and hands the stage back with tcgen05.commit; four accumulators take turns, each the sum of 8 stages,
+// and four warps add those sums in registers (round-to-nearest) and write the tile to global memory.  Every wait is bounded; a wait that runs out records SPD_ETIMEOUT in the
 // context's state, the block waits for its copies in flight, frees its tensor memory and returns.
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -31,6 +31,8 @@ constexpr int kTcStageBytes = 3 * kTcTermBytes + kTcWBytes;  // 64 KB
 constexpr int kTcStages = 3;
 constexpr int kTcThreads = 192;                // producer warp, issuing warp, four warps for the accumulator
 constexpr int kTcWBoxRows = 32;                // the weights' tensor maps describe boxes of 32 rows x 64 columns
+constexpr int kTcSegSteps = 8;                 // stages summed inside tensor memory before the sum moves to registers
+constexpr int kTcAccs = 4;                     // accumulators in rotation: 4 x 128 columns = all of tensor memory
 constexpr unsigned long long kTcWaitNs = 1500ull * 1000ull * 1000ull;
 
 // ---------------------------------------------------------------- PTX: tensor memory and tcgen05
@@ -88,7 +90,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 
 struct TcShared {
-  uint64_t full[kTcStages], empty[kTcStages], accum;
+  uint64_t full[kTcStages], empty[kTcStages], acc_full[kTcAccs], acc_empty[kTcAccs];
   uint32_t tmem_base;
   int dead;
 };
@@ -129,10 +131,13 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], 1);
     }
-    mbar_init(&sh.accum, 1);
+    for (int a = 0; a < kTcAccs; ++a) {
+      mbar_init(&sh.acc_full[a], 1);
+      mbar_init(&sh.acc_empty[a], 4);  // one arrival per warp that reads the accumulator
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tc_alloc(&sh.tmem_base, kTcN);
+  if (warp == 1) tc_alloc(&sh.tmem_base, kTcAccs * kTcN);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -174,45 +179,60 @@ __global__ void __launch_bounds__(kTcThreads, 1)
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int ks = 0; ks < nk; ++ks) {
-        if (!tc_wait(sh, st, &sh.full[stage], phase, 410)) { ok = false; break; }
+        const int seg = ks / kTcSegSteps, in_seg = ks - seg * kTcSegSteps, a = seg % kTcAccs;
+        if (in_seg == 0 && !tc_wait(sh, st, &sh.acc_empty[a], (uint32_t)((seg / kTcAccs) & 1) ^ 1u, 430)) break;  // its last sum has been read
+        if (!tc_wait(sh, st, &sh.full[stage], phase, 410)) break;
         tc_fence_after();
         const uint32_t base = ring + stage * (uint32_t)kTcStageBytes;
 #pragma unroll
         for (int j = 0; j < 3; ++j)
 #pragma unroll
           for (int kk = 0; kk < kTcKB / 16; ++kk)  // 16 columns = 32 bytes further into the swizzled rows
-            tc_mma(tmem, tc_desc(base + j * kTcTermBytes + kk * 32), tc_desc(base + 3 * kTcTermBytes + kk * 32), idesc,
-                   (uint32_t)((ks | j | kk) != 0));
+            tc_mma(tmem + (uint32_t)(a * kTcN), tc_desc(base + j * kTcTermBytes + kk * 32), tc_desc(base + 3 * kTcTermBytes + kk * 32),
+                   idesc, (uint32_t)((in_seg | j | kk) != 0));
         tc_commit(&sh.empty[stage]);  // the stage is free once these have read it
+        if (in_seg == kTcSegSteps - 1 || ks == nk - 1) tc_commit(&sh.acc_full[a]);  // the segment's sum is complete
         if (++stage == (uint32_t)kTcStages) { stage = 0; phase ^= 1u; }
       }
-      if (ok) tc_commit(&sh.accum);
     }
     __syncwarp();
   } else {
-    // accumulator to global memory: warp w may read lanes 32 (w % 4) .. 32 (w % 4) + 31, a token per thread
+    // The sums of kTcSegSteps stages each move from tensor memory to registers, where they are added with
+    // round-to-nearest: the tensor cores add into their accumulator with truncation, whose error grows with the
+    // length of the chain.  Warp w may read lanes 32 (w % 4) .. 32 (w % 4) + 31, a token per thread.
     const int quarter = warp & 3;
-    const bool ok = tc_wait(sh, st, &sh.accum, 0u, 420);
-    tc_fence_after();
-    if (ok) {
-      float *row = Y + (size_t)(m0 + quarter * 32 + lane) * N;
-#pragma unroll 1
+    float sum[kTcN];
+#pragma unroll
+    for (int j = 0; j < kTcN; ++j) sum[j] = 0.f;
+    const int nseg = (nk + kTcSegSteps - 1) / kTcSegSteps;
+    bool ok = true;
+    for (int seg = 0; seg < nseg; ++seg) {
+      const int a = seg % kTcAccs;
+      if (!tc_wait(sh, st, &sh.acc_full[a], (uint32_t)((seg / kTcAccs) & 1), 420)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
       for (int c0 = 0; c0 < kTcN; c0 += 32) {
         uint32_t r[32];
-        tc_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+        tc_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * kTcN + c0), r);
 #pragma unroll
-        for (int j = 0; j < 32; j += 4)
-          if (n0 + c0 + j < N)
-            *reinterpret_cast<float4 *>(row + n0 + c0 + j) =
-                make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+        for (int j = 0; j < 32; ++j) sum[c0 + j] += __uint_as_float(r[j]);
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
+    }
+    if (ok) {
+      float *row = Y + (size_t)(m0 + quarter * 32 + lane) * N + n0;
+#pragma unroll
+      for (int j = 0; j < kTcN; j += 4)
+        if (n0 + j < N) *reinterpret_cast<float4 *>(row + j) = make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tc_dealloc(tmem, kTcN);
+    tc_dealloc(tmem, kTcAccs * kTcN);
   }
 }
 

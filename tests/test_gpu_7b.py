@@ -25,8 +25,8 @@ def big():
     del weights
     dtabs = P.build_ngram_tables(tables, dev)
     torch.cuda.empty_cache()
-    ctx = P.SpdContext(wl.shape, packed, dtabs, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, wl.kv_dtype)
-    cfg = so.make_config(wl.shape, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, wl.kv_dtype)
+    ctx = P.SpdContext(wl.shape, packed, dtabs, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 192, wl.kv_dtype)
+    cfg = so.make_config(wl.shape, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 192, wl.kv_dtype)
     orc = so.Oracle(cfg, host, tables)
     yield wl, ctx, orc, tables, prefix
     ctx.close()
@@ -46,6 +46,24 @@ def test_7b_steps_match_oracle(big):
     assert max(s["eps_z"] for s in errs) < 2e-3
     flips = sum(s.get("cache_flips", 0) for s in stats)
     print("7B parity: max logit error %.3g, cache values rounded the other way: %d" % (max(s["eps_z"] for s in errs), flips))
+
+
+def test_7b_long_prefix_on_tensor_cores(big):
+    """A 150-token prefix at full size: 144 tokens through the tcgen05 products and the tensor-core attention (two
+    jobs, since this context's 192 positions cap a job at 128 tokens: a full tile, then a tile with 16 tokens in
+    it), the last 6 tokens and the first timestep through the 16-token kernel."""
+    wl, ctx, orc, tables, _ = big
+    prefix = si.make_prefix(wl.prefix_kind, 150, wl.shape.vocab, wl.zipf_s, seed=41)
+    stats = []
+    before = ctx.spd_launch_count()
+    compare_first_step(ctx, orc, prefix, stats)
+    assert ctx.spd_launch_count() - before == 2 * 9 * wl.shape.n_layers + 1
+    for _ in range(2):
+        compare_step(ctx, orc, stats)
+    errs = [s for s in stats if "eps_z" in s]
+    assert max(s["eps_z"] for s in errs) < 2e-3
+    flips = sum(s.get("cache_flips", 0) for s in stats)
+    print("7B long prefix: max logit error %.3g, cache values rounded the other way: %d" % (max(s["eps_z"] for s in errs), flips))
 
 
 def test_7b_one_launch_equals_single_steps(big):
