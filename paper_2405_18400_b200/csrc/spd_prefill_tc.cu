@@ -116,7 +116,7 @@ __device__ __forceinline__ bool tc_wait(TcShared &sh, State *st, uint64_t *bar, 
 
 // Y[m0 .. m0+127][n0 .. n0+127] of Y = X W^T.  tmap_x: the term tiles, a [3 * x_term_rows][C] bf16 matrix in boxes
 // of 128 rows x 64 columns (term j's tokens start at row j * x_term_rows); tmap_w: W [N][C] in boxes of 32 rows x
-// 64 columns.  Rows and columns past either matrix arrive as zeros.  grid = (ceil(N / 128), tokens / 128).
+// 64 columns.  Rows and columns past either matrix arrive as zeros.  grid = (ceil(tokens / 128), ceil(N / 128)).
 __global__ void __launch_bounds__(kTcThreads, 1)
     spd_tc_gemm_kernel(const void *tmap_x, const void *tmap_w, float *Y, int N, int C, int x_term_rows, State *st) {
   extern __shared__ __align__(16) uint8_t tc_smem_raw[];
@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   __shared__ TcShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nk = (C + kTcKB - 1) / kTcKB;
-  const int n0 = blockIdx.x * kTcN, m0 = blockIdx.y * kTcM;
+  const int m0 = blockIdx.x * kTcM, n0 = blockIdx.y * kTcN;  // token tiles vary fastest: blocks that share weight rows run together
   if (threadIdx.x == 0) {
     sh.dead = 0;
     for (int s = 0; s < kTcStages; ++s) {
@@ -177,7 +177,6 @@ __global__ void __launch_bounds__(kTcThreads, 1)
     if (lane == 0) {
       const uint32_t idesc = tc_idesc(kTcM, kTcN);
       uint32_t stage = 0, phase = 0;
-      bool ok = true;
       for (int ks = 0; ks < nk; ++ks) {
         const int seg = ks / kTcSegSteps, in_seg = ks - seg * kTcSegSteps, a = seg % kTcAccs;
         if (in_seg == 0 && !tc_wait(sh, st, &sh.acc_empty[a], (uint32_t)((seg / kTcAccs) & 1) ^ 1u, 430)) break;  // its last sum has been read
@@ -655,7 +654,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
   cudaError_t e = cudaSuccess;
   auto gemm = [&](const uint8_t *xmap, int which, int N, int C) {
     if (e != cudaSuccess) return;
-    const dim3 grid((N + spd::kTcN - 1) / spd::kTcN, (n + spd::kTcM - 1) / spd::kTcM);
+    const dim3 grid((n + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
     spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, j.w_tmaps + (size_t)which * spd::kTensorMapBytes, j.y, N, C,
                                                                          j.x_term_rows, j.st);
     e = cudaGetLastError();
