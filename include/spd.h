@@ -270,6 +270,15 @@ int spd_score_static(const spd_config *cfg, const spd_ngram_table *tables, int32
  */
 int spd_debug_expire(spd_ctx *ctx);
 
+/*
+ * The same for the long-prefix path's products (tcgen05 kernel): one tile is launched whose producer announces
+ * its first stage of operands but never copies it, so that the issuing thread's wait for that stage (1.5 s) runs
+ * out; the block records SPD_ETIMEOUT, waits for the copies it did issue, frees its tensor memory and returns.
+ * Returns what the device recorded.  SPD_ESTATE when the context has no long-prefix path (max_pos < 130 or a head
+ * size other than 64 or 128).  The context stays usable: prefill it again.
+ */
+int spd_debug_expire_products(spd_ctx *ctx);
+
 /* Number of kernel launches this context has enqueued so far. */
 int64_t spd_launch_count(const spd_ctx *ctx);
 

@@ -66,7 +66,7 @@ _lib: Optional[C.CDLL] = None
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
            "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
-           "spd_sample", "spd_debug_nucleus", "spd_debug_expire"]
+           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products"]
 
 
 def load_library() -> C.CDLL:
@@ -105,6 +105,7 @@ def load_library() -> C.CDLL:
     L.spd_debug_score.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_debug_nucleus.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_void_p]
     L.spd_debug_expire.argtypes = [C.c_void_p]
+    L.spd_debug_expire_products.argtypes = [C.c_void_p]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
     L.spd_set_ring.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
@@ -242,6 +243,10 @@ class SpdContext:
     def spd_debug_expire(self) -> int:
         """Status the device recorded when one block withheld its barrier arrival (SPD_ETIMEOUT = -7)."""
         return int(self.lib.spd_debug_expire(self.h))
+
+    def spd_debug_expire_products(self) -> int:
+        """Status the device recorded when a stage of the long-prefix products never arrived (SPD_ETIMEOUT = -7)."""
+        return int(self.lib.spd_debug_expire_products(self.h))
 
     def spd_debug_nucleus(self, logits, top_p: float, temperature: float, u: float) -> int:
         z = np.ascontiguousarray(logits, dtype=np.float32)

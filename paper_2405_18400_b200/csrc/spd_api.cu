@@ -214,6 +214,28 @@ int launch(spd_ctx *ctx, int mode, int n_iters, int pos0, int step0) {
   return SPD_OK;
 }
 
+// The long-prefix path's view of a context (tokens and positions are filled in per job).
+spd::TcJob tc_job(spd_ctx *ctx) {
+  const spd::KParams &kp = ctx->kp;
+  spd::TcJob job;
+  job.L = kp.L; job.d = kp.d; job.H = kp.H; job.hd = kp.hd; job.f = kp.f; job.max_pos = kp.max_pos; job.kv_bf16 = kp.kv_bf16;
+  job.eps = kp.eps;
+  job.layers = ctx->layers_host.data();
+  job.tok_emb = kp.tok_emb;
+  job.w_tmaps = ctx->ws + ctx->lay.pf_tmaps;
+  job.x_tmaps = ctx->ws + ctx->lay.tc_tmaps;
+  job.kcache = kp.kcache; job.vcache = kp.vcache; job.rope = kp.rope;
+  job.h = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_h);
+  job.y = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_y);
+  job.q = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_q);
+  job.x = reinterpret_cast<uint16_t *>(ctx->ws + ctx->lay.tc_x);
+  job.x_term_rows = ctx->tc_rows;
+  job.st = kp.st;
+  job.ids = nullptr;
+  job.pos0 = job.n_tok = 0;
+  return job;
+}
+
 // Runs prefix tokens [first, first + count) (positions alike), the last of which ends the prefix, through the
 // prefill kernel, kPfTokens at a time: their keys and values enter the cache, and the last launch goes on to
 // the LM head on the prefix's last token and the first timestep (Eq. 1).
@@ -226,20 +248,7 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
   if (ctx->tc_rows > 0 && count > spd::kTcTile) {
     const int tc_total = count - ((count - 1) % spd::kPfTokens + 1);
     SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream));
-    spd::TcJob job;
-    job.L = kp.L; job.d = kp.d; job.H = kp.H; job.hd = kp.hd; job.f = kp.f; job.max_pos = kp.max_pos; job.kv_bf16 = kp.kv_bf16;
-    job.eps = kp.eps;
-    job.layers = ctx->layers_host.data();
-    job.tok_emb = kp.tok_emb;
-    job.w_tmaps = ctx->ws + ctx->lay.pf_tmaps;
-    job.x_tmaps = ctx->ws + ctx->lay.tc_tmaps;
-    job.kcache = kp.kcache; job.vcache = kp.vcache; job.rope = kp.rope;
-    job.h = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_h);
-    job.y = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_y);
-    job.q = reinterpret_cast<float *>(ctx->ws + ctx->lay.tc_q);
-    job.x = reinterpret_cast<uint16_t *>(ctx->ws + ctx->lay.tc_x);
-    job.x_term_rows = ctx->tc_rows;
-    job.st = kp.st;
+    spd::TcJob job = tc_job(ctx);
     while (tc_done < tc_total) {
       const int n = tc_total - tc_done < ctx->tc_rows ? tc_total - tc_done : ctx->tc_rows;
       job.ids = base + first + tc_done;
@@ -805,6 +814,20 @@ int spd_debug_expire(spd_ctx *ctx) {
   if (e == cudaSuccess) e = spd_internal_prefill_launch(&kp, ctx->grid, ctx->stream);
   kp.pf_stall = 0;
   if (e != cudaSuccess) return cuda_fail(e, "prefill launch");
+  ctx->launches += 1;
+  return check_device_error(ctx);
+}
+
+int spd_debug_expire_products(spd_ctx *ctx) {
+  if (!ctx) return SPD_EINVAL;
+  if (ctx->tc_rows == 0) return SPD_ESTATE;
+  int rc = set_device(ctx);
+  if (rc) return rc;
+  ctx->prefilled = false;
+  const spd::TcJob job = tc_job(ctx);
+  cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream);
+  if (e == cudaSuccess) e = spd_internal_tc_stall(&job, ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(e, "long-prefix launch");
   ctx->launches += 1;
   return check_device_error(ctx);
 }

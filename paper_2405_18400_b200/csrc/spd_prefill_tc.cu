@@ -117,8 +117,10 @@ __device__ __forceinline__ bool tc_wait(TcShared &sh, State *st, uint64_t *bar, 
 // Y[m0 .. m0+127][n0 .. n0+127] of Y = X W^T.  tmap_x: the term tiles, a [3 * x_term_rows][C] bf16 matrix in boxes
 // of 128 rows x 64 columns (term j's tokens start at row j * x_term_rows); tmap_w: W [N][C] in boxes of 32 rows x
 // 64 columns.  Rows and columns past either matrix arrive as zeros.  grid = (ceil(tokens / 128), ceil(N / 128)).
+// stall (test hook): the producer announces its first stage but issues no copies for it, so the wait for that
+// stage runs out.
 __global__ void __launch_bounds__(kTcThreads, 1)
-    spd_tc_gemm_kernel(const void *tmap_x, const void *tmap_w, float *Y, int N, int C, int x_term_rows, State *st) {
+    spd_tc_gemm_kernel(const void *tmap_x, const void *tmap_w, float *Y, int N, int C, int x_term_rows, State *st, int stall) {
   extern __shared__ __align__(16) uint8_t tc_smem_raw[];
   uint8_t *smem = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
   __shared__ TcShared sh;
@@ -153,6 +155,10 @@ __global__ void __launch_bounds__(kTcThreads, 1)
         if (!tc_wait(sh, st, &sh.empty[stage], phase ^ 1u, 400)) { ok = false; break; }
         mbar_expect_tx(&sh.full[stage], (uint32_t)kTcStageBytes);
         const uint32_t base = ring + stage * (uint32_t)kTcStageBytes;
+        if (stall && ks == 0) {
+          if (++stage == (uint32_t)kTcStages) { stage = 0; phase ^= 1u; }
+          continue;  // nothing in flight for this stage
+        }
 #pragma unroll
         for (int j = 0; j < 3; ++j) tc_box_load(base + j * kTcTermBytes, tmap_x, ks * kTcKB, j * x_term_rows + m0, &sh.full[stage]);
 #pragma unroll
@@ -641,6 +647,13 @@ extern "C" cudaError_t spd_internal_tc_prepare(void) {
   return e;
 }
 
+// Test hook: one tile of the first layer's QKV product whose first stage never arrives (see the kernel's `stall`).
+extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t s) {
+  const spd::TcJob &j = *job;
+  spd::spd_tc_gemm_kernel<<<dim3(1, 1), spd::kTcThreads, tc_gemm_smem(), s>>>(j.x_tmaps, j.w_tmaps, j.y, 3 * j.d, j.d, j.x_term_rows, j.st, 1);
+  return cudaGetLastError();
+}
+
 // Enqueues the decoder over j.n_tok tokens (at most j.x_term_rows) at positions j.pos0 ..: their keys and values
 // enter the cache.  The products run over whole tiles of 128 tokens: the rows past n_tok of the last tile hold
 // whatever an earlier job left, give rows of Y that nothing reads (a row of Y depends on its own token only).
@@ -656,7 +669,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
     if (e != cudaSuccess) return;
     const dim3 grid((n + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
     spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, j.w_tmaps + (size_t)which * spd::kTensorMapBytes, j.y, N, C,
-                                                                         j.x_term_rows, j.st);
+                                                                         j.x_term_rows, j.st, 0);
     e = cudaGetLastError();
     ++count;
   };

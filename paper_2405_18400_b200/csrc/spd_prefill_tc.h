@@ -27,4 +27,5 @@ struct TcJob {
 }  // namespace spd
 
 extern "C" cudaError_t spd_internal_tc_prepare(void);
+extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);

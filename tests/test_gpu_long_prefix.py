@@ -65,3 +65,32 @@ def test_reset_after_long_prefix(tiny_inputs):
     compare_first_step(ctx, orc, None, reset_draft=1)
     compare_step(ctx, orc)
     ctx.close()
+
+
+def test_expired_wait_in_the_products_is_reported_and_the_context_stays_usable(tiny_inputs):
+    """A stage of operands that never arrives: the issuing thread's bounded wait runs out, the block records
+    SPD_ETIMEOUT, frees its tensor memory and ends by itself; the same context then prefills a long prefix as a
+    fresh one does.  A context without the long-prefix path refuses the hook."""
+    import time
+    import paper_2405_18400_b200 as P
+    wl, _, _, _ = tiny_inputs
+    prefix = si.make_prefix("zipf", 300, wl.shape.vocab, 1.1, seed=77)
+    ctx, _ = make_tiny_pair(tiny_inputs, max_pos=512)
+    ref, _ = make_tiny_pair(tiny_inputs, max_pos=512)
+    ids0, g0 = ref.spd_prefill(prefix)
+    t0 = time.perf_counter()
+    status = ctx.spd_debug_expire_products()
+    dt = time.perf_counter() - t0
+    assert status == -7
+    assert 1.0 < dt < 10.0
+    with pytest.raises(P.SpdError) as e:            # no drafts to continue
+        ctx.spd_step()
+    assert e.value.status == -2
+    ids, g = ctx.spd_prefill(prefix)
+    assert ids.tolist() == ids0.tolist() and np.array_equal(g, g0)
+    a, _, _ = ctx.spd_generate(4, 5)
+    b, _, _ = ref.spd_generate(4, 5)
+    assert a.tolist() == b.tolist()
+    small, _ = make_tiny_pair(tiny_inputs, max_pos=64)
+    assert small.spd_debug_expire_products() == -2
+    ctx.close(); ref.close(); small.close()
