@@ -51,6 +51,16 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
+def measured_peak_bf16():
+    """Dense bf16 peak of a kernel timed alone (the driver's cuBLAS burst figure), TFLOP/s."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
 def step_bytes(wl, k, T):
     """Algorithmic bytes one decode step must move: every weight once, norm gains, k embedding rows,
     the KV cache of T positions, one 32-byte sector per table probe."""
@@ -231,6 +241,30 @@ def run_ours(args, wl):
            "ms_per_request": e2e_s * 1e3 if e2e_s else None,
            "ms_to_first_drafts": min(first_t) * 1e3 if first_t else None}
 
+    # ---- long prefixes: the prefill alone, device-timed, against the tensor roofline of its tcgen05 products
+    prefill_rec = None
+    if wl.prefix_len > 128 and not args.no_e2e:
+        ts = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.spd_prefill(prefix)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        pf_ms = max_over_ranks(float(np.median(ts)), dev, world)
+        n_tc = wl.prefix_len - ((wl.prefix_len - 1) % 16 + 1)
+        sh = wl.shape
+        layer_params = sh.n_layers * (4 * sh.d_model * sh.d_model + 3 * sh.d_model * sh.d_ffn)
+        tflop = n_tc * layer_params * 2 * 3 / 1e12
+        tpeak, tkind = measured_peak_bf16()
+        prefill_rec = {"ms": pf_ms, "tokens": wl.prefix_len, "tokens_through_tcgen05_products": n_tc, "bound": "tensor",
+                       "achieved": tflop / (pf_ms * 1e-3), "peak": tpeak, "unit": "TFLOP/s", "frac": tflop / (pf_ms * 1e-3) / tpeak,
+                       "peak_kind": tkind,
+                       "note": "whole spd_prefill call (products, attention, row-wise kernels, the last tokens' launch of the 16-token "
+                               "kernel with LM head and first timestep); arithmetic = tokens x layer weights x 2 x 3 bf16 terms per float32 activation"}
+
     # ---- the same number of drafts from k separate single-draft passes through the same kernels
     kpass = None
     if rank == 0 and not args.no_kpass and k > 1:
@@ -277,6 +311,8 @@ def run_ours(args, wl):
     }
     if kpass:
         out["k_pass"] = kpass
+    if prefill_rec:
+        out["prefill"] = prefill_rec
     ctx.close()
 
     if rank == 0 and host_weights is not None:
