@@ -94,3 +94,35 @@ def test_expired_wait_in_the_products_is_reported_and_the_context_stays_usable(t
     small, _ = make_tiny_pair(tiny_inputs, max_pos=64)
     assert small.spd_debug_expire_products() == -2
     ctx.close(); ref.close(); small.close()
+
+
+def test_long_prefix_13b_width():
+    """Two layers at the 13B shape's width (d_model 5120, 40 heads of 128, d_ffn 13824): 80 and 216 stages per
+    row (10 and 27 accumulator segments, so the four accumulators are reused several times), 120 / 40 / 216 / 40
+    row tiles, a job of 512 tokens and a partial one."""
+    import torch
+    import paper_2405_18400_b200 as P
+    from oracle import spd_oracle as so
+
+    shape = si.ModelShape("w13b", 2, 5120, 40, 13824, 2000)
+    dev = torch.device("cuda:0")
+    weights = si.make_weights(shape, seed=21, device=dev)
+    host = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in weights.items()}
+    tables = si.make_ngram_tables(shape.vocab, 1.1, 50_000, (2, 3), 5000, seed=22)
+    lam = [0.3, 0.2] + [0.0] * 6
+    packed = P.pack_weights(weights, dev, consume=True)
+    del weights
+    dtabs = P.build_ngram_tables(tables, dev)
+    ctx = P.SpdContext(shape, packed, dtabs, 3, (2, 3), lam, 0.4, 0.2, 0.05, 640, "bf16")
+    cfg = so.make_config(shape, 3, (2, 3), lam, 0.4, 0.2, 0.05, 640, "bf16")
+    orc = so.Oracle(cfg, host, sorted(tables, key=lambda t: int(t["n"])))
+    m = 600
+    prefix = si.make_prefix("zipf", m, shape.vocab, 1.1, seed=23)
+    stats = []
+    compare_first_step(ctx, orc, prefix, stats)
+    assert ctx.spd_launch_count() == _expected_launches(m, 2, 512)
+    for _ in range(2):
+        compare_step(ctx, orc, stats)
+    assert max(s["eps_z"] for s in stats if "eps_z" in s) < 2e-3
+    ctx.close()
+    orc.close()
