@@ -42,7 +42,7 @@ struct Layout {
       trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, tc_tmaps, tc_h, tc_q, tc_y, tc_x, total;
 };
 
-// Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 128 tokens send
+// Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 64 tokens send
 // all but their last 1..16 tokens through the tensor-core path.
 int tc_rows(const spd_config &c) {
   const int hd = c.d_model / c.n_heads;
@@ -245,7 +245,7 @@ int prefill_tokens(spd_ctx *ctx, int first, int count) {
   int rc = SPD_OK;
   // Long run of tokens: all but the last 1..16 go through the tensor-core path, in jobs of up to tc_rows tokens.
   int tc_done = 0;
-  if (ctx->tc_rows > 0 && count > spd::kTcTile) {
+  if (ctx->tc_rows > 0 && count > spd::kTcMinPrefix) {
     const int tc_total = count - ((count - 1) % spd::kPfTokens + 1);
     SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream));
     spd::TcJob job = tc_job(ctx);

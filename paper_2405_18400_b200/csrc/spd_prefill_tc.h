@@ -6,6 +6,8 @@ namespace spd {
 
 constexpr int kTcTile = 128;      // tokens per tile of the tensor-core products
 constexpr int kTcMaxTokens = 512; // tokens one job takes at most
+constexpr int kTcMinPrefix = 64;  // runs of more tokens than this take the path: a job of up to 128 tokens costs about 2.7 launches
+                                  // of the 16-token kernel (7B shape: 12.6 ms against 4.66 ms), so four launches before the last pay for it
 
 struct TcJob {
   int32_t L, d, H, hd, f, max_pos, kv_bf16;

@@ -1,4 +1,4 @@
-"""Prefixes of more than 128 tokens: all but the last 1..16 tokens go through the tensor-core path (tcgen05
+"""Prefixes of more than 64 tokens: all but the last 1..16 tokens go through the tensor-core path (tcgen05
 products over tiles of 128 tokens, up to 512 tokens per job), the rest through the 16-token prefill kernel,
 which ends with the first timestep (Eq. 1).  Both fill the same cache; the first timestep and the steps after
 it are compared with the oracle as for short prefixes."""
@@ -12,16 +12,16 @@ pytestmark = pytest.mark.gpu
 
 
 def _expected_launches(m, layers, job_tokens):
-    tc = m - ((m - 1) % 16 + 1) if m > 128 else 0
+    tc = m - ((m - 1) % 16 + 1) if m > 64 else 0
     jobs = -(-tc // job_tokens) if tc else 0
     return jobs * 9 * layers + (m - tc + 15) // 16
 
 
 @pytest.mark.parametrize("kv_dtype", ["bf16", "f32"])
-@pytest.mark.parametrize("m", [129, 293, 700])
+@pytest.mark.parametrize("m", [65, 129, 293, 700])
 def test_long_prefix_tiny(tiny_inputs, m, kv_dtype):
     """Tiny shape: d_ffn = 688 leaves a ragged last 64-column stage and 2 d_ffn = 1376 a ragged last row tile;
-    129 = one tile and one token, 293 = one job of 288 tokens (a last tile of 32), 700 = a job of 512 tokens and
+    65 = the shortest prefix that takes the path (a tile with 64 tokens in it), 129 = one tile and one token, 293 = one job of 288 tokens (a last tile of 32), 700 = a job of 512 tokens and
     one of 176."""
     wl, _, _, _ = tiny_inputs
     prefix = si.make_prefix("zipf", m, wl.shape.vocab, 1.1, seed=500 + m)
