@@ -126,3 +126,23 @@ def test_long_prefix_13b_width():
     assert max(s["eps_z"] for s in stats if "eps_z" in s) < 2e-3
     ctx.close()
     orc.close()
+
+
+def test_both_prefill_paths_agree(tiny_inputs):
+    """The same 100-token prefix through the 16-token kernel alone (a context of 128 positions has no long-prefix
+    buffers) and through the long-prefix path (a context of 512 positions): same drafts, logits equal to float
+    rounding, and the same continuation."""
+    wl, _, _, _ = tiny_inputs
+    prefix = si.make_prefix("zipf", 100, wl.shape.vocab, 1.1, seed=4242)
+    a, _ = make_tiny_pair(tiny_inputs, max_pos=128, kv_dtype="f32")
+    b, _ = make_tiny_pair(tiny_inputs, max_pos=512, kv_dtype="f32")
+    ids_a, g_a = a.spd_prefill(prefix)
+    ids_b, g_b = b.spd_prefill(prefix)
+    assert a.spd_launch_count() == 7 and b.spd_launch_count() == 9 * wl.shape.n_layers + 1
+    za, zb = a.spd_debug_read("LOGITS"), b.spd_debug_read("LOGITS")
+    assert np.abs(za - zb).max() < 1e-4
+    assert ids_a.tolist() == ids_b.tolist() and np.abs(g_a - g_b).max() < 1e-3
+    ta, _, _ = a.spd_generate(5, 6)
+    tb, _, _ = b.spd_generate(5, 6)
+    assert ta.tolist() == tb.tolist()
+    a.close(); b.close()
