@@ -29,9 +29,8 @@ import torch
 
 import spd_inputs as si
 
-# dram bytes (read + write) / algorithmic bytes measured by ncu on the 4-layer case of the same kernel
-# (profiles/spd_decode_kernel_7b_k3.md); traffic grows in proportion to the layers streamed.  Set to None
-# whenever the kernel changes until the counters are taken again.
+# dram bytes (read + write) / algorithmic bytes measured by ncu on a 4-layer case of the same kernel; traffic
+# grows in proportion to the layers streamed.  None whenever the kernel has changed since the counters were taken.
 TRAFFIC_RATIO = 1.003
 
 METRIC = "k-draft tokens/s"

@@ -85,7 +85,7 @@ typedef struct {
 } spd_weights;
 
 /*
- * One n-gram order's frequency store (Section 4: "each unique n-gram and its count") as two
+ * One n-gram order's frequency store (Section 4: a table of the distinct n-grams with how often each occurs) as two
  * open-addressing hash tables in DEVICE memory, BORROWED, produced by spd_ngram_build.  A slot is
  * 16 bytes: six uint16 token ids (unused ones 0) then a uint32 count; count 0 marks an empty slot.
  * `ngram` maps n tokens -> count; `ctx` maps the first n-1 tokens -> sum of the counts of all stored
@@ -189,7 +189,8 @@ const char *spd_last_cuda_error(void);
  * HOST int64 counts (> 0).  spd_ngram_plan reports the slot numbers to allocate (powers of two, at
  * least twice the entries); spd_ngram_build fills caller-provided HOST buffers of ngram_slots*16 and
  * ctx_slots*16 bytes, which the caller then copies to the device.  SPD_ERANGE if a token id exceeds
- * 65535 or a count or context total exceeds 2^32-1; SPD_EINVAL if keys are not strictly increasing.
+ * 65535 or a count or context total exceeds 2^32-2 (counts are unsigned 32-bit on the device and
+ * 2^32-1 is reserved); SPD_EINVAL if keys are not strictly increasing.
  */
 int spd_ngram_plan(int32_t n, int64_t n_entries, const int32_t *keys, uint64_t *ngram_slots, uint64_t *ctx_slots);
 int spd_ngram_build(int32_t n, int64_t n_entries, const int32_t *keys, const int64_t *counts, uint64_t ngram_slots,
@@ -203,12 +204,13 @@ int spd_ngram_build(int32_t n, int64_t n_entries, const int32_t *keys, const int
  *   SPD_DBG_LOGP_IN   float [k]            draft log-probabilities before the last step's selection
  *   SPD_DBG_SCORE     float [k*k]          score of option i*k+j (-inf = dropped)
  *   SPD_DBG_PNG       float [k*k]          Eq. 5 value of option i*k+j
- *   SPD_DBG_CNT       int32 [k*k][8]       n-gram count per option and table (-1 = order skipped)
- *   SPD_DBG_TOT       int32 [k][8]         context total per draft and table (-1 = order skipped)
+ *   SPD_DBG_CNT       uint32 [k*k][8]      n-gram count per option and table (0xffffffff = order skipped)
+ *   SPD_DBG_TOT       uint32 [k][8]        context total per draft and table (0xffffffff = order skipped)
  *   SPD_DBG_SEL       int32 [k]            chosen options i*k+j, best first
  *   SPD_DBG_LOGP      float [k]            current draft log-probabilities
  *   SPD_DBG_HIST_IN   int32 [k][8]         last 8 tokens of each draft before the last step's selection (right-aligned)
  *   SPD_DBG_TRACE     float [n_layers][2][d_model]  residual after attention / after the FFN of the last LM pass
+ *                     (recorded only while spd_debug_trace has switched it on; zeros otherwise)
  *   SPD_DBG_HIDDEN    float [d_model]      residual stream after the last LM pass
  *   SPD_DBG_KCACHE    float [n_layers][T][d_model]  cached keys of the T positions written so far (T = prefix
  *                     length + tokens generated - 1), widened to float32;  SPD_DBG_VCACHE likewise for values
@@ -219,6 +221,12 @@ enum {
   SPD_DBG_TOT, SPD_DBG_SEL, SPD_DBG_LOGP, SPD_DBG_HIST_IN, SPD_DBG_TRACE, SPD_DBG_HIDDEN, SPD_DBG_KCACHE, SPD_DBG_VCACHE
 };
 int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes);
+
+/*
+ * Test hook: switches the recording of the per-layer residual trace (SPD_DBG_TRACE) on (on != 0) or off for the
+ * launches that follow.  Off after spd_create, so that the decoding path writes no instrumentation.
+ */
+int spd_debug_trace(spd_ctx *ctx, int on);
 
 /*
  * Test hook for the scoring stage alone (Eq. 2, 4-7): overwrites the draft state with the given
@@ -253,7 +261,8 @@ int spd_debug_nucleus(spd_ctx *ctx, const float *logits, float top_p, float temp
  *            out_gamma float [k] (Eq. 4), out_score float [k*k] (-inf = dropped option).
  * Limits of the fixed scratch: k <= SPD_MAX_K (16), n_tables <= 8, hist_len <= 8; anything larger is
  * refused with SPD_ERANGE.  The first call on each device looks up the array's device address (that
- * device must be current); make that first call before any stream capture begins.  All calls on a
+ * device must be current); make that first call before any stream capture begins (which says nothing about
+ * whether a later call can be captured: no claim is made either way).  All calls on a
  * device share the one array, which still holds the previous call's data when the next begins (each
  * call overwrites it completely before launching); two calls whose device work overlaps, from
  * different streams or threads, race on it, so serialise them.  Synchronises the stream before returning.

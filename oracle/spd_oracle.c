@@ -80,6 +80,7 @@ typedef struct {
   int force_T;
   double force_slack;
   int64_t force_flips, force_bad;
+  double force_need;    /* largest slack an adopted value needed since the last orc_follow_cache */
   /* last step's intermediates */
   int32_t cand_tok[ORC_MAX_K];
   double cand_lp[ORC_MAX_K];
@@ -175,19 +176,40 @@ static float quant_kv(const orc_config *c, double x) {
 /*
  * The cache value for the exact value x.  Rounding to the cache type is a decision that float
  * rounding can tip either way when x lies within rounding error of the midpoint of two
- * representable values.  When the tests supply another implementation's cache value `other`, it is adopted
- * if it is a rounding of some value within `slack` of x (|other - x| below the spacing of the cache type
- * in x's binade plus slack, slack being the caller's bound on the other side's float error in absolute
- * terms: for values near zero that error exceeds the local spacing); anything else is counted as a
- * mismatch and not adopted.
+ * representable values.  When the tests supply another implementation's cache value `other`, it is
+ * adopted only if it is what round-to-nearest gives for some value within `slack` of x, i.e. if
+ * round(x - slack) <= other <= round(x + slack) and `other` is representable (slack = the caller's
+ * bound on the other side's float error in absolute terms).  With slack far below the local spacing
+ * this admits the exact value's other neighbour only when x is within slack of the midpoint; a value
+ * on the far side of the interval (x a tenth of the way from a to b, other = b), a truncation, or
+ * anything further away is counted as a mismatch and not adopted.  Near zero, where the spacing is
+ * below slack, it admits the few values a float error of that size can reach.  force_need keeps the
+ * largest slack any adopted value needed, so that the tests can report how tight their bound is.
  */
+static double kv_neighbour(const orc_config *c, float v, int upwards) {
+  const uint32_t step = c->kv_dtype == 1 ? 0x10000u : 1u;
+  uint32_t u;
+  memcpy(&u, &v, 4);
+  if (v == 0.0f) u = (upwards ? 0u : 0x80000000u) + step;
+  else if ((v > 0.0f) == (upwards != 0)) u += step;   /* away from zero */
+  else u -= step;                                     /* towards zero */
+  float r;
+  memcpy(&r, &u, 4);
+  return (double)r;
+}
+
 static float follow_kv(orc_ctx *o, double x, const float *other) {
   float own = quant_kv(&o->c, x);
   if (!other) return own;
   if (*other == own) return own;
-  double spacing = x == 0.0 ? 0.0 : ldexp(1.0, ilogb(x) - (o->c.kv_dtype == 1 ? 7 : 23));
-  if (fabs((double)*other - x) < spacing + o->force_slack) {
+  const double v = (double)*other;
+  const float lo = quant_kv(&o->c, x - o->force_slack), hi = quant_kv(&o->c, x + o->force_slack);
+  if (quant_kv(&o->c, v) == *other && *other >= lo && *other <= hi) {
+    /* the error that tips the rounding to `other`: distance from x to the nearer end of other's rounding interval */
+    const double need = v > (double)own ? 0.5 * (v + kv_neighbour(&o->c, *other, 0)) - x
+                                        : x - 0.5 * (v + kv_neighbour(&o->c, *other, 1));
     o->force_flips++;
+    if (need > o->force_need) o->force_need = need;
     return *other;
   }
   o->force_bad++;
@@ -584,6 +606,8 @@ void orc_step_commit(orc_ctx *o, const int32_t *sel, const double *new_logP) {
  * follow_kv); NULL switches it off.
  * flips / bad (either may be NULL) report how many values were adopted / refused since the last call.
  */
+double orc_follow_need(const orc_ctx *o) { return o->force_need; }
+
 void orc_follow_cache(orc_ctx *o, const float *k, const float *v, int T, double slack, int64_t *flips, int64_t *bad) {
   if (flips) *flips = o->force_flips;
   if (bad) *bad = o->force_bad;
@@ -592,6 +616,7 @@ void orc_follow_cache(orc_ctx *o, const float *k, const float *v, int T, double 
   o->force_T = T;
   o->force_slack = slack;
   o->force_flips = o->force_bad = 0;
+  o->force_need = 0.0;
 }
 
 /*

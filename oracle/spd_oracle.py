@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
         L.orc_feed_token.argtypes = [C.c_void_p, C.c_int32]
         L.orc_set_logP.argtypes = [C.c_void_p, C.c_void_p]
         L.orc_follow_cache.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_void_p]
+        L.orc_follow_need.argtypes = [C.c_void_p]
+        L.orc_follow_need.restype = C.c_double
         for name in ("orc_logits", "orc_trace", "orc_logP", "orc_gamma_now", "orc_cand_tok", "orc_cand_lp",
                      "orc_scores", "orc_png_last", "orc_cnt_last", "orc_tot_last", "orc_sel_last", "orc_drafts",
                      "orc_kcache", "orc_vcache"):
@@ -205,8 +207,10 @@ class Oracle:
 
     def follow_cache(self, k=None, v=None, slack: float = 0.0):
         """Follow the given cache contents (float32 [L, T, d]) in later passes; returns (adopted, refused)
-        counts accumulated since the previous call.  slack = absolute float error allowed for the other side."""
+        counts accumulated since the previous call.  slack = absolute float error allowed for the other side.
+        `follow_need` then holds the largest slack any adopted value needed over that period."""
         flips, bad = C.c_int64(), C.c_int64()
+        self.follow_need = float(lib().orc_follow_need(self.h))
         if k is None:
             self._fk = self._fv = None
             lib().orc_follow_cache(self.h, None, None, 0, 0.0, C.byref(flips), C.byref(bad))

@@ -66,7 +66,7 @@ _lib: Optional[C.CDLL] = None
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
            "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
-           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products"]
+           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace"]
 
 
 def load_library() -> C.CDLL:
@@ -105,6 +105,7 @@ def load_library() -> C.CDLL:
     L.spd_debug_score.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_debug_nucleus.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_void_p]
     L.spd_debug_expire.argtypes = [C.c_void_p]
+    L.spd_debug_trace.argtypes = [C.c_void_p, C.c_int]
     L.spd_debug_expire_products.argtypes = [C.c_void_p]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
@@ -240,6 +241,9 @@ class SpdContext:
         _check(self.lib.spd_reset(self.h, int(draft), ids.ctypes.data, g.ctypes.data), "spd_reset")
         return ids, g
 
+    def spd_debug_trace(self, on: bool) -> None:
+        _check(self.lib.spd_debug_trace(self.h, 1 if on else 0), "spd_debug_trace")
+
     def spd_debug_expire(self) -> int:
         """Status the device recorded when one block withheld its barrier arrival (SPD_ETIMEOUT = -7)."""
         return int(self.lib.spd_debug_expire(self.h))
@@ -301,7 +305,7 @@ class SpdContext:
         k, c = self.k, self.cfg
         shapes = {"LOGITS": (np.float32, (c.vocab,)), "CAND_TOK": (np.int32, (k,)), "CAND_LP": (np.float32, (k,)),
                   "LOGP_IN": (np.float32, (k,)), "SCORE": (np.float32, (k * k,)), "PNG": (np.float32, (k * k,)),
-                  "CNT": (np.int32, (k * k, 8)), "TOT": (np.int32, (k, 8)), "SEL": (np.int32, (k,)),
+                  "CNT": (np.uint32, (k * k, 8)), "TOT": (np.uint32, (k, 8)), "SEL": (np.int32, (k,)),
                   "LOGP": (np.float32, (k,)), "HIST_IN": (np.int32, (k, 8)),
                   "TRACE": (np.float32, (c.n_layers, 2, c.d_model)), "HIDDEN": (np.float32, (c.d_model,))}
         if what in ("KCACHE", "VCACHE"):
@@ -309,6 +313,10 @@ class SpdContext:
         dt, shp = shapes[what]
         out = np.zeros(shp, dt)
         _check(self.lib.spd_debug_read(self.h, DBG[what], out.ctypes.data, out.nbytes), "spd_debug_read")
+        if what in ("CNT", "TOT"):      # unsigned 32-bit on the device, 0xffffffff = order skipped: as int64 with -1
+            wide = out.astype(np.int64)
+            wide[out == np.uint32(0xffffffff)] = -1
+            return wide
         return out
 
     def spd_debug_score(self, hist: np.ndarray, logp, cand_tok, cand_lp) -> None:

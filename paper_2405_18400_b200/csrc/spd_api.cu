@@ -414,7 +414,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.hist_tok = reinterpret_cast<int32_t *>(ws + lay.hist_tok); kp.hist_par = reinterpret_cast<int32_t *>(ws + lay.hist_par);
   kp.prefix = reinterpret_cast<int32_t *>(ws + lay.prefix);
   kp.ns_u = reinterpret_cast<const float *>(ws + lay.ns_u);
-  kp.trace = reinterpret_cast<float *>(ws + lay.trace);
+  kp.trace = nullptr;  // the per-layer residual trace is test instrumentation: spd_debug_trace switches it on
   kp.pf_h = reinterpret_cast<float *>(ws + lay.pf_h); kp.pf_q = reinterpret_cast<float *>(ws + lay.pf_q);
   kp.pf_xh = reinterpret_cast<uint16_t *>(ws + lay.pf_xh); kp.pf_xo = reinterpret_cast<uint16_t *>(ws + lay.pf_xo);
   kp.pf_xu = reinterpret_cast<uint16_t *>(ws + lay.pf_xu);
@@ -750,6 +750,12 @@ int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes) {
     }
     default: return SPD_EINVAL;
   }
+}
+
+int spd_debug_trace(spd_ctx *ctx, int on) {
+  if (!ctx) return SPD_EINVAL;
+  ctx->kp.trace = on ? reinterpret_cast<float *>(ctx->ws + ctx->lay.trace) : nullptr;
+  return SPD_OK;
 }
 
 int spd_debug_score(spd_ctx *ctx, const int32_t *hist, int32_t hist_len, const float *logp, const int32_t *cand_tok,

@@ -27,6 +27,7 @@ namespace spd {
 
 constexpr unsigned long long kWaitNs = 1500ull * 1000ull * 1000ull;  // 1.5 s per wait
 constexpr int kErrTable = -6, kErrTimeout = -7;
+constexpr uint32_t kSkipped = 0xffffffffu;  // in the count / total arrays: this order does not apply to the draft
 
 // ---------------------------------------------------------------- block context
 struct Blk {
@@ -635,13 +636,14 @@ __device__ void attention_phase(Blk &b, int layer, int pos) {
 }
 
 // ---------------------------------------------------------------- the method's tail (block 0)
-__device__ __forceinline__ int probe(Blk &b, const SpdSlot *tab, uint64_t mask, uint32_t w0, uint32_t w1, uint32_t w2) {
+// Count stored under the key (1 .. 2^32 - 2), 0 when the key is absent.
+__device__ __forceinline__ uint32_t probe(Blk &b, const SpdSlot *tab, uint64_t mask, uint32_t w0, uint32_t w1, uint32_t w2) {
   uint64_t idx = spd_key_hash(w0, w1, w2) & mask;
   const uint64_t limit = mask + 1 < 16384 ? mask + 1 : 16384;
   for (uint64_t i = 0; i < limit; ++i) {
     const uint4 s = __ldg(reinterpret_cast<const uint4 *>(tab + idx));
     if (s.w == 0u) return 0;
-    if (s.x == w0 && s.y == w1 && s.z == w2) return (int)s.w;
+    if (s.x == w0 && s.y == w1 && s.z == w2) return s.w;
     idx = (idx + 1) & mask;
   }
   if (mask + 1 > limit) give_up(b, kErrTable, 400);
@@ -654,8 +656,8 @@ __device__ void tail_score_select(Blk &b, bool first, int step) {
   const KParams &p = *b.p;
   State *st = p.st;
   const int tid = threadIdx.x, k = p.k, nt = p.n_tables;
-  int *s_cnt = reinterpret_cast<int *>(b.part);           // [k*k][8]
-  int *s_tot = s_cnt + kMaxK * kMaxK * kMaxTables;         // [k][8]
+  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(b.part);  // [k*k][8]; kSkipped where the order does not apply
+  uint32_t *s_tot = s_cnt + kMaxK * kMaxK * kMaxTables;    // [k][8]
   float *s_png = reinterpret_cast<float *>(s_tot + kMaxK * kMaxTables);  // [k*k]
   float *s_score = s_png + kMaxK * kMaxK;                  // [k*k]
   named_sync(1, kConsumerThreads);
@@ -678,7 +680,7 @@ __device__ void tail_score_select(Blk &b, bool first, int step) {
         ti = r % nt;
       }
       const TableDev &tb = p.tab[ti];
-      int res = -1;
+      uint32_t res = kSkipped;
       if (tb.n >= p.n_min && tb.n <= p.n_max && wl >= tb.n - 1) {
         int32_t key[6];
 #pragma unroll
@@ -698,10 +700,10 @@ __device__ void tail_score_select(Blk &b, bool first, int step) {
       const int i = tid / k;
       float png = 0.f;
       for (int ti = 0; ti < nt; ++ti) {
-        const int c = s_cnt[tid * kMaxTables + ti], t = s_tot[i * kMaxTables + ti];
+        const uint32_t c = s_cnt[tid * kMaxTables + ti], t = s_tot[i * kMaxTables + ti];
         st->cnt[tid][ti] = c;
         if (tid % k == 0) st->tot[i][ti] = t;
-        if (t > 0) png = fmaf(p.lambda[p.tab[ti].n - 2], (float)c / (float)t, png);
+        if (t != kSkipped && t > 0u) png = fmaf(p.lambda[p.tab[ti].n - 2], (float)c / (float)t, png);
       }
       s_png[tid] = png;
       st->png[tid] = png;

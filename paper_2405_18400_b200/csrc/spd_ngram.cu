@@ -60,14 +60,14 @@ int spd_ngram_build(int32_t n, int64_t n_entries, const int32_t *keys, const int
   uint64_t total = 0;
   for (int64_t i = 0; i < n_entries; ++i) {
     const int32_t *row = keys + i * n;
-    if (counts[i] <= 0 || counts[i] > 0xffffffffll) return SPD_ERANGE;
+    if (counts[i] <= 0 || counts[i] > 0xfffffffell) return SPD_ERANGE;
     uint32_t w0, w1, w2;
     spd_pack_key(row, n, w0, w1, w2);
     insert(ng, ngram_slots - 1, w0, w1, w2, (uint32_t)counts[i]);
     total += (uint64_t)counts[i];
     // the context's total is written when its run of entries ends
     if (i + 1 == n_entries || compare_rows(row, row + n, n - 1) != 0) {
-      if (total > 0xffffffffull) return SPD_ERANGE;
+      if (total > 0xfffffffeull) return SPD_ERANGE;
       spd_pack_key(row, n - 1, w0, w1, w2);
       insert(cx, ctx_slots - 1, w0, w1, w2, (uint32_t)total);
       total = 0;

@@ -49,8 +49,8 @@ struct State {
   float logP_in[kMaxK];
   int32_t win_in[kMaxK][kWin];
   float score[kMaxK * kMaxK], png[kMaxK * kMaxK];
-  int32_t cnt[kMaxK * kMaxK][kMaxTables];
-  int32_t tot[kMaxK][kMaxTables];
+  uint32_t cnt[kMaxK * kMaxK][kMaxTables];  // 0xffffffff: order skipped
+  uint32_t tot[kMaxK][kMaxTables];
   int32_t sel[kMaxK];
 };
 

@@ -35,24 +35,40 @@ def top_gap(values, k):
     return float(np.min(-np.diff(v))) if v.size > 1 else math.inf
 
 
-def _follow(ctx, orc, positions):
+U32 = 2.0 ** -24      # unit roundoff of float32
+
+# Bound on the device's float error in a cache value before it is rounded to bf16, in units of
+# U32 * (layers + 1) * rms(cache).  A cache value of layer l is a float32 dot product over d terms (error of a
+# few U32 relative to the rms of the values, the partial sums being added as a tree) of a residual stream
+# that carries the errors of the l layers before it, each of the same kind; the sum grows at most linearly in
+# l.  Decode steps accumulate in float32 with round-to-nearest (measured: need <= ~3 of these units); the
+# prefill kernels accumulate inside the tensor cores, which truncate every addition of a 96-instruction chain
+# (measured: need <= ~40 units).  The constants leave a factor of about four over what was measured.
+SLACK_UNITS = {"decode": 12.0, "prefill": 160.0}
+# Share of the new cache values that may round the other way (measured: 0.1 % on decode steps, 1 % in prefill).
+FLIP_RATE = {"decode": 0.004, "prefill": 0.03}
+
+
+def _follow(ctx, orc, positions, path):
     """With a bf16 cache the oracle adopts the device's cache values wherever they are a valid rounding of its
     own exact values (rounding is a decision float error can tip; the rest of the pass is then comparable)."""
     if orc.cfg.kv_dtype != 1:
         return False
     kc, vc = ctx.spd_debug_read("KCACHE", positions), ctx.spd_debug_read("VCACHE", positions)
-    # the device accumulates in float32: allow its values an absolute error of 2e-5 of the cache's scale
-    orc.follow_cache(kc, vc, slack=2e-5 * float(max(np.abs(kc).max(), np.abs(vc).max())))
+    rms = math.sqrt(0.5 * (float(np.mean(kc.astype(np.float64) ** 2)) + float(np.mean(vc.astype(np.float64) ** 2))))
+    orc._slack_unit = U32 * (orc.cfg.n_layers + 1) * rms
+    orc.follow_cache(kc, vc, slack=SLACK_UNITS[path] * orc._slack_unit)
     return True
 
 
-def _followed(orc, new_positions, stats):
+def _followed(orc, new_positions, stats, path):
     flips, bad = orc.follow_cache(None)
     total = 2 * orc.cfg.n_layers * orc.cfg.d_model * new_positions
     assert bad == 0, "%d cache values are not a rounding of the oracle's" % bad
-    assert flips <= 0.02 * total + 8, (flips, total)
+    assert flips <= FLIP_RATE[path] * total + 8, (flips, total)
     if stats is not None:
-        stats.append({"cache_flips": flips, "cache_values": total})
+        stats.append({"cache_flips": flips, "cache_values": total, "path": path,
+                      "slack_units_needed": orc.follow_need / orc._slack_unit})
 
 
 def _sync_logp(ctx, orc, eps_z):
@@ -74,10 +90,10 @@ def compare_first_step(ctx, orc, prefix, stats=None, reset_draft=None, device=No
     else:
         prefix = orc.drafts()[reset_draft].tolist()
         ids, g = ctx.spd_reset(reset_draft)
-    following = _follow(ctx, orc, len(prefix))
+    following = _follow(ctx, orc, len(prefix), "prefill")
     ids_o, g_o = orc.prefill(prefix)
     if following:
-        _followed(orc, len(prefix), stats)
+        _followed(orc, len(prefix), stats, "prefill")
     z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
     eps_z = float(np.abs(z - z_o).max())
     assert eps_z <= LOGIT_TOL, eps_z
@@ -101,10 +117,10 @@ def compare_step(ctx, orc, stats=None):
     hist_o = orc.drafts()
     logP_o = orc.logP()
     ids, par, g = ctx.spd_step()
-    following = _follow(ctx, orc, orc.T() + 1)
+    following = _follow(ctx, orc, orc.T() + 1, "decode")
     orc.step_forward()
     if following:
-        _followed(orc, 1, stats)
+        _followed(orc, 1, stats, "decode")
     z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
     eps_z = float(np.abs(z - z_o).max())
     assert eps_z <= LOGIT_TOL, eps_z
@@ -147,3 +163,91 @@ def compare_step(ctx, orc, stats=None):
         stats.append({"eps_z": eps_z, "eps_s": eps_s, "dgamma": dg, "tie_free": tie_free})
     _sync_logp(ctx, orc, eps_z)
     return ids, par, g
+
+
+def free_run(ctx, orc, prefix, n_steps, perturb_logP=None):
+    """The whole request on both sides with NO forcing: the oracle never sees the device's cache or its
+    log-probabilities.  The only following is the margin rule's: on a step whose oracle margins are below twice the
+    measured float error the oracle takes the device's (checked) choice.  Nothing is asserted here: every timestep
+    gives a record with the measured logit error `eps_z`, the bound `acc` on gamma's error that the logit errors so
+    far imply (accumulated 4 eps / tau), and the verdicts `logits_ok` (within LOGIT_TOL), `ints_ok` (kept tokens,
+    n-gram counts and totals exact; choices and parents exact on tie-free steps, else within the margin) and
+    `gamma_ok` (within max(GAMMA_TOL, acc)).  The comparison stops where the drafts part.
+
+    `ctx` may be a second oracle instead of the device context (same read-outs through `_OracleAsDevice`), which
+    shows how two exact implementations drift apart from a float-sized difference alone."""
+    k, tau = ctx.k, orc.cfg.tau
+    rec = []
+    ids, g = ctx.spd_prefill(prefix)
+    if perturb_logP is not None:
+        perturb_logP(ctx)
+    ids_o, g_o = orc.prefill(prefix)
+    z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
+    eps_z = float(np.abs(z - z_o).max())
+    acc = 4 * eps_z / tau
+    same = ids.tolist() == ids_o.tolist()
+    dg = float(np.abs(g - g_o).max())
+    rec.append({"eps_z": eps_z, "acc": acc, "dgamma": dg, "same": same, "tie_free": top_gap(z_o, k) > 2 * eps_z,
+                "logits_ok": eps_z <= LOGIT_TOL, "ints_ok": same, "gamma_ok": dg <= max(GAMMA_TOL, acc)})
+    for _ in range(n_steps):
+        if not same:
+            break
+        ids, par, g = ctx.spd_step()
+        orc.step_forward()
+        z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
+        eps_z = float(np.abs(z - z_o).max())
+        acc += 4 * eps_z / tau
+        cand, cand_o = ctx.spd_debug_read("CAND_TOK"), orc.cand_tok()
+        sel_o, _, _ = orc.step_score()
+        sel = ctx.spd_debug_read("SEL")
+        sc, sc_o = ctx.spd_debug_read("SCORE").astype(np.float64), orc.scores()
+        fin = np.isfinite(sc_o)
+        nt = orc.tables.n
+        r = {"eps_z": eps_z, "acc": acc, "logits_ok": eps_z <= LOGIT_TOL, "gamma_ok": False,
+             "near_tie_logits": top_gap(z_o, k) <= 2 * eps_z}
+        same = (cand.tolist() == cand_o.tolist() and np.array_equal(np.isfinite(sc), fin)
+                and np.array_equal(ctx.spd_debug_read("CNT")[:, :nt], orc.counts())
+                and np.array_equal(ctx.spd_debug_read("TOT")[:, :nt], orc.totals()))
+        if same:
+            eps_s = float(np.abs(sc[fin] - sc_o[fin]).max())
+            r["eps_s"] = eps_s
+            r["tie_free"] = top_gap(sc_o, k) > 2 * eps_s
+            if r["tie_free"]:
+                same = sel.tolist() == sel_o.tolist()
+            else:
+                kth = np.sort(sc_o[fin])[::-1][k - 1]
+                same = all(sc_o[q] >= kth - 2 * eps_s for q in sel) and len(set(sel.tolist())) == k
+            same = same and par.tolist() == (sel // k).tolist() and ids.tolist() == cand[sel % k].tolist()
+        if same:
+            orc.step_commit(sel, sc_o[sel])      # the oracle's own scores: only the choice is the device's
+            r["dgamma"] = float(np.abs(orc.gamma() - g).max())
+            r["gamma_ok"] = r["dgamma"] <= max(GAMMA_TOL, acc)
+        r["same"] = r["ints_ok"] = same
+        rec.append(r)
+    return rec
+
+
+def show_run(title, rec):
+    print(title)
+    print("  logit error per step: " + " ".join("%.2g" % r["eps_z"] for r in rec))
+    print("  gamma error per step: " + " ".join("%.2g" % r.get("dgamma", float("nan")) for r in rec))
+    print("  gamma bound (acc. 4 eps / tau): " + " ".join("%.2g" % r["acc"] for r in rec))
+    print("  drafts equal for %d timesteps" % sum(r["same"] for r in rec))
+
+
+class OracleAsDevice:
+    """A second oracle behind the read-outs free_run takes from the device context, free-running too."""
+
+    def __init__(self, orc):
+        self.o, self.k = orc, orc.cfg.k
+
+    def spd_prefill(self, prefix):
+        return self.o.prefill(prefix)
+
+    def spd_step(self):
+        return self.o.step()
+
+    def spd_debug_read(self, what):
+        o = self.o
+        return {"LOGITS": o.logits, "CAND_TOK": o.cand_tok, "SEL": o.sel, "SCORE": o.scores, "CNT": o.counts,
+                "TOT": o.totals}[what]().copy()

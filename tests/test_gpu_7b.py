@@ -28,9 +28,33 @@ def big():
     ctx = P.SpdContext(wl.shape, packed, dtabs, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 192, wl.kv_dtype)
     cfg = so.make_config(wl.shape, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 192, wl.kv_dtype)
     orc = so.Oracle(cfg, host, tables)
+    extra = {}
+
+    def make(k=wl.k, kv_dtype=wl.kv_dtype, max_pos=192):
+        """Another context / oracle pair over the same packed weights and tables."""
+        key = (k, kv_dtype, max_pos)
+        if key not in extra:
+            c = P.SpdContext(wl.shape, packed, dtabs, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, max_pos, kv_dtype)
+            o = so.Oracle(so.make_config(wl.shape, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, max_pos, kv_dtype), host, tables)
+            extra[key] = (c, o)
+        return extra[key]
+
+    def drop(key):
+        c, o = extra.pop(key)
+        c.close()
+        o.close()
+
+    Big.make, Big.drop = staticmethod(make), staticmethod(drop)
     yield wl, ctx, orc, tables, prefix
+    for key in list(extra):
+        drop(key)
     ctx.close()
     orc.close()
+
+
+class Big:
+    """Set by the fixture: make(k, kv_dtype, max_pos) -> (context, oracle) sharing the fixture's weights and tables."""
+    make = drop = None
 
 
 def test_7b_steps_match_oracle(big):
@@ -46,6 +70,8 @@ def test_7b_steps_match_oracle(big):
     assert max(s["eps_z"] for s in errs) < 2e-3
     flips = sum(s.get("cache_flips", 0) for s in stats)
     print("7B parity: max logit error %.3g, cache values rounded the other way: %d" % (max(s["eps_z"] for s in errs), flips))
+    print("  slack units needed: " + ", ".join("%s %.1f (%d/%d)" % (s["path"], s["slack_units_needed"], s["cache_flips"], s["cache_values"])
+                                              for s in stats if "path" in s))
 
 
 def test_7b_long_prefix_on_tensor_cores(big):
@@ -64,6 +90,8 @@ def test_7b_long_prefix_on_tensor_cores(big):
     assert max(s["eps_z"] for s in errs) < 2e-3
     flips = sum(s.get("cache_flips", 0) for s in stats)
     print("7B long prefix: max logit error %.3g, cache values rounded the other way: %d" % (max(s["eps_z"] for s in errs), flips))
+    print("  slack units needed: " + ", ".join("%s %.1f (%d/%d)" % (s["path"], s["slack_units_needed"], s["cache_flips"], s["cache_values"])
+                                              for s in stats if "path" in s))
 
 
 def test_7b_one_launch_equals_single_steps(big):
@@ -142,3 +170,66 @@ def test_7b_nucleus_splice(big):
         assert new_all.tolist() == seq[len(prefix):] and ids2.tolist() == ids.tolist() and np.array_equal(g, g2)
         assert np.array_equal(ctx.spd_debug_read("LOGITS"), z_last)
     compare_first_step(ctx, orc, seq, None, device=(ids2, g2))
+
+
+def _drift_of_exact_arithmetic(wl, host_pair, prefix, first_logP, n):
+    """Two float64 oracles on the same request, one of which starts from the device's first-timestep
+    log-probabilities (a float-sized difference, nothing else): how far apart exact arithmetic alone lets the two
+    runs drift, per step."""
+    from tests.gpu_common import OracleAsDevice, free_run
+
+    a, b = host_pair
+    return free_run(OracleAsDevice(a), b, prefix, n, perturb_logP=lambda dev: dev.o.set_logP(first_logP))
+
+
+@pytest.mark.parametrize("kv_dtype", ["f32", "bf16"])
+def test_7b_free_running(big, kv_dtype):
+    """The benchmark's request (15-token prefix, 3 drafts of 10 tokens) with NO forcing of the oracle.
+
+    At tau = 0.06 the method itself amplifies differences: a logit difference e moves gamma by up to 4 e / tau = 67 e,
+    gamma weights the next input (Eq. 3), and the next logits move in proportion.  The run is therefore gated on the
+    steps where the question is still about the implementation: the first timestep always, and every later step while
+    the bound on gamma's error that the logit errors so far imply (accumulated 4 eps / tau) is below 0.05; there
+    logits must be within 2e-2, integers exact (margin rule on near-ties) and gamma within its bound.  All steps are
+    printed, beside the drift of two float64 oracles that differ only by the device's first-timestep
+    log-probabilities: where those two part, no implementation can be expected to follow, and on every step the
+    device must stay as close to the oracle as that exact pair stays to each other (twice its distance + 2e-2).
+    With the bf16 cache the first timestep already differs by about 1e-2 (one cache value in a hundred of the
+    prefill rounds the other way in float32 than in float64), so only that step is gated."""
+    from tests.gpu_common import LOGIT_TOL, free_run, show_run
+
+    wl, ctx0, orc0, tables, prefix = big
+    ctx, orc = (ctx0, orc0) if kv_dtype == wl.kv_dtype else Big.make(kv_dtype=kv_dtype)
+    n = wl.gen_tokens - 1
+    rec = free_run(ctx, orc, prefix, n)
+    show_run("7B free-running, %s cache" % kv_dtype, rec)
+    ctx.spd_prefill(prefix)
+    first_logP = ctx.spd_debug_read("LOGP").astype(np.float64)
+    other = Big.make(kv_dtype=kv_dtype, max_pos=191)[1]     # a second oracle of the same kind
+    drift = _drift_of_exact_arithmetic(wl, (other, orc), prefix, first_logP, n)
+    show_run("  two float64 oracles, one started from the device's first-timestep log-probabilities", drift)
+    gated = [r for i, r in enumerate(rec) if i == 0 or rec[i - 1]["acc"] <= 0.05]
+    assert all(r["logits_ok"] and r["ints_ok"] and r["gamma_ok"] for r in gated), gated
+    if kv_dtype == "f32":
+        assert len(gated) >= 2
+    # on every step the device is no further from the oracle than exact arithmetic drifts from the same start
+    for r, d in zip(rec, drift):
+        assert r["eps_z"] <= 2 * d["eps_z"] + LOGIT_TOL, (r["eps_z"], d["eps_z"])
+    assert sum(r["same"] for r in rec) >= sum(d["same"] for d in drift) - 1
+    Big.drop((wl.k, kv_dtype, 191))
+    if kv_dtype != wl.kv_dtype:
+        Big.drop((wl.k, kv_dtype, 192))
+
+
+@pytest.mark.parametrize("k", [2, 4, 6, 8])
+def test_7b_draft_counts(big, k):
+    """The k sweep of the benchmark's workload family at full width: first timestep and two steps per k."""
+    wl, _, _, tables, prefix = big
+    ctx, orc = Big.make(k=k)
+    stats = []
+    compare_first_step(ctx, orc, prefix, stats)
+    for _ in range(2):
+        ids, par, g = compare_step(ctx, orc, stats)
+        assert abs(float(g.sum()) - 1.0) < 1e-5 and np.all(np.diff(g) <= 0)
+    assert max(s["eps_z"] for s in stats if "eps_z" in s) < 2e-3
+    Big.drop((k, wl.kv_dtype, 192))

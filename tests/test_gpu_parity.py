@@ -14,6 +14,7 @@ pytestmark = pytest.mark.gpu
 def test_tiny_workload_stepwise(tiny_inputs, kv_dtype):
     wl, weights, tables, prefix = tiny_inputs
     ctx, orc = make_tiny_pair(tiny_inputs, kv_dtype=kv_dtype)
+    ctx.spd_debug_trace(True)
     stats = []
     compare_first_step(ctx, orc, prefix, stats)
     tr, tr_o = ctx.spd_debug_read("TRACE").astype(np.float64), orc.trace()
@@ -195,6 +196,34 @@ def test_every_stored_ngram_is_found_and_absent_ones_miss(tiny_inputs):
     ctx.close()
 
 
+def test_counts_beyond_two_to_the_31(tiny_inputs):
+    """Counts and context totals of a web-scale corpus pass 2^31: the device reads them as unsigned 32-bit numbers
+    (a 3e9 total, a 4e9 count), and the n-gram probability is their ratio as in the oracle."""
+    wl, weights, _, prefix = tiny_inputs
+    big_tables = [{"n": 2, "keys": torch.tensor([[5, 7], [5, 9], [6, 7]], dtype=torch.int32),
+                   "counts": torch.tensor([2_500_000_000, 500_000_000, 4_000_000_000], dtype=torch.int64)},
+                  {"n": 3, "keys": torch.tensor([[4, 5, 7], [4, 5, 9]], dtype=torch.int32),
+                   "counts": torch.tensor([2_147_483_648, 2_147_483_646], dtype=torch.int64)}]
+    k = 3
+    ctx, orc = make_tiny_pair(tiny_inputs, k=k, tables=big_tables + [{"n": 4, "keys": torch.zeros((0, 4), dtype=torch.int32),
+                                                                      "counts": torch.zeros(0, dtype=torch.int64)}])
+    hist = np.array([[1, 2, 3, 4, 5], [1, 2, 3, 4, 6], [1, 2, 3, 9, 5]], np.int32)
+    cand = np.array([7, 9, 11], np.int32)
+    logP = np.array([-0.1, -0.2, -0.3], np.float32)
+    cand_lp = np.array([-0.5, -0.7, -0.9], np.float32)
+    ctx.spd_debug_score(hist, logP, cand, cand_lp)
+    want = so.score_stage(orc.cfg, orc.tables, hist, logP, cand, cand_lp)
+    cnt, tot = ctx.spd_debug_read("CNT")[:, :3], ctx.spd_debug_read("TOT")[:, :3]
+    assert np.array_equal(cnt, want["cnt"]) and np.array_equal(tot, want["tot"])
+    assert tot[0, 0] == 3_000_000_000 and cnt[3, 0] == 4_000_000_000 and tot[0, 1] == 4_294_967_294
+    assert np.abs(ctx.spd_debug_read("PNG") - want["png"]).max() < 1e-6
+    sc = ctx.spd_debug_read("SCORE").astype(np.float64)
+    fin = np.isfinite(want["score"])
+    assert np.array_equal(np.isfinite(sc), fin) and np.abs(sc[fin] - want["score"][fin]).max() < 2e-5
+    assert ctx.spd_debug_read("SEL").tolist() == want["sel"].tolist()
+    ctx.close()
+
+
 def test_self_generated_corpus_gives_hits_end_to_end(tiny_inputs):
     """Tables counted over text the model itself produces (greedy continuations of random prefixes)
     make the n-gram lookups hit during real decoding, so the interpolation path runs end to end."""
@@ -346,3 +375,24 @@ def test_expired_wait_is_reported_and_the_context_stays_usable(tiny_inputs):
     b, _, _ = ref.spd_generate(4, 5)
     assert a.tolist() == b.tolist()
     ctx.close(); ref.close()
+
+
+@pytest.mark.parametrize("kv_dtype", ["f32", "bf16"])
+def test_tiny_free_running(tiny_inputs, kv_dtype):
+    """The whole tiny request (first timestep + 8 steps) with no forcing of the oracle: it never sees the device's
+    cache or log-probabilities.  Every step is gated for both cache types: logits within 2e-2, kept tokens, counts,
+    choices and parents exact (margin rule on near-ties), gamma within max(1e-4, accumulated 4 eps / tau).  Then the
+    same request as one launch of all steps gives the same drafts."""
+    from tests.gpu_common import free_run, show_run
+
+    wl, weights, tables, prefix = tiny_inputs
+    ctx, orc = make_tiny_pair(tiny_inputs, kv_dtype=kv_dtype)
+    rec = free_run(ctx, orc, prefix, wl.gen_tokens)
+    show_run("tiny free-running, %s cache" % kv_dtype, rec)
+    assert len(rec) == wl.gen_tokens + 1
+    assert all(r["logits_ok"] and r["ints_ok"] and r["gamma_ok"] for r in rec)
+    toks = orc.drafts()[:, len(prefix):]
+    ctx.spd_prefill(prefix)
+    got, lp, g = ctx.spd_generate(wl.gen_tokens, wl.gen_tokens + 1)
+    assert np.array_equal(got, toks) and np.abs(g - orc.gamma()).max() <= max(GAMMA_TOL, rec[-1]["acc"])
+    ctx.close()

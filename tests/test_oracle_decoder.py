@@ -141,6 +141,13 @@ def test_bf16_cache_holds_bf16_values(tiny_inputs):
     assert np.all(k[:, 16:] == 0)
 
 
+def _bf16_step(a, up):
+    """The bf16 value next to each (bf16-representable, non-zero) float32 value, upwards or downwards."""
+    bits = a.astype(np.float32).view(np.uint32).astype(np.int64)
+    away = (a > 0) == up
+    return (bits + np.where(away, 1 << 16, -(1 << 16))).astype(np.uint32).view(np.float32)
+
+
 def test_cache_following_adopts_only_valid_roundings(tiny_inputs):
     wl, weights, tables, prefix = tiny_inputs
     cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "bf16")
@@ -152,25 +159,75 @@ def test_cache_following_adopts_only_valid_roundings(tiny_inputs):
     b.follow_cache(k, v)
     b.prefill(prefix)
     assert b.follow_cache(None) == (0, 0) and np.array_equal(b.logits(), z0)      # its own values: nothing to adopt
-    # layer 0 keys moved one bf16 value up or down: adopted where that is the exact value's other neighbour,
-    # refused where it is two values away
+    # the exact layer-0 keys (layer 0 does not depend on the cache type): a float32 cache keeps them to 2^-24
+    cfg32 = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "f32")
+    e = so.Oracle(cfg32, weights, tables)
+    e.prefill(prefix)
+    x = e.kv_cache()[0][0, :16].astype(np.float64)
+    own = k[0].astype(np.float64)
+    assert np.all(own != 0)
+    toward = _bf16_step(k[0], x > own)        # the exact value's other neighbour
+    beyond = _bf16_step(k[0], x <= own)       # the neighbour on the far side of the cache value
+    mid_dist = np.abs(0.5 * (own + toward.astype(np.float64)) - x)   # distance of x from the rounding boundary
+    # (1) without slack no neighbour is a rounding of x (exact midpoints aside: none here)
     k2 = k.copy()
-    bits = k2[0].view(np.uint32)
-    up = np.random.default_rng(0).random(bits.shape) < 0.5
-    bits[up] += np.uint32(1 << 16)
-    bits[~up] -= np.uint32(1 << 16)
+    k2[0] = toward
     c = so.Oracle(cfg, weights, tables)
-    c.follow_cache(k2, v)
+    c.follow_cache(k2, v, slack=0.0)
     c.prefill(prefix)
-    flips, bad = c.follow_cache(None)
+    assert np.array_equal(c.kv_cache()[0][0, :16], k[0])
+    assert c.follow_cache(None)[1] >= k[0].size
+    # (2) with slack s exactly the values within s of the boundary flip: half a spacing plus s, not a whole spacing
+    s_ = float(np.median(mid_dist))
+    clear = np.abs(mid_dist - s_) > 1e-6 * np.abs(x)
+    c = so.Oracle(cfg, weights, tables)
+    c.follow_cache(k2, v, slack=s_)
+    c.prefill(prefix)
     got = c.kv_cache()[0][0, :16]
-    adopted, refused = int(np.count_nonzero(got == k2[0])), int(np.count_nonzero(got == k[0]))
-    assert adopted + refused == k2[0].size and adopted > 0.3 * k2[0].size and refused > 0.3 * k2[0].size
-    assert flips >= adopted and bad >= refused      # later layers, now fed different inputs, add to both counts
-    # values that are no rounding of the exact ones are refused and counted
+    assert np.array_equal((got == toward)[clear], (mid_dist <= s_)[clear])
+    assert np.array_equal(got[mid_dist > s_ + 1e-6 * np.abs(x)], k[0][mid_dist > s_ + 1e-6 * np.abs(x)])
+    flips, bad = c.follow_cache(None)
+    assert flips > 0.3 * k[0].size and bad > 0.3 * k[0].size and 0 < c.follow_need <= s_
+    # (3) the far-side neighbour is never a rounding of x, even with a slack of half a spacing
     k3 = k.copy()
-    k3[1, 3, :7] += 1.0
+    k3[0] = beyond
+    c = so.Oracle(cfg, weights, tables)
+    c.follow_cache(k3, v, slack=float(np.min(np.abs(toward.astype(np.float64) - own))) * 0.49)
+    c.prefill(prefix)
+    assert np.array_equal(c.kv_cache()[0][0, :16], k[0]) and c.follow_cache(None)[0] == 0
+    # (4) values that are no rounding of the exact ones are refused and counted
+    k4 = k.copy()
+    k4[1, 3, :7] += 1.0
     d = so.Oracle(cfg, weights, tables)
-    d.follow_cache(k3, v)
+    d.follow_cache(k4, v, slack=1e-6)
     d.prefill(prefix)
     assert d.follow_cache(None) == (0, 7) and np.array_equal(d.logits(), z0)
+
+
+def test_cache_following_slack_covers_values_near_zero(tiny_inputs):
+    """Near zero the spacing of bf16 is far below any float error: there the slack, not the spacing, decides.  A value
+    moved by less than the slack (many bf16 steps near zero) is adopted with the slack and refused without it."""
+    wl, weights, tables, prefix = tiny_inputs
+    cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "bf16")
+    a = so.Oracle(cfg, weights, tables)
+    a.prefill(prefix)
+    k, v = (x[:, :16].copy() for x in a.kv_cache())
+    small = np.argsort(np.abs(k[0]).ravel())[:8]           # the layer-0 keys closest to zero: |value| < 2e-3,
+    slack = 2e-4                                           # bf16 spacing there <= 8e-6, far below this slack
+    assert np.abs(k[0].ravel()[small]).max() < 2e-3
+    moved = k.copy()
+    flat = moved[0].reshape(-1)
+    t = torch.from_numpy(flat[small] + np.float32(0.5 * slack)).to(torch.bfloat16).to(torch.float32).numpy()
+    changed = t != flat[small]
+    assert changed.all()                                   # half a slack crosses many bf16 steps for these
+    flat[small] = t
+    for s_, adopted in ((slack, True), (0.0, False)):
+        c = so.Oracle(cfg, weights, tables)
+        c.follow_cache(moved, v, slack=s_)
+        c.prefill(prefix)
+        got = c.kv_cache()[0][0, :16].reshape(-1)[small]
+        flips, bad = c.follow_cache(None)
+        if adopted:
+            assert np.array_equal(got, t) and bad == 0 and flips >= changed.sum()
+        else:
+            assert np.array_equal(got[changed], k[0].reshape(-1)[small][changed]) and bad >= changed.sum()

@@ -1,11 +1,14 @@
 """spd_score_static: the scoring stage for callers that cannot allocate device memory (they hold device
 pointers to the tables but have no allocator to obtain a workspace from, so spd_create is closed to
 them).  Its scratch is a fixed array inside the library, shared by all calls, so the check runs it twice in
-a row on different inputs and compares each result with the workspace-based entry point."""
+a row on different inputs and compares each result with the workspace-based entry point and with the CPU
+oracle's scoring stage, and watches the device's free memory across the calls."""
 import numpy as np
 import pytest
+import torch
 
 import spd_inputs as si
+from oracle import spd_oracle as so
 
 pytestmark = pytest.mark.gpu
 
@@ -35,14 +38,27 @@ def test_static_scratch_entry_point_matches_workspace_entry_point(tiny_inputs):
     rng = np.random.default_rng(2024)
     ctxs = {}
     hits = 0
+    otabs = so.NgramTables(sorted(tables, key=lambda t: int(t["n"])))
     # two calls in a row (then more): a larger k first, so that the second call would see leftovers if
     # the shared array were not rewritten
     for k, hist_len in [(5, 8), (3, 8), (16, 2), (2, 5)]:
         if k not in ctxs:
             ctxs[k] = P.SpdContext(wl.shape, packed, dtabs, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64)
         hist, logp, cand, cand_lp = _case(tables, rng, k, wl.shape.vocab, hist_len)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         sel, out_lp, gamma, score = spd_score_static(k, wl.shape.vocab, wl.orders, wl.lambdas(), wl.alpha, wl.delta,
                                                      dtabs, hist, logp, cand, cand_lp)
+        assert torch.cuda.mem_get_info()[0] == free_before            # the call took no device memory
+        # against the CPU oracle's scoring stage on the same inputs (Eq. 5-7, Eq. 2, Eq. 4)
+        cfg = so.make_config(wl.shape, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "bf16")
+        want = so.score_stage(cfg, otabs, hist, logp, cand, cand_lp)
+        fin = np.isfinite(want["score"])
+        assert np.array_equal(np.isfinite(score), fin) and np.abs(score[fin] - want["score"][fin]).max() < 2e-5
+        srt = np.sort(want["score"][fin])[::-1][: k + 1]
+        if np.min(-np.diff(srt)) > 1e-4:
+            assert sel.tolist() == want["sel"].tolist()
+            assert np.abs(out_lp - want["logP"]).max() < 2e-5 and np.abs(gamma - want["gamma"]).max() < 1e-4
         ctx = ctxs[k]
         ctx.spd_debug_score(hist, logp, cand, cand_lp)
         want_score = ctx.spd_debug_read("SCORE")
@@ -70,4 +86,8 @@ def test_static_scratch_entry_point_refuses_oversized_requests(tiny_inputs):
     with pytest.raises(P.SpdError) as e:
         spd_score_static(3, wl.shape.vocab, wl.orders, wl.lambdas(), wl.alpha, wl.delta, dtabs,
                          np.zeros((3, 9), np.int32), z[:3], np.arange(3, dtype=np.int32), z[:3])
+    assert e.value.status == -3
+    with pytest.raises(P.SpdError) as e:      # more tables than the fixed scratch was laid out for
+        spd_score_static(3, wl.shape.vocab, wl.orders, wl.lambdas(), wl.alpha, wl.delta, [dtabs[0]] * 9,
+                         np.zeros((3, 8), np.int32), z[:3], np.arange(3, dtype=np.int32), z[:3])
     assert e.value.status == -3
