@@ -31,7 +31,7 @@ import spd_inputs as si
 
 # dram bytes (read + write) / algorithmic bytes measured by ncu on a 4-layer case of the same kernel; traffic
 # grows in proportion to the layers streamed.  None whenever the kernel has changed since the counters were taken.
-TRAFFIC_RATIO = 1.003
+TRAFFIC_RATIO = None
 
 METRIC = "k-draft tokens/s"
 UNIT = "tokens/s"
@@ -67,6 +67,13 @@ def step_bytes(wl, k, T):
     kvb = 2 if wl.kv_dtype == "bf16" else 4
     return (s.step_weight_bytes + 2 * (2 * s.n_layers + 1) * s.d_model + k * s.d_model * 2
             + s.n_layers * 2 * T * s.d_model * kvb + (k + k * k) * len(wl.orders) * 32)
+
+
+def config_of(wl, k, world, reps):
+    """The workload's description, the same in both arms."""
+    return {"workload": "%s: %s-shape decoder, prefix %d, k=%d, bs1, n-gram n=%d..%d, %d entries/order" % (
+        wl.name, wl.shape.name, wl.prefix_len, k, min(wl.orders), max(wl.orders), wl.retain),
+        "l2": "inputs_exceed_l2", "kv_dtype": wl.kv_dtype, "parallelism": "replicas x%d" % world, "reps": reps}
 
 
 def max_over_ranks(x: float, dev, world: int) -> float:
@@ -256,13 +263,14 @@ def run_ours(args, wl):
         n_tc = wl.prefix_len - ((wl.prefix_len - 1) % 16 + 1)
         sh = wl.shape
         layer_params = sh.n_layers * (4 * sh.d_model * sh.d_model + 3 * sh.d_model * sh.d_ffn)
-        tflop = n_tc * layer_params * 2 * 3 / 1e12
+        tflop = n_tc * layer_params * 2 / 1e12           # the method's own arithmetic: tokens x weights x 2
         tpeak, tkind = measured_peak_bf16()
         prefill_rec = {"ms": pf_ms, "tokens": wl.prefix_len, "tokens_through_tcgen05_products": n_tc, "bound": "tensor",
                        "achieved": tflop / (pf_ms * 1e-3), "peak": tpeak, "unit": "TFLOP/s", "frac": tflop / (pf_ms * 1e-3) / tpeak,
-                       "peak_kind": tkind,
+                       "peak_kind": tkind, "issued_tflops": 3 * tflop / (pf_ms * 1e-3), "issued_frac": 3 * tflop / (pf_ms * 1e-3) / tpeak,
                        "note": "whole spd_prefill call (products, attention, row-wise kernels, the last tokens' launch of the 16-token "
-                               "kernel with LM head and first timestep); arithmetic = tokens x layer weights x 2 x 3 bf16 terms per float32 activation"}
+                               "kernel with LM head and first timestep); achieved / frac count the method's arithmetic (tokens x layer "
+                               "weights x 2); issued_* count what the tensor cores execute, three bf16 terms per float32 activation"}
 
     # ---- the same number of drafts from k separate single-draft passes through the same kernels
     kpass = None
@@ -301,9 +309,7 @@ def run_ours(args, wl):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": "%s: %s-shape decoder, prefix %d, k=%d, bs1, n-gram n=%s, %d entries/order" % (
-            wl.name, wl.shape.name, wl.prefix_len, k, "%d..%d" % (min(wl.orders), max(wl.orders)), wl.retain),
-            "l2": "inputs_exceed_l2", "kv_dtype": wl.kv_dtype, "parallelism": "replicas x%d" % world, "reps": reps},
+        "config": config_of(wl, k, world, reps),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": TRAFFIC_RATIO * bytes_step * K if TRAFFIC_RATIO else None, "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_decode_kernel"},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
@@ -372,8 +378,7 @@ def run_reference(args, wl):
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": K_run, "warmup": W,
            "ms_per_step": dt / K_run * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
            "data": "synthetic",
-           "config": {"workload": "%s: %s-shape decoder, prefix %d, k=%d, bs1, n-gram n=%d..%d, %d entries/order" % (
-               wl.name, wl.shape.name, wl.prefix_len, k, min(wl.orders), max(wl.orders), wl.retain)},
+           "config": config_of(wl, k, 1, args.reps),
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out), flush=True)

@@ -52,7 +52,9 @@ typedef struct spd_ctx spd_ctx; /* opaque; small host object owned by the librar
  * Method: k drafts (1..SPD_MAX_K); n-gram orders n_min..n_max (2..SPD_MAX_N) with interpolation
  * weights lambda[n-2] (Eq. 5, Appendix B); alpha of Eq. 6; tau = softmax temperature applied to
  * the logits before anything else; delta of Eq. 7 (0 < delta <= 1; the paper gives no value).
- * eos_id must be -1 (stopping on a token is not implemented).  kv_dtype: 0 = float32 cache, 1 = bf16
+ * eos_id: the stop token, -1 for none (Section 3 and Algorithm 1 generate "until max generation length or stop
+ * token"; which draft's token counts is not said: here decoding ends with the timestep in which the most
+ * probable draft emits it, see spd_finished).  kv_dtype: 0 = float32 cache, 1 = bf16
  * cache (keys after the rotary embedding and values are rounded to nearest even when stored).
  * stream: a cudaStream_t (NULL = the legacy default stream).
  */
@@ -137,7 +139,9 @@ int spd_step(spd_ctx *ctx, int32_t *out_ids, int32_t *out_parent, float *out_gam
  * HOST outputs, any may be NULL: out_tokens [k][*out_len] row-major = all tokens generated so far
  * by each surviving draft (the first-timestep token included, the prefix excluded); out_len = that
  * length; out_logp [k] = log of the draft probabilities P of Eq. 2; out_gamma [k].
- * out_tokens must have room for k * (tokens generated so far + n_steps) entries.
+ * out_tokens must have room for k * (tokens generated so far + n_steps) entries.  With a stop token the launch
+ * ends after the timestep in which the most probable draft emits it: *out_len is then smaller than asked for
+ * (rows of out_tokens are *out_len apart), and spd_finished turns 1.
  */
 int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *out_len, float *out_logp,
                  float *out_gamma);
@@ -287,6 +291,13 @@ int spd_debug_expire(spd_ctx *ctx);
  * size other than 64 or 128).  The context stays usable: prefill it again.
  */
 int spd_debug_expire_products(spd_ctx *ctx);
+
+/*
+ * 1 once the most probable draft has ended with the stop token (cfg.eos_id; always 0 without one), as seen by the
+ * last synchronising call.  spd_step / spd_generate / spd_generate_async then return SPD_ESTATE until the context is
+ * prefilled or reset again.  The drafts stay readable; the paper does not say what happens to the other drafts.
+ */
+int spd_finished(const spd_ctx *ctx);
 
 /* Number of kernel launches this context has enqueued so far. */
 int64_t spd_launch_count(const spd_ctx *ctx);

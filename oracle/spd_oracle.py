@@ -186,6 +186,16 @@ class Oracle:
             raise ValueError("orc_step: out of positions")
         return ids, par, g
 
+    def generate(self, max_steps: int, eos_id: int = -1) -> int:
+        """Algorithm 1's loop, "until max generation length or stop token": steps until max_steps are taken or the
+        most probable draft (drafts are ordered by probability) has just emitted eos_id.  The paper does not say
+        which draft's token counts; the most probable one is this implementation's reading.  Returns the steps taken."""
+        for n in range(max_steps):
+            ids, _, _ = self.step()
+            if eos_id >= 0 and int(ids[0]) == eos_id:
+                return n + 1
+        return max_steps
+
     def step_forward(self) -> None:
         if lib().orc_step_forward(self.h):
             raise ValueError("orc_step_forward: out of positions")

@@ -66,7 +66,7 @@ _lib: Optional[C.CDLL] = None
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
            "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
-           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace"]
+           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished"]
 
 
 def load_library() -> C.CDLL:
@@ -106,6 +106,7 @@ def load_library() -> C.CDLL:
     L.spd_debug_nucleus.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_void_p]
     L.spd_debug_expire.argtypes = [C.c_void_p]
     L.spd_debug_trace.argtypes = [C.c_void_p, C.c_int]
+    L.spd_finished.argtypes = [C.c_void_p]
     L.spd_debug_expire_products.argtypes = [C.c_void_p]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
@@ -177,7 +178,7 @@ class SpdContext:
     def __init__(self, shape, packed: Dict[str, object], tables: Sequence[Dict[str, object]], k: int,
                  orders: Sequence[int], lam: Sequence[float], alpha: float, tau: float, delta: float, max_pos: int,
                  kv_dtype: str = "bf16", rms_eps: float = 1e-5, rope_theta: float = 10000.0,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, eos_id: int = -1):
         L = load_library()
         self.lib = L
         self.k = k
@@ -192,7 +193,7 @@ class SpdContext:
         cfg.n_min, cfg.n_max = (min(orders), max(orders)) if len(orders) else (2, 2)
         for i in range(MAX_ORDERS):
             cfg.lam[i] = float(lam[i]) if i < len(lam) else 0.0
-        cfg.alpha, cfg.tau, cfg.delta, cfg.eos_id = alpha, tau, delta, -1
+        cfg.alpha, cfg.tau, cfg.delta, cfg.eos_id = alpha, tau, delta, eos_id
         cfg.kv_dtype = {"f32": 0, "bf16": 1}[kv_dtype]
         self.stream = stream
         cfg.stream = stream.cuda_stream if stream is not None else None
@@ -278,15 +279,19 @@ class SpdContext:
         return ids, par, g
 
     def spd_generate(self, n_steps: int, total_len: int):
-        """total_len = tokens per draft after the call (tokens so far + n_steps)."""
-        toks = np.zeros((self.k, total_len), np.int32)
+        """total_len = tokens per draft after the call (tokens so far + n_steps); fewer come back when the stop
+        token ended the run early."""
+        toks = np.zeros(self.k * total_len, np.int32)
         ln = C.c_int32()
         lp = np.zeros(self.k, np.float32)
         g = np.zeros(self.k, np.float32)
         _check(self.lib.spd_generate(self.h, n_steps, toks.ctypes.data, C.byref(ln), lp.ctypes.data, g.ctypes.data),
                "spd_generate")
-        assert ln.value == total_len, (ln.value, total_len)
-        return toks, lp, g
+        assert ln.value == total_len or (self.cfg.eos_id >= 0 and ln.value < total_len), (ln.value, total_len)
+        return toks[: self.k * ln.value].reshape(self.k, ln.value).copy(), lp, g
+
+    def spd_finished(self) -> bool:
+        return bool(self.lib.spd_finished(self.h))
 
     def spd_generate_async(self, n_steps: int) -> None:
         _check(self.lib.spd_generate_async(self.h, n_steps), "spd_generate_async")

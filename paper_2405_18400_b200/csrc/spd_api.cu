@@ -63,7 +63,7 @@ bool valid_config(const spd_config *c) {
   if (c->n_min < 2 || c->n_max > SPD_MAX_N) return false;
   if (!(c->tau > 0.f) || !(c->delta > 0.f) || c->delta > 1.f || !(c->alpha >= 0.f) || c->alpha > 1.f) return false;
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
-  if (c->eos_id != -1) return false;
+  if (c->eos_id < -1 || c->eos_id >= c->vocab) return false;
   if (c->kv_dtype != 0 && c->kv_dtype != 1) return false;
   return true;
 }
@@ -170,6 +170,8 @@ struct spd_ctx {
   std::vector<spd::LayerW> layers_host;  // the layer table, for the long-prefix path's launches
   int tc_rows;     // tokens one long-prefix job takes (0: path unused)
   int32_t n_gen;   // tokens generated per draft
+  bool stopped;    // the most probable draft ended with the stop token: no further steps until the next prefill
+  bool decoding;   // the last launch was a run of decode steps (the device's token count is the one to take over)
   int64_t launches;
 };
 
@@ -189,12 +191,19 @@ int pick_ring(const spd_config &c, int32_t stage_bytes, int32_t n_stages, int32_
   return SPD_OK;
 }
 
+// Waits for the stream and returns what the device recorded; with a stop token configured, also takes over the
+// device's count of generated tokens and its stop flag (a launch may have ended before its last step).
 int check_device_error(spd_ctx *ctx) {
-  int32_t err[2] = {0, 0};
-  SPD_CUDA(cudaMemcpyAsync(err, ctx->ws + ctx->lay.state + offsetof(spd::State, err), sizeof err, cudaMemcpyDeviceToHost,
+  int32_t head[6] = {0, 0, 0, 0, 0, 0};  // stop, abort flag, err, err_info, win_len, n_gen
+  static_assert(offsetof(spd::State, n_gen) - offsetof(spd::State, stop) == 5 * sizeof(int32_t), "the fields read here are adjacent");
+  SPD_CUDA(cudaMemcpyAsync(head, ctx->ws + ctx->lay.state + offsetof(spd::State, stop), sizeof head, cudaMemcpyDeviceToHost,
                            ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));
-  return err[0];
+  if (head[2] == 0 && ctx->cfg.eos_id >= 0 && ctx->decoding) {
+    ctx->n_gen = head[5];
+    if (head[0]) ctx->stopped = true;
+  }
+  return head[2];
 }
 
 // Bytes of the state's head that every launch zeroes: with `keep_err` (later launches of a multi-launch call)
@@ -351,6 +360,8 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   ctx->ws = static_cast<uint8_t *>(workspace);
   ctx->stream = static_cast<cudaStream_t>(cfg->stream);
   ctx->prefilled = false;
+  ctx->decoding = false;
+  ctx->stopped = ctx->decoding = false;
   ctx->m = ctx->n_gen = 0;
   ctx->launches = 0;
   auto fail = [&](int rc) {
@@ -422,6 +433,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   kp.pf_ss = reinterpret_cast<float *>(ws + lay.pf_ss);
   kp.pf_part = reinterpret_cast<float *>(ws + lay.pf_part); kp.pf_ml = reinterpret_cast<float2 *>(ws + lay.pf_ml);
   kp.pf_cnt = reinterpret_cast<unsigned int *>(ws + lay.pf_cnt);
+  kp.eos_id = cfg->eos_id;
 
   // rotary table: cos / sin of pos * theta^(-2i/hd), evaluated in double and rounded once
   std::vector<float2> rope((size_t)cfg->max_pos * (hd / 2));
@@ -516,6 +528,7 @@ int spd_prefill(spd_ctx *ctx, const int32_t *prefix_ids, int32_t m, int32_t *out
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix, prefix_ids, (size_t)m * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));  // st and the caller's ids may go out of scope
   ctx->prefilled = false;
+  ctx->decoding = false;
   if ((rc = prefill_tokens(ctx, 0, m))) return rc;
   int32_t ids[SPD_MAX_K];
   float gamma[SPD_MAX_K];
@@ -525,6 +538,7 @@ int spd_prefill(spd_ctx *ctx, const int32_t *prefix_ids, int32_t m, int32_t *out
   ctx->prefilled = true;
   ctx->m = m;
   ctx->n_gen = 1;
+  ctx->stopped = c.eos_id >= 0 && ids[0] == c.eos_id;
   ctx->prefix.assign(prefix_ids, prefix_ids + m);
   for (int i = 0; i < c.k; ++i) {
     if (out_ids) out_ids[i] = ids[i];
@@ -564,6 +578,7 @@ int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma) {
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.prefix + (size_t)m * 4, seq.data(), (size_t)n * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));
   ctx->prefilled = false;
+  ctx->decoding = false;
   if ((rc = prefill_tokens(ctx, m, n))) return rc;
   int32_t ids[SPD_MAX_K];
   float gamma[SPD_MAX_K];
@@ -573,6 +588,7 @@ int spd_reset(spd_ctx *ctx, int32_t draft, int32_t *out_ids, float *out_gamma) {
   ctx->prefilled = true;
   ctx->m = m2;
   ctx->n_gen = 1;
+  ctx->stopped = c.eos_id >= 0 && ids[0] == c.eos_id;
   for (int i = 0; i < k; ++i) {
     if (out_ids) out_ids[i] = ids[i];
     if (out_gamma) out_gamma[i] = gamma[i];
@@ -595,6 +611,7 @@ int spd_sample(spd_ctx *ctx, int32_t n_new, float top_p, float temperature, cons
   SPD_CUDA(cudaMemcpyAsync(ctx->ws + ctx->lay.ns_u, uniforms, (size_t)n_new * 4, cudaMemcpyHostToDevice, ctx->stream));
   SPD_CUDA(cudaStreamSynchronize(ctx->stream));  // the caller's array may go out of scope
   ctx->prefilled = false;
+  ctx->decoding = false;
   // pass i draws token m + i from the logits of the pass before (the first from those the prefill left),
   // feeds it at position m + i; the last pass ends with the first-timestep decision
   spd::KParams &kp = ctx->kp;
@@ -617,6 +634,7 @@ int spd_sample(spd_ctx *ctx, int32_t n_new, float top_p, float temperature, cons
   ctx->prefilled = true;
   ctx->m = m + n_new;
   ctx->n_gen = 1;
+  ctx->stopped = c.eos_id >= 0 && ids[0] == c.eos_id;
   for (int i = 0; i < n_new; ++i)
     if (out_new) out_new[i] = fresh[i];
   for (int i = 0; i < c.k; ++i) {
@@ -628,14 +646,15 @@ int spd_sample(spd_ctx *ctx, int32_t n_new, float top_p, float temperature, cons
 
 int spd_generate_async(spd_ctx *ctx, int32_t n_steps) {
   if (!ctx) return SPD_EINVAL;
-  if (!ctx->prefilled) return SPD_ESTATE;
+  if (!ctx->prefilled || ctx->stopped) return SPD_ESTATE;
   if (n_steps < 1) return SPD_ERANGE;
   const int pos0 = ctx->m + ctx->n_gen - 1;  // position of the first superposed input of this launch
   if (pos0 + n_steps > ctx->cfg.max_pos || ctx->n_gen + n_steps > ctx->cfg.max_pos) return SPD_ERANGE;
   int rc = set_device(ctx);
   if (rc) return rc;
   if ((rc = launch(ctx, spd::kModeDecode, n_steps, pos0, ctx->n_gen))) return rc;
-  ctx->n_gen += n_steps;
+  ctx->n_gen += n_steps;  // with a stop token: until spd_sync reads the device's count
+  ctx->decoding = true;
   return SPD_OK;
 }
 
@@ -654,7 +673,7 @@ int spd_step(spd_ctx *ctx, int32_t *out_ids, int32_t *out_parent, float *out_gam
   const int k = ctx->cfg.k;
   int32_t ids[SPD_MAX_K], par[SPD_MAX_K];
   float gamma[SPD_MAX_K];
-  const size_t row = (size_t)(ctx->n_gen - 1) * k * 4;
+  const size_t row = (size_t)(ctx->n_gen - 1) * k * 4;  // a launch always completes its first step
   SPD_CUDA(cudaMemcpyAsync(ids, ctx->ws + ctx->lay.hist_tok + row, (size_t)k * 4, cudaMemcpyDeviceToHost, ctx->stream));
   SPD_CUDA(cudaMemcpyAsync(par, ctx->ws + ctx->lay.hist_par + row, (size_t)k * 4, cudaMemcpyDeviceToHost, ctx->stream));
   if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
@@ -670,6 +689,7 @@ int spd_step(spd_ctx *ctx, int32_t *out_ids, int32_t *out_parent, float *out_gam
 int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *out_len, float *out_logp, float *out_gamma) {
   int rc = spd_generate_async(ctx, n_steps);
   if (rc) return rc;
+  if ((rc = spd_sync(ctx))) return rc;  // with a stop token the run may have ended early: n_gen is the device's from here on
   const int k = ctx->cfg.k, len = ctx->n_gen;
   std::vector<int32_t> tok((size_t)len * k), par((size_t)len * k);
   float logp[SPD_MAX_K], gamma[SPD_MAX_K];
@@ -677,7 +697,7 @@ int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *ou
   SPD_CUDA(cudaMemcpyAsync(par.data(), ctx->ws + ctx->lay.hist_par, par.size() * 4, cudaMemcpyDeviceToHost, ctx->stream));
   if ((rc = read_state(ctx, offsetof(spd::State, logP), logp, sizeof logp))) return rc;
   if ((rc = read_state(ctx, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
-  if ((rc = spd_sync(ctx))) return rc;
+  SPD_CUDA(cudaStreamSynchronize(ctx->stream));
   if (out_tokens) {
     // follow each surviving draft's parent links back to the first timestep
     for (int r = 0; r < k; ++r) {
@@ -697,6 +717,8 @@ int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *ou
 }
 
 int64_t spd_launch_count(const spd_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int spd_finished(const spd_ctx *ctx) { return ctx && ctx->stopped ? 1 : 0; }
 
 int spd_debug_read(spd_ctx *ctx, int what, void *host_buf, size_t bytes) {
   if (!ctx || !host_buf) return SPD_EINVAL;
@@ -808,6 +830,7 @@ int spd_debug_expire(spd_ctx *ctx) {
   int rc = set_device(ctx);
   if (rc) return rc;
   ctx->prefilled = false;
+  ctx->decoding = false;
   SPD_CUDA(cudaMemsetAsync(ctx->ws + ctx->lay.prefix, 0, 4, ctx->stream));  // token 0 at position 0
   ctx->kp.pf_stall = 1;
   spd::KParams &kp = ctx->kp;
@@ -830,6 +853,7 @@ int spd_debug_expire_products(spd_ctx *ctx) {
   int rc = set_device(ctx);
   if (rc) return rc;
   ctx->prefilled = false;
+  ctx->decoding = false;
   const spd::TcJob job = tc_job(ctx);
   cudaError_t e = cudaMemsetAsync(ctx->ws + ctx->lay.state, 0, head_bytes(false), ctx->stream);
   if (e == cudaSuccess) e = spd_internal_tc_stall(&job, ctx->stream);

@@ -59,7 +59,7 @@ __device__ __forceinline__ void ns_mass(float z, float inv_t, float m, unsigned 
 // s.prefix, the mass above it in s.above, and mass and count of the logits equal to it in s.tie_*.  With
 // `fraction` > 0 the target is first set to ceil(fraction * total mass).  If rounding left the target above
 // the total, the last token is located.
-__device__ void ns_search(NsShared &s, const float *logits, int V, float inv_t, float m, float fraction) {
+static __device__ void ns_search(NsShared &s, const float *logits, int V, float inv_t, float m, float fraction) {
   const int tid = threadIdx.x, warp = tid >> 5;
   int decided = 0;
   for (int pass = 0; pass < 6; ++pass) {
@@ -159,7 +159,7 @@ __device__ void ns_search(NsShared &s, const float *logits, int V, float inv_t, 
 
 // Draws one token from the nucleus of softmax(logits / T) with the uniform number u in [0, 1).  Every
 // consumer thread of the block calls it; all get the token.
-__device__ __noinline__ int ns_sample(const float *logits, int V, float inv_t, float top_p, float u, uint8_t *scratch) {
+static __device__ __noinline__ int ns_sample(const float *logits, int V, float inv_t, float top_p, float u, uint8_t *scratch) {
   NsShared &s = *reinterpret_cast<NsShared *>(scratch);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   named_sync(1, kConsumerThreads);

@@ -36,7 +36,7 @@ struct TableDev {
 // Draft state and the last step's intermediates, in device memory.
 struct State {
   unsigned int bar;         // grid barrier counter (zeroed by the host before every launch)
-  unsigned int reserved0;
+  unsigned int stop;        // set once the most probable draft's new token is the stop token (zeroed with `bar`)
   unsigned int abort_flag;  // set by any thread that gave up a wait
   int32_t err, err_info;
   int32_t win_len;          // valid tokens in each history window
@@ -99,6 +99,7 @@ struct KParams {
   // prefill kernel only (kept behind the fields the decode kernel reads: its code is sensitive to their offsets)
   float *pf_ss;              // [grid][kPfTokens] per block: sums of squares of the residual values it produced
   int32_t pf_stall;          // prefill kernel, test hook: block 0 withholds its arrival at the grid barriers
+  int32_t eos_id;            // stop token (-1: none): decoding ends with the step in which the most probable draft emits it
 };
 
 }  // namespace spd

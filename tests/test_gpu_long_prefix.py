@@ -146,3 +146,70 @@ def test_both_prefill_paths_agree(tiny_inputs):
     tb, _, _ = b.spd_generate(5, 6)
     assert ta.tolist() == tb.tolist()
     a.close(); b.close()
+
+
+def test_long_context_decode_7b_width():
+    """The long-prefix workload's regime at the 7B shape's width (d_model 4096, 32 heads of 128, d_ffn 11008; two
+    layers keep the CPU oracle's dense pass over 2048 tokens to half a minute): a 2048-token prefix through four
+    jobs of the long-prefix path and one launch of the 16-token kernel, then decode steps over more than 2048
+    cached positions, where every head's positions are split over four blocks (bf16 cache, 16-byte loads, eight
+    positions in flight per warp) and the partial results merged."""
+    import torch
+    import paper_2405_18400_b200 as P
+    from oracle import spd_oracle as so
+
+    shape = si.ModelShape("w7b", 2, 4096, 32, 11008, 2000)
+    dev = torch.device("cuda:0")
+    weights = si.make_weights(shape, seed=31, device=dev)
+    host = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in weights.items()}
+    tables = si.make_ngram_tables(shape.vocab, 1.1, 50_000, (2, 3), 5000, seed=32)
+    lam = [0.3, 0.2] + [0.0] * 6
+    packed = P.pack_weights(weights, dev, consume=True)
+    del weights
+    dtabs = P.build_ngram_tables(tables, dev)
+    ctx = P.SpdContext(shape, packed, dtabs, 3, (2, 3), lam, 0.4, 0.2, 0.05, 2304, "bf16")
+    cfg = so.make_config(shape, 3, (2, 3), lam, 0.4, 0.2, 0.05, 2304, "bf16")
+    orc = so.Oracle(cfg, host, sorted(tables, key=lambda t: int(t["n"])))
+    m = 2048
+    prefix = si.make_prefix("zipf", m, shape.vocab, 1.1, seed=33)
+    stats = []
+    compare_first_step(ctx, orc, prefix, stats)
+    assert ctx.spd_launch_count() == _expected_launches(m, 2, 512)
+    for _ in range(3):
+        ids, par, g = compare_step(ctx, orc, stats)
+        assert abs(float(g.sum()) - 1.0) < 1e-5
+    assert max(s["eps_z"] for s in stats if "eps_z" in s) < 2e-3
+    print("7B width, 2048-token prefix: max logit error %.3g; cache values rounded the other way: %s" % (
+        max(s["eps_z"] for s in stats if "eps_z" in s), [(s["path"], s["cache_flips"]) for s in stats if "path" in s]))
+    ctx.close()
+    orc.close()
+
+
+def test_prefix_of_64_tokens_13b_width():
+    """A 64-token prefix at the 13B shape's width: four launches of the 16-token kernel (the longest prefix that
+    does not take the long-prefix path), five drafts, then decode steps."""
+    import torch
+    import paper_2405_18400_b200 as P
+    from oracle import spd_oracle as so
+
+    shape = si.ModelShape("w13b", 2, 5120, 40, 13824, 2000)
+    dev = torch.device("cuda:0")
+    weights = si.make_weights(shape, seed=41, device=dev)
+    host = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in weights.items()}
+    tables = si.make_ngram_tables(shape.vocab, 1.05, 50_000, (2, 3), 5000, seed=42)
+    lam = [0.3, 0.2] + [0.0] * 6
+    packed = P.pack_weights(weights, dev, consume=True)
+    del weights
+    dtabs = P.build_ngram_tables(tables, dev)
+    ctx = P.SpdContext(shape, packed, dtabs, 5, (2, 3), lam, 0.4, 0.2, 0.05, 256, "bf16")
+    cfg = so.make_config(shape, 5, (2, 3), lam, 0.4, 0.2, 0.05, 256, "bf16")
+    orc = so.Oracle(cfg, host, sorted(tables, key=lambda t: int(t["n"])))
+    prefix = si.make_prefix("zipf", 64, shape.vocab, 1.05, seed=43)
+    stats = []
+    compare_first_step(ctx, orc, prefix, stats)
+    assert ctx.spd_launch_count() == 4
+    for _ in range(3):
+        compare_step(ctx, orc, stats)
+    assert max(s["eps_z"] for s in stats if "eps_z" in s) < 2e-3
+    ctx.close()
+    orc.close()

@@ -396,3 +396,54 @@ def test_tiny_free_running(tiny_inputs, kv_dtype):
     got, lp, g = ctx.spd_generate(wl.gen_tokens, wl.gen_tokens + 1)
     assert np.array_equal(got, toks) and np.abs(g - orc.gamma()).max() <= max(GAMMA_TOL, rec[-1]["acc"])
     ctx.close()
+
+
+def test_stop_token_ends_the_run(tiny_inputs):
+    """Algorithm 1 generates "until max generation length or stop token".  With the stop token set to the token the
+    oracle's most probable draft emits at its fourth step, one launch asked for eight steps ends after that step on
+    the device as in the oracle's loop: same length, same drafts, the context reports itself finished and refuses
+    further steps until it is prefilled again; step-by-step calls stop at the same place."""
+    import paper_2405_18400_b200 as P
+
+    wl, weights, tables, prefix = tiny_inputs
+    _, orc = make_tiny_pair(tiny_inputs, kv_dtype="f32")
+    orc.prefill(prefix)
+    tops = []
+    for _ in range(6):
+        ids, _, _ = orc.step()
+        tops.append(int(ids[0]))
+    eos = tops[3]
+    want_steps = tops.index(eos) + 1
+    orc.prefill(prefix)
+    assert orc.generate(8, eos) == want_steps
+    want = orc.drafts()[:, len(prefix):]
+    packed = P.pack_weights(weights, "cuda:0")
+    dtabs = P.build_ngram_tables(tables, "cuda:0")
+    ctx = P.SpdContext(wl.shape, packed, dtabs, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, wl.max_pos, "f32",
+                       eos_id=eos)
+    ctx.spd_prefill(prefix)
+    assert not ctx.spd_finished()
+    toks, lp, g = ctx.spd_generate(8, 9)
+    assert toks.shape == (wl.k, 1 + want_steps) and np.array_equal(toks, want)
+    assert ctx.spd_finished() and abs(float(g.sum()) - 1) < 1e-5
+    assert np.abs(g - orc.gamma()).max() < 1e-3
+    with pytest.raises(P.SpdError) as e:
+        ctx.spd_step()
+    assert e.value.status == -2
+    # the same by single steps; a fresh prefill clears the flag
+    ctx.spd_prefill(prefix)
+    assert not ctx.spd_finished()
+    n = 0
+    while not ctx.spd_finished():
+        ids, par, g2 = ctx.spd_step()
+        n += 1
+        assert n <= 8
+    assert n == want_steps and int(ids[0]) == eos and np.array_equal(g, g2)
+    # a stop token that never comes changes nothing
+    never = next(t for t in range(wl.shape.vocab) if t not in want and t not in tops)
+    ctx2 = P.SpdContext(wl.shape, packed, dtabs, wl.k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, wl.max_pos, "f32",
+                        eos_id=never)
+    ctx2.spd_prefill(prefix)
+    toks2, _, _ = ctx2.spd_generate(want_steps, 1 + want_steps)
+    assert np.array_equal(toks2, want) and not ctx2.spd_finished()
+    ctx.close(); ctx2.close()

@@ -46,7 +46,7 @@ def test_workspace_bytes_and_config_checks(lib):
     assert lib.spd_workspace_bytes(C.byref(_cfg(kv_dtype=0)), C.byref(n32)) == 0 and n32.value - n.value == kv
     bad = [dict(k=0), dict(k=17), dict(vocab=70000), dict(d_model=250), dict(n_heads=3), dict(n_heads=16),
            dict(n_min=1), dict(n_max=7), dict(tau=0.0), dict(delta=0.0), dict(delta=1.5), dict(alpha=1.5),
-           dict(eos_id=2), dict(kv_dtype=2), dict(max_pos=1), dict(d_ffn=20000)]
+           dict(eos_id=-2), dict(eos_id=4096), dict(kv_dtype=2), dict(max_pos=1), dict(d_ffn=20000)]
     for kw in bad:
         assert lib.spd_workspace_bytes(C.byref(_cfg(**kw)), C.byref(n)) == -1, kw
     assert lib.spd_workspace_bytes(None, C.byref(n)) == -1

@@ -283,3 +283,30 @@ def test_equal_last_tokens_make_the_step_an_ordinary_decode_step(tiny_inputs):
         b.step()
     b.feed_token(int(ids[0]))
     assert np.abs(a.logits() - b.logits()).max() < 1e-9
+
+
+def test_generation_stops_after_the_stop_token(tiny_inputs):
+    """Algorithm 1's loop condition: with a stop token the run ends with the step in which the most probable draft
+    emits it and is otherwise unchanged; without one, or with one that never comes, all steps are taken."""
+    wl, weights, tables, prefix = tiny_inputs
+    cfg = so.make_config(wl.shape, 3, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, 64, "f32")
+    a = so.Oracle(cfg, weights, tables)
+    a.prefill(prefix)
+    assert a.generate(6) == 6
+    full = a.drafts()[:, len(prefix):].copy()
+    tops = []                       # the most probable draft's newest token after each step
+    b = so.Oracle(cfg, weights, tables)
+    b.prefill(prefix)
+    for _ in range(6):
+        ids, _, _ = b.step()
+        tops.append(int(ids[0]))
+    eos = tops[3]
+    first = tops.index(eos)         # it may also have come earlier
+    c = so.Oracle(cfg, weights, tables)
+    c.prefill(prefix)
+    assert c.generate(6, eos) == first + 1
+    assert c.drafts().shape[1] == len(prefix) + 1 + first + 1
+    never = next(t for t in range(wl.shape.vocab) if t not in full)
+    d = so.Oracle(cfg, weights, tables)
+    d.prefill(prefix)
+    assert d.generate(6, never) == 6 and np.array_equal(d.drafts()[:, len(prefix):], full)
