@@ -151,6 +151,81 @@ def make_inputs(wl, device, rank):
     return weights, tables, prefix
 
 
+def run_batched(args, wl, P, dev, rank, world, packed, dtabs, k, K, W):
+    """B requests stepped together: one pass over the weights per timestep (the paper's remark that batching is
+    complementary).  Every request has its own prefix, cache and draft state."""
+    B = args.batch
+    max_pos = max(192, wl.prefix_len + W + K + 2)
+    ctxs, prefixes = [], []
+    for r in range(B):
+        ctxs.append(P.SpdContext(wl.shape, packed, dtabs, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, max_pos, wl.kv_dtype))
+        prefixes.append(si.make_prefix(wl.prefix_kind, wl.prefix_len, wl.shape.vocab, wl.zipf_s, seed=2, tensor_id=rank * 1000 + r))
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = dev.index
+    sampler = ClockSampler(gpu_id)
+    ms_list, launches = [], 0
+    sampler.start()
+    time.sleep(0.3)
+    for rep in range(max(1, args.reps)):
+        for c, pf in zip(ctxs, prefixes):
+            c.spd_prefill(pf)
+        P.spd_batch_generate(ctxs, W)
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+        l0 = ctxs[0].spd_launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        P.spd_batch_generate(ctxs, K)
+        e1.record()
+        torch.cuda.synchronize()
+        launches = ctxs[0].spd_launch_count() - l0
+        ms_list.append(e0.elapsed_time(e1))
+    time.sleep(0.2)
+    clocks = sampler.stop()
+    ms = max_over_ranks(float(np.median(ms_list)), dev, world)
+    s = wl.shape
+    T_mid = wl.prefix_len + W + (K + 1) // 2
+    kvb = 2 if wl.kv_dtype == "bf16" else 4
+    per_request = k * s.d_model * 2 + s.n_layers * 2 * T_mid * s.d_model * kvb + (k + k * k) * len(wl.orders) * 32
+    bytes_step = s.step_weight_bytes + 2 * (2 * s.n_layers + 1) * s.d_model + B * per_request
+    peak, peak_kind = measured_peak_gbs()
+    achieved = bytes_step * K / (ms * 1e-3) / 1e9
+    # end to end: host ids in, ids / parents / gamma of every request out, per timestep
+    e2e = None
+    if not args.no_e2e:
+        gen = wl.gen_tokens
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for c, pf in zip(ctxs, prefixes):
+            c.spd_prefill(pf)
+        for _ in range(gen - 1):
+            P.spd_batch_step(ctxs)
+        dt = max_over_ranks(time.perf_counter() - t0, dev, world)
+        e2e = {"value": world * B * k * gen / dt, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len * B / gen,
+               "d2h_bytes_per_step": 12.0 * k * B, "ms_per_request_batch": dt * 1e3,
+               "what": "%d x spd_prefill(host ids), then %d spd_batch_step calls returning every request's ids, parents and gamma "
+                       "to the host" % (B, gen - 1)}
+    cfg = config_of(wl, k, world, max(1, args.reps))
+    cfg["workload"] = cfg["workload"].replace("bs1", "bs%d (batched timesteps, one pass over the weights per step)" % B)
+    out = {"metric": METRIC, "value": job_throughput(world, k * B, K, ms), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+           "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": cfg,
+           "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                        "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_tc_gemm_kernel",
+                        "note": "weights once per timestep + per request its KV cache, embedding rows and table probes; the products' "
+                                "share of the step is in the launch list under profiles/"},
+           "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "batch": B}
+    for c in ctxs:
+        c.close()
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+
+
 def run_ours(args, wl):
     import paper_2405_18400_b200 as P
 
@@ -176,6 +251,12 @@ def run_ours(args, wl):
     dtabs = P.build_ngram_tables(tables, dev)
     torch.cuda.empty_cache()
     log("[bench] pack + table build %.1fs" % (time.time() - t0))
+    if args.batch > 1:
+        run_batched(args, wl, P, dev, rank, world, packed, dtabs, k, K, W)
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
     max_pos = max(wl.max_pos, wl.prefix_len + W + K + 2)
     ctx = P.SpdContext(wl.shape, packed, dtabs, k, wl.orders, wl.lambdas(), wl.alpha, wl.tau, wl.delta, max_pos, wl.kv_dtype)
     if args.stage_bytes or args.stages:
@@ -402,6 +483,7 @@ def main():
     ap.add_argument("--retain", type=int, default=0, help="profiling only: n-grams kept per order")
     ap.add_argument("--stream-len", type=int, default=0, help="profiling only: tokens of the n-gram corpus")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batch", type=int, default=1, help="requests stepped together (batched timesteps); 1 = the single-request kernel")
     args = ap.parse_args()
     if args.warmup < 1:
         args.warmup = 1

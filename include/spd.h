@@ -293,6 +293,24 @@ int spd_debug_expire(spd_ctx *ctx);
 int spd_debug_expire_products(spd_ctx *ctx);
 
 /*
+ * Batched timesteps (the paper's closing remark that batching is complementary to Superposed Decoding: every
+ * request of a batch still needs only one pass for its k drafts).  ctxs: HOST array of n different contexts
+ * (1 <= n <= 128) over the same weights, device and stream, each prefilled on its own prefix, none with a stop
+ * token; the first one lends its workspace and must have the long-prefix path (max_pos >= 130, head size 64 or
+ * 128).  One timestep of all n requests streams the weights once: the requests' superposed inputs (Eq. 3) are the
+ * token rows of the tensor-core products, each request keeps its own KV cache, position and draft state, and its
+ * step is the one spd_step takes (Eq. 2-7).  spd_batch_generate enqueues n_steps timesteps and synchronises once;
+ * every context can afterwards be read (spd_debug_read), stepped alone or in another batch.  spd_batch_step takes
+ * one timestep and returns HOST rows of SPD_MAX_K entries per request (the first k used, any array may be NULL):
+ * out_ids[r][i], out_parent[r][i], out_gamma[r][i] as spd_step gives them for request r.
+ * SPD_ERANGE: n beyond 128 or the leading context without the long-prefix path, or a request out of positions;
+ * SPD_EINVAL: contexts of different models, devices or streams, a context twice, a stop token configured;
+ * SPD_ESTATE: a request not prefilled.  A device error of any request is returned (the first one found).
+ */
+int spd_batch_generate(spd_ctx *const *ctxs, int32_t n, int32_t n_steps);
+int spd_batch_step(spd_ctx *const *ctxs, int32_t n, int32_t *out_ids, int32_t *out_parent, float *out_gamma);
+
+/*
  * 1 once the most probable draft has ended with the stop token (cfg.eos_id; always 0 without one), as seen by the
  * last synchronising call.  spd_step / spd_generate / spd_generate_async then return SPD_ESTATE until the context is
  * prefilled or reset again.  The drafts stay readable; the paper does not say what happens to the other drafts.

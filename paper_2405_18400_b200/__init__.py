@@ -5,7 +5,7 @@ arguments (torch is used for device memory and streams).  Importing it does not 
 library; the first use does, and fails loudly if the library is missing and cannot be built.
 """
 from .binding import (SpdConfig, SpdError, SpdContext, build_ngram_tables, pack_weights, load_library,
-                      DBG, status_name)
+                      DBG, status_name, spd_batch_generate, spd_batch_step)
 
 __all__ = ["SpdConfig", "SpdError", "SpdContext", "build_ngram_tables", "pack_weights", "load_library", "DBG",
-           "status_name"]
+           "status_name", "spd_batch_generate", "spd_batch_step"]

@@ -66,7 +66,7 @@ _lib: Optional[C.CDLL] = None
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
            "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
-           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished"]
+           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished", "spd_batch_generate", "spd_batch_step"]
 
 
 def load_library() -> C.CDLL:
@@ -107,6 +107,8 @@ def load_library() -> C.CDLL:
     L.spd_debug_expire.argtypes = [C.c_void_p]
     L.spd_debug_trace.argtypes = [C.c_void_p, C.c_int]
     L.spd_finished.argtypes = [C.c_void_p]
+    L.spd_batch_generate.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    L.spd_batch_step.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_debug_expire_products.argtypes = [C.c_void_p]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
@@ -331,6 +333,25 @@ class SpdContext:
         cand_lp = np.ascontiguousarray(cand_lp, dtype=np.float32)
         _check(self.lib.spd_debug_score(self.h, hist.ctypes.data, hist.shape[1], logp.ctypes.data, cand_tok.ctypes.data,
                                         cand_lp.ctypes.data), "spd_debug_score")
+
+
+def _ctx_array(ctxs: Sequence["SpdContext"]):
+    return (C.c_void_p * len(ctxs))(*[c.h for c in ctxs])
+
+
+def spd_batch_generate(ctxs: Sequence["SpdContext"], n_steps: int) -> None:
+    """n_steps timesteps of all the contexts together, one pass over the weights per timestep."""
+    _check(load_library().spd_batch_generate(_ctx_array(ctxs), len(ctxs), n_steps), "spd_batch_generate")
+
+
+def spd_batch_step(ctxs: Sequence["SpdContext"]):
+    """One timestep of all the contexts together.  Returns per context (ids, parents, gamma) as spd_step does."""
+    n = len(ctxs)
+    ids = np.zeros((n, MAX_K), np.int32)
+    par = np.zeros((n, MAX_K), np.int32)
+    g = np.zeros((n, MAX_K), np.float32)
+    _check(load_library().spd_batch_step(_ctx_array(ctxs), n, ids.ctypes.data, par.ctypes.data, g.ctypes.data), "spd_batch_step")
+    return [(ids[r, : c.k].copy(), par[r, : c.k].copy(), g[r, : c.k].copy()) for r, c in enumerate(ctxs)]
 
 
 def spd_score_static(k: int, vocab: int, orders: Sequence[int], lam: Sequence[float], alpha: float, delta: float,

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libspd.so")
-SOURCES = ["spd_kernel.cu", "spd_prefill.cu", "spd_prefill_tc.cu", "spd_api.cu", "spd_ngram.cu"]
+SOURCES = ["spd_kernel.cu", "spd_prefill.cu", "spd_prefill_tc.cu", "spd_batch.cu", "spd_api.cu", "spd_ngram.cu"]
 
 
 def _nvcc() -> str:

@@ -16,6 +16,8 @@ extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm);
 extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm);
 extern "C" cudaError_t spd_internal_prefill_launch(const spd::KParams *p, int grid, cudaStream_t stream);
+extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd::KParams *kps, int n, int V, const __nv_bfloat16 *final_norm,
+                                               float *y_logits, cudaStream_t s, int *launches);
 
 namespace {
 
@@ -39,7 +41,8 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
-      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, tc_tmaps, tc_h, tc_q, tc_y, tc_x, total;
+      trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, tc_tmaps, tc_h, tc_q, tc_y, tc_x, bt_kp, bt_y,
+      total;
 };
 
 // Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 64 tokens send
@@ -117,6 +120,9 @@ Layout make_layout(const spd_config &c, int grid) {
   L.tc_q = take(tcr * c.d_model * 4);
   L.tc_y = take(tcr * wide * 4);
   L.tc_x = take(3 * tcr * (size_t)(c.d_model > c.d_ffn ? c.d_model : c.d_ffn) * 2);
+  // batched timesteps led by this context: the requests' parameters and their rows of logits
+  L.bt_kp = take(tcr ? (size_t)spd::kTcTile * sizeof(spd::KParams) : 0);
+  L.bt_y = take(tcr ? (size_t)spd::kTcTile * c.vocab * 4 : 0);
   L.total = off;
   return L;
 }
@@ -712,6 +718,100 @@ int spd_generate(spd_ctx *ctx, int32_t n_steps, int32_t *out_tokens, int32_t *ou
   for (int i = 0; i < k; ++i) {
     if (out_logp) out_logp[i] = logp[i];
     if (out_gamma) out_gamma[i] = gamma[i];
+  }
+  return SPD_OK;
+}
+
+namespace {
+
+// Checks a batch and enqueues n_steps timesteps of it; the requests' host-side counters move on.
+int batch_enqueue(spd_ctx *const *ctxs, int32_t n, int32_t n_steps) {
+  if (!ctxs || n < 1 || !ctxs[0]) return SPD_EINVAL;
+  spd_ctx *lead = ctxs[0];
+  if (lead->tc_rows < 1 || n > spd::kTcTile || n > lead->tc_rows) return SPD_ERANGE;
+  if (n_steps < 1) return SPD_ERANGE;
+  const spd_config &c0 = lead->cfg;
+  for (int r = 0; r < n; ++r) {
+    spd_ctx *x = ctxs[r];
+    if (!x) return SPD_EINVAL;
+    for (int q = 0; q < r; ++q)
+      if (ctxs[q] == x) return SPD_EINVAL;  // a request appears once
+    const spd_config &c = x->cfg;
+    if (c.n_layers != c0.n_layers || c.d_model != c0.d_model || c.n_heads != c0.n_heads || c.d_ffn != c0.d_ffn || c.vocab != c0.vocab ||
+        c.rms_eps != c0.rms_eps || x->device != lead->device || x->stream != lead->stream || x->kp.tok_emb != lead->kp.tok_emb ||
+        x->kp.lm_head != lead->kp.lm_head || x->layers_host[0].wqkv != lead->layers_host[0].wqkv)
+      return SPD_EINVAL;  // one model, one device, one stream
+    if (c.eos_id != -1) return SPD_EINVAL;  // stopping on a token is a single-request feature
+    if (!x->prefilled || x->stopped) return SPD_ESTATE;
+    const int pos0 = x->m + x->n_gen - 1;
+    if (pos0 + n_steps > c.max_pos || x->n_gen + n_steps > c.max_pos) return SPD_ERANGE;
+  }
+  int rc = set_device(lead);
+  if (rc) return rc;
+  // the requests' parameters in row order; pos0 = m - 1, so that a request's next position is pos0 + n_gen on the device
+  std::vector<spd::KParams> kps(n);
+  for (int r = 0; r < n; ++r) {
+    kps[r] = ctxs[r]->kp;
+    kps[r].pos0 = ctxs[r]->m - 1;
+    SPD_CUDA(cudaMemsetAsync(ctxs[r]->ws + ctxs[r]->lay.state, 0, head_bytes(false), lead->stream));
+  }
+  spd::KParams *dkp = reinterpret_cast<spd::KParams *>(lead->ws + lead->lay.bt_kp);
+  SPD_CUDA(cudaMemcpyAsync(dkp, kps.data(), kps.size() * sizeof(spd::KParams), cudaMemcpyHostToDevice, lead->stream));
+  SPD_CUDA(cudaStreamSynchronize(lead->stream));  // `kps` leaves scope
+  const spd::TcJob job = tc_job(lead);
+  for (int s = 0; s < n_steps; ++s) {
+    int launched = 0;
+    const cudaError_t e = spd_internal_batch_step(&job, dkp, n, c0.vocab, lead->kp.final_norm,
+                                                  reinterpret_cast<float *>(lead->ws + lead->lay.bt_y), lead->stream, &launched);
+    lead->launches += launched;
+    if (e != cudaSuccess) return cuda_fail(e, "batched timestep");
+  }
+  for (int r = 0; r < n; ++r) {
+    ctxs[r]->n_gen += n_steps;
+    ctxs[r]->decoding = false;
+  }
+  return SPD_OK;
+}
+
+int batch_wait(spd_ctx *const *ctxs, int32_t n) {
+  int first = SPD_OK;
+  for (int r = 0; r < n; ++r) {
+    const int rc = check_device_error(ctxs[r]);
+    if (rc) {
+      ctxs[r]->prefilled = false;
+      if (!first) first = rc;
+    }
+  }
+  return first;
+}
+
+}  // namespace
+
+int spd_batch_generate(spd_ctx *const *ctxs, int32_t n, int32_t n_steps) {
+  int rc = batch_enqueue(ctxs, n, n_steps);
+  if (rc) return rc;
+  return batch_wait(ctxs, n);
+}
+
+int spd_batch_step(spd_ctx *const *ctxs, int32_t n, int32_t *out_ids, int32_t *out_parent, float *out_gamma) {
+  int rc = batch_enqueue(ctxs, n, 1);
+  if (rc) return rc;
+  if ((rc = batch_wait(ctxs, n))) return rc;
+  for (int r = 0; r < n; ++r) {
+    spd_ctx *x = ctxs[r];
+    const int k = x->cfg.k;
+    int32_t ids[SPD_MAX_K], par[SPD_MAX_K];
+    float gamma[SPD_MAX_K];
+    const size_t row = (size_t)(x->n_gen - 1) * k * 4;
+    SPD_CUDA(cudaMemcpyAsync(ids, x->ws + x->lay.hist_tok + row, (size_t)k * 4, cudaMemcpyDeviceToHost, x->stream));
+    SPD_CUDA(cudaMemcpyAsync(par, x->ws + x->lay.hist_par + row, (size_t)k * 4, cudaMemcpyDeviceToHost, x->stream));
+    if ((rc = read_state(x, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
+    SPD_CUDA(cudaStreamSynchronize(x->stream));
+    for (int i = 0; i < k; ++i) {
+      if (out_ids) out_ids[r * SPD_MAX_K + i] = ids[i];
+      if (out_parent) out_parent[r * SPD_MAX_K + i] = par[i];
+      if (out_gamma) out_gamma[r * SPD_MAX_K + i] = gamma[i];
+    }
   }
   return SPD_OK;
 }

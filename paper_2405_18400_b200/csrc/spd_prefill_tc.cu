@@ -647,6 +647,26 @@ extern "C" cudaError_t spd_internal_tc_prepare(void) {
   return e;
 }
 
+// Launchers for the batched timestep (spd_batch.cu), which runs the same products and row-wise kernels on a tile of
+// requests instead of prefix tokens.
+extern "C" cudaError_t spd_internal_tc_gemm(const void *xmap, const void *wmap, float *Y, int n_tok, int N, int C, int x_term_rows,
+                                            spd::State *st, cudaStream_t s) {
+  const dim3 grid((n_tok + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
+  spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, wmap, Y, N, C, x_term_rows, st, 0);
+  return cudaGetLastError();
+}
+
+extern "C" cudaError_t spd_internal_tc_resid_norm(float *h, const float *y, const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int n_tok,
+                                                  int d, float eps, cudaStream_t s) {
+  spd::spd_tc_resid_norm_kernel<<<n_tok, 256, 0, s>>>(h, y, nullptr, nullptr, gain, X, term_stride, d, eps);
+  return cudaGetLastError();
+}
+
+extern "C" cudaError_t spd_internal_tc_swiglu(const float *Y, uint16_t *X, size_t term_stride, int n_tok, int f, cudaStream_t s) {
+  spd::spd_tc_swiglu_kernel<<<n_tok, 256, 0, s>>>(Y, X, term_stride, f);
+  return cudaGetLastError();
+}
+
 // Test hook: one tile of the first layer's QKV product whose first stage never arrives (see the kernel's `stall`).
 extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t s) {
   const spd::TcJob &j = *job;

@@ -31,3 +31,9 @@ struct TcJob {
 extern "C" cudaError_t spd_internal_tc_prepare(void);
 extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);
+// The long-prefix path's products and row-wise kernels for other callers (the batched timestep).
+extern "C" cudaError_t spd_internal_tc_gemm(const void *xmap, const void *wmap, float *Y, int n_tok, int N, int C, int x_term_rows,
+                                            spd::State *st, cudaStream_t s);
+extern "C" cudaError_t spd_internal_tc_resid_norm(float *h, const float *y, const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int n_tok,
+                                                  int d, float eps, cudaStream_t s);
+extern "C" cudaError_t spd_internal_tc_swiglu(const float *Y, uint16_t *X, size_t term_stride, int n_tok, int f, cudaStream_t s);

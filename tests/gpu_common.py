@@ -108,19 +108,20 @@ def compare_first_step(ctx, orc, prefix, stats=None, reset_draft=None, device=No
     return ids, g
 
 
-def compare_step(ctx, orc, stats=None):
+def compare_step(ctx, orc, stats=None, stepped=None, path="decode"):
     """One later timestep on both sides.  Exact ids / parents / counts when the oracle's margins exceed
     twice the measured float error; otherwise the device's choice must be one the oracle rates within
-    that error of its own, and the oracle follows it."""
+    that error of its own, and the oracle follows it.  `stepped` = (ids, parents, gamma) when the device has
+    already taken the step (as one request of a batch); `path` names the kernels that wrote the new cache row."""
     k = ctx.k
     tau, alpha = orc.cfg.tau, orc.cfg.alpha
     hist_o = orc.drafts()
     logP_o = orc.logP()
-    ids, par, g = ctx.spd_step()
-    following = _follow(ctx, orc, orc.T() + 1, "decode")
+    ids, par, g = ctx.spd_step() if stepped is None else stepped
+    following = _follow(ctx, orc, orc.T() + 1, path)
     orc.step_forward()
     if following:
-        _followed(orc, 1, stats, "decode")
+        _followed(orc, 1, stats, path)
     z, z_o = ctx.spd_debug_read("LOGITS").astype(np.float64), orc.logits()
     eps_z = float(np.abs(z - z_o).max())
     assert eps_z <= LOGIT_TOL, eps_z
