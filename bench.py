@@ -246,7 +246,7 @@ def run_ours(args, wl):
         host_weights = {n: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for n, v in weights.items()}
         log("[bench] weights to host %.1fs" % (time.time() - t0))
     t0 = time.time()
-    packed = P.pack_weights(weights, dev, consume=True)
+    packed = P.pack_weights(weights, dev, consume=True, images=not args.no_images)
     del weights
     dtabs = P.build_ngram_tables(tables, dev)
     torch.cuda.empty_cache()
@@ -483,6 +483,8 @@ def main():
     ap.add_argument("--retain", type=int, default=0, help="profiling only: n-grams kept per order")
     ap.add_argument("--stream-len", type=int, default=0, help="profiling only: tokens of the n-gram corpus")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-images", action="store_true",
+                    help="comparison only: no fragment-order weight images, decode timesteps on the float32 multiply loop")
     ap.add_argument("--batch", type=int, default=1, help="requests stepped together (batched timesteps); 1 = the single-request kernel")
     args = ap.parse_args()
     if args.warmup < 1:

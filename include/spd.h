@@ -79,11 +79,17 @@ typedef struct {
  *   wo        [d_model][d_model]
  *   wgate_up  [2*d_ffn][d_model]    row 2j = gate row j, row 2j+1 = up row j (interleaved)
  *   wdown     [d_model][d_ffn]
+ * Optional second images of lm_head, wqkv, wo and wgate_up in fragment order (spd_pack_image), same sizes: with all
+ * four present (every layer), d_model a multiple of 32, d_ffn of 4 and vocab of 8, the decode timesteps (Section 3,
+ * "Next Timesteps") multiply these matrices on the tensor cores; the row-major ones are still what the first
+ * timestep's kernels read.  Null members: every timestep uses the row-major matrices.
  */
 typedef struct {
   const void *tok_emb, *final_norm, *lm_head;
   const void *const *attn_norm, *const *wqkv, *const *wo;
   const void *const *ffn_norm, *const *wgate_up, *const *wdown;
+  const void *lm_head_img;
+  const void *const *wqkv_img, *const *wo_img, *const *wgate_up_img;
 } spd_weights;
 
 /*
@@ -186,6 +192,17 @@ int spd_destroy(spd_ctx *ctx);
 const char *spd_strerror(int status);
 /* Text of the last CUDA runtime error seen by this thread's calls ("" if none). */
 const char *spd_last_cuda_error(void);
+
+/*
+ * Fragment order of a weight matrix for the decode timesteps' products y = W x (Section 3: every later timestep is
+ * one pass of the superposed input through the decoder).  w: DEVICE, bf16 row-major [rows][cols], rows a multiple
+ * of 8, cols a multiple of 32; out: DEVICE, rows * cols * 2 bytes, 16-byte aligned, not overlapping w.  Every block
+ * of 8 rows x 32 columns is stored as 32 vectors of 16 bytes, vector 4 g + t = row g's column pairs 2t, 2t+8,
+ * 2t+16, 2t+24 of the block (the operand registers of two m16n8k16 tensor-core instructions for that lane); blocks
+ * of one 8-row unit follow one another in column order, units in row order.  Enqueued on `stream` (a cudaStream_t,
+ * may be null), not synchronised.  SPD_EINVAL for null pointers or sizes that do not divide; SPD_ECUDA.
+ */
+int spd_pack_image(const void *w, int32_t rows, int32_t cols, void *out, void *stream);
 
 /*
  * N-gram table construction (host side; the tables of Section 4 re-laid as hash tables).

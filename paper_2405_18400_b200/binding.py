@@ -53,7 +53,8 @@ _PP = C.POINTER(C.c_void_p)
 
 class _Weights(C.Structure):
     _fields_ = [("tok_emb", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)] + [
-        (n, _PP) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "wgate_up", "wdown")]
+        (n, _PP) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "wgate_up", "wdown")] + [("lm_head_img", C.c_void_p)] + [
+        (n, _PP) for n in ("wqkv_img", "wo_img", "wgate_up_img")]
 
 
 class _Table(C.Structure):
@@ -66,7 +67,7 @@ _lib: Optional[C.CDLL] = None
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
            "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
-           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished", "spd_batch_generate", "spd_batch_step"]
+           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished", "spd_batch_generate", "spd_batch_step", "spd_pack_image"]
 
 
 def load_library() -> C.CDLL:
@@ -110,6 +111,7 @@ def load_library() -> C.CDLL:
     L.spd_batch_generate.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     L.spd_batch_step.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_debug_expire_products.argtypes = [C.c_void_p]
+    L.spd_pack_image.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
     L.spd_set_ring.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
@@ -150,10 +152,25 @@ def build_ngram_tables(tables: Sequence[Dict[str, object]], device: str | torch.
     return out
 
 
-def pack_weights(weights: Dict[str, object], device: str | torch.device = "cuda:0", consume: bool = False) -> Dict[str, object]:
+def _image(t: torch.Tensor) -> Optional[torch.Tensor]:
+    """Fragment-order image of a bf16 matrix (spd_pack_image), or None when its shape does not divide."""
+    rows, cols = t.shape
+    if rows % 8 or cols % 32 or t.dtype != torch.bfloat16:
+        return None
+    out = torch.empty_like(t)
+    with torch.cuda.device(t.device):
+        _check(load_library().spd_pack_image(t.data_ptr(), rows, cols, out.data_ptr(), torch.cuda.current_stream(t.device).cuda_stream),
+               "spd_pack_image")
+    return out
+
+
+def pack_weights(weights: Dict[str, object], device: str | torch.device = "cuda:0", consume: bool = False,
+                 images: bool = True) -> Dict[str, object]:
     """Lays the decoder's tensors out as spd_weights wants them, on `device`: wqkv = rows of W_q, W_k,
     W_v stacked; wgate_up = gate and up rows interleaved.  With consume=True the per-layer inputs are
-    dropped from `weights` as they are packed (halves peak memory)."""
+    dropped from `weights` as they are packed (halves peak memory).  images=True adds the fragment-order
+    images of lm_head, wqkv, wo and wgate_up that let the decode timesteps use the tensor cores (all four or
+    none: shapes that do not divide leave them out)."""
     dev = torch.device(device)
     out: Dict[str, object] = {k: weights[k].to(dev).contiguous() for k in ("tok_emb", "final_norm", "lm_head")}
     for k in ("attn_norm", "wqkv", "wo", "ffn_norm", "wgate_up", "wdown"):
@@ -170,6 +187,12 @@ def pack_weights(weights: Dict[str, object], device: str | torch.device = "cuda:
         if consume:
             for k in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown"):
                 weights[k][l] = None
+    if images and dev.type == "cuda":
+        img: Dict[str, object] = {"lm_head_img": _image(out["lm_head"])}
+        for k in ("wqkv", "wo", "wgate_up"):
+            img[k + "_img"] = [_image(t) for t in out[k]]
+        if img["lm_head_img"] is not None and all(t is not None for k in ("wqkv", "wo", "wgate_up") for t in img[k + "_img"]):
+            out.update(img)
     return out
 
 
@@ -208,6 +231,12 @@ class SpdContext:
             arr = (C.c_void_p * shape.n_layers)(*[t.data_ptr() for t in packed[name]])
             self._keep.append(arr)
             setattr(w, name, C.cast(arr, _PP))
+        if "lm_head_img" in packed:
+            w.lm_head_img = packed["lm_head_img"].data_ptr()
+            for name in ("wqkv_img", "wo_img", "wgate_up_img"):
+                arr = (C.c_void_p * shape.n_layers)(*[t.data_ptr() for t in packed[name]])
+                self._keep.append(arr)
+                setattr(w, name, C.cast(arr, _PP))
         tabs = (_Table * max(1, len(tables)))()
         for i, t in enumerate(tables):
             tabs[i].n, tabs[i].ngram_slots, tabs[i].ctx_slots = t["n"], t["ngram_slots"], t["ctx_slots"]

@@ -16,6 +16,7 @@ extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm);
 extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm);
 extern "C" cudaError_t spd_internal_prefill_launch(const spd::KParams *p, int grid, cudaStream_t stream);
+extern "C" cudaError_t spd_internal_pack_image(const void *w, void *out, int rows, int cols, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd::KParams *kps, int n, int V, const __nv_bfloat16 *final_norm,
                                                float *y_logits, cudaStream_t s, int *launches);
 
@@ -34,7 +35,7 @@ int cuda_fail(cudaError_t e, const char *what) {
     if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
   } while (0)
 
-constexpr size_t kPartBytes = 20480;  // per-block scratch after the ring: row partials / attention merge / tail
+constexpr size_t kPartBytes = spd::kScratchBytes;  // per-block scratch after the ring: row partials / attention merge / tail
 constexpr size_t kSmemLimit = 232448; // 227 KB opt-in maximum per block on sm_100
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -183,12 +184,18 @@ struct spd_ctx {
 
 namespace {
 
-int pick_ring(const spd_config &c, int32_t stage_bytes, int32_t n_stages, int32_t *out_stage, int32_t *out_n) {
+// Shared memory behind the scratch area that the fragment-order multiply loop needs for the activation vector: 12
+// vectors of 16 bytes per 32 columns.
+size_t frag_bytes(const spd_config &c) { return (size_t)c.d_model / 32 * 192; }
+
+// reserve: bytes of shared memory kept back behind the ring and the scratch area.
+int pick_ring(const spd_config &c, int32_t stage_bytes, int32_t n_stages, size_t reserve, int32_t *out_stage, int32_t *out_n) {
   const size_t maxrow = (size_t)2 * (c.d_model > c.d_ffn ? c.d_model : c.d_ffn);
   size_t sb = stage_bytes > 0 ? (size_t)stage_bytes : 32768;
   if (stage_bytes <= 0 && sb < maxrow) sb = align_up(maxrow, 1024);
   if (sb % 128 || sb < maxrow) return SPD_EINVAL;
-  const size_t avail = kSmemLimit - kPartBytes - 2048;  // static shared memory and alignment slack
+  if (reserve + kPartBytes + 4096 >= kSmemLimit) return SPD_EINVAL;
+  const size_t avail = kSmemLimit - kPartBytes - 4096 - reserve;  // 4096: static shared memory and alignment slack
   int ns = n_stages > 0 ? n_stages : (int)(avail / sb);
   if (ns > spd::kMaxStages) ns = spd::kMaxStages;
   if (ns < 2 || (size_t)ns * sb > avail) return SPD_EINVAL;
@@ -384,9 +391,17 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
 
   spd::KParams &kp = ctx->kp;
   std::memset(&kp, 0, sizeof kp);
-  int rc = pick_ring(*cfg, 0, 0, &kp.stage_bytes, &kp.n_stages);
+  // Fragment-order images: all or none, and only for shapes the tensor-core multiply loop serves.
+  bool img = w->lm_head_img && w->wqkv_img && w->wo_img && w->wgate_up_img && cfg->d_model % 32 == 0 && cfg->vocab % spd::kUnitRows == 0 &&
+             (2 * cfg->d_ffn) % spd::kUnitRows == 0;
+  for (int l = 0; l < cfg->n_layers && img; ++l) img = w->wqkv_img[l] && w->wo_img[l] && w->wgate_up_img[l];
+  int rc = pick_ring(*cfg, 0, 0, img ? frag_bytes(*cfg) : 0, &kp.stage_bytes, &kp.n_stages);
+  if (rc && img) {  // no room for the fragments: the float32 multiply loop
+    img = false;
+    rc = pick_ring(*cfg, 0, 0, 0, &kp.stage_bytes, &kp.n_stages);
+  }
   if (rc) return fail(rc);
-  ctx->dyn_smem = (size_t)kp.stage_bytes * kp.n_stages + kPartBytes;
+  ctx->dyn_smem = (size_t)kp.stage_bytes * kp.n_stages + kPartBytes + (img ? frag_bytes(*cfg) : 0);
   int per_sm = 0;
   e = spd_internal_prepare(ctx->dyn_smem, &per_sm);
   if (e != cudaSuccess) return fail(cuda_fail(e, "kernel attributes"));
@@ -456,6 +471,15 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
     layers[l].ffn_norm = static_cast<const __nv_bfloat16 *>(w->ffn_norm[l]);
     layers[l].wgate_up = static_cast<const __nv_bfloat16 *>(w->wgate_up[l]);
     layers[l].wdown = static_cast<const __nv_bfloat16 *>(w->wdown[l]);
+    layers[l].wqkv_img = layers[l].wo_img = layers[l].wgate_up_img = nullptr;
+  }
+  if (img) {
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      layers[l].wqkv_img = static_cast<const __nv_bfloat16 *>(w->wqkv_img[l]);
+      layers[l].wo_img = static_cast<const __nv_bfloat16 *>(w->wo_img[l]);
+      layers[l].wgate_up_img = static_cast<const __nv_bfloat16 *>(w->wgate_up_img[l]);
+    }
+    kp.lm_head_img = static_cast<const __nv_bfloat16 *>(w->lm_head_img);
   }
   // tensor maps of the matrices in the order the prefill kernel walks them
   std::vector<CUtensorMap> tmaps((size_t)4 * cfg->n_layers + 1);
@@ -503,10 +527,11 @@ int spd_destroy(spd_ctx *ctx) {
 int spd_set_ring(spd_ctx *ctx, int32_t stage_bytes, int32_t n_stages) {
   if (!ctx) return SPD_EINVAL;
   int32_t sb, ns;
-  int rc = pick_ring(ctx->cfg, stage_bytes, n_stages, &sb, &ns);
+  const size_t reserve = ctx->kp.lm_head_img ? frag_bytes(ctx->cfg) : 0;
+  int rc = pick_ring(ctx->cfg, stage_bytes, n_stages, reserve, &sb, &ns);
   if (rc) return rc;
   if ((rc = set_device(ctx))) return rc;
-  const size_t dyn = (size_t)sb * ns + kPartBytes;
+  const size_t dyn = (size_t)sb * ns + kPartBytes + reserve;
   int per_sm = 0;
   SPD_CUDA(spd_internal_prepare(dyn > ctx->dyn_smem ? dyn : ctx->dyn_smem, &per_sm));
   if (per_sm < 1) return SPD_EINVAL;
@@ -817,6 +842,13 @@ int spd_batch_step(spd_ctx *const *ctxs, int32_t n, int32_t *out_ids, int32_t *o
 }
 
 int64_t spd_launch_count(const spd_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int spd_pack_image(const void *w, int32_t rows, int32_t cols, void *out, void *stream) {
+  if (!w || !out || rows < spd::kUnitRows || cols < 32 || rows % spd::kUnitRows || cols % 32 || ((uintptr_t)w % 16) || ((uintptr_t)out % 16)) return SPD_EINVAL;
+  const cudaError_t e = spd_internal_pack_image(w, out, rows, cols, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "spd_pack_image");
+  return SPD_OK;
+}
 
 int spd_finished(const spd_ctx *ctx) { return ctx && ctx->stopped ? 1 : 0; }
 

@@ -26,17 +26,28 @@
 
 namespace spd {
 
+// The block's shared memory.  The kernels' loops name these variables directly (their addresses are constants)
+// instead of carrying pointers to them in registers.
+extern __shared__ __align__(128) uint8_t smem[];  // the ring's stages, then the scratch area (row partials / attention merge / tail)
+__shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages];
+__shared__ __align__(16) float s_red[64];
+__shared__ float2 s_rope[128];  // the current position's row of the rotary table (head sizes up to 256)
+constexpr int kGainSlots = 256;  // gain pointers kept in shared memory: models of up to 127 layers (deeper ones read them late)
+__shared__ const __nv_bfloat16 *s_gain_ptrs[kGainSlots];
+__shared__ int s_dead, s_quit;
+
+__device__ __forceinline__ float *scratch_base(const KParams &p) { return reinterpret_cast<float *>(smem + (size_t)p.n_stages * p.stage_bytes); }
 
 // Bounded wait on an mbarrier phase.  Returns at once when the block is already giving up.
 __device__ __forceinline__ void wait_mbar(Blk &b, uint64_t *bar, uint32_t parity, int info) {
   if (mbar_try_wait(bar, parity)) return;
-  if (*b.dead) return;
+  if (s_dead) return;
   unsigned long long t0 = globaltimer();
   uint32_t n = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++n & 31u) == 0) {
-      if (*b.dead) return;
-      if (ld_relaxed(&b.p->st->abort_flag)) { *b.dead = 1; return; }
+      if (s_dead) return;
+      if (ld_relaxed(&b.p->st->abort_flag)) { s_dead = 1; return; }
       if (globaltimer() - t0 > kWaitNs) { give_up(b, kErrTimeout, info); return; }
     }
   }
@@ -48,7 +59,7 @@ __device__ __forceinline__ bool grid_barrier(Blk &b) {
   named_sync(1, kConsumerThreads);
   if (threadIdx.x == 0) {
     b.bar_target += gridDim.x;
-    if (!*b.dead) {
+    if (!s_dead) {
       unsigned int *bar = &b.p->st->bar;
       __threadfence();
       atomicAdd(bar, 1u);
@@ -56,15 +67,15 @@ __device__ __forceinline__ bool grid_barrier(Blk &b) {
       uint32_t n = 0;
       while ((int)(ld_acquire(bar) - b.bar_target) < 0) {
         if ((++n & 63u) == 0) {
-          if (ld_relaxed(&b.p->st->abort_flag)) { *b.dead = 1; break; }
+          if (ld_relaxed(&b.p->st->abort_flag)) { s_dead = 1; break; }
           if (globaltimer() - t0 > kWaitNs) { give_up(b, kErrTimeout, 100); break; }
         }
       }
     }
-    *b.quit = *b.dead;
+    s_quit = s_dead;
   }
   named_sync(1, kConsumerThreads);
-  return *b.quit != 0;
+  return s_quit != 0;
 }
 
 __device__ __forceinline__ void cta_rows(int R, int gran, int &r0, int &r1) {
@@ -94,34 +105,73 @@ __device__ __forceinline__ void produce_matrix(Blk &b, Producer &pr, const __nv_
     const int t1 = min(t0 + kTile, r1);
     for (int r = t0; r < t1; r += rpc) {
       const int n = min(rpc, t1 - r);
-      wait_mbar(b, &b.empty[pr.stage], pr.phase ^ 1u, 200);
-      if (*b.dead) return;
+      wait_mbar(b, &s_empty[pr.stage], pr.phase ^ 1u, 200);
+      if (s_dead) return;
       const uint32_t bytes = (uint32_t)n * rowbytes;
-      mbar_expect_tx(&b.full[pr.stage], bytes);
-      bulk_load(b.ring + (size_t)pr.stage * p.stage_bytes, (const uint8_t *)W + (size_t)r * rowbytes, bytes,
-                &b.full[pr.stage]);
+      mbar_expect_tx(&s_full[pr.stage], bytes);
+      bulk_load(smem + (size_t)pr.stage * p.stage_bytes, (const uint8_t *)W + (size_t)r * rowbytes, bytes,
+                &s_full[pr.stage]);
       if (pr.issued < (uint32_t)p.n_stages) ++pr.issued;
       if (++pr.stage == (uint32_t)p.n_stages) { pr.stage = 0; pr.phase ^= 1u; }
     }
   }
 }
 
-template <bool kSampler>
+constexpr int kPairBytes = kUnitRows * 64;  // a unit's share of a pair of 16-column blocks: 4 lanes of 16 bytes per row
+// Bytes of a fragment-order unit that one ring stage takes: whole pairs of 16-column blocks.
+__device__ __forceinline__ uint32_t img_chunk(const KParams &p) { return (uint32_t)p.stage_bytes / kPairBytes * kPairBytes; }
+
+// A matrix in fragment order (spd_pack_image): the units of this block, each unit in stages of img_chunk bytes and a
+// shorter last one.
+__device__ __forceinline__ void produce_image(Blk &b, Producer &pr, const __nv_bfloat16 *img, int R, int C) {
+  const KParams &p = *b.p;
+  int r0, r1;
+  cta_rows(R, kUnitRows, r0, r1);
+  const uint32_t unit_bytes = (uint32_t)C * 2u * kUnitRows;
+  for (int r = r0; r < r1; r += kUnitRows) {
+    const uint8_t *src = reinterpret_cast<const uint8_t *>(img) + (size_t)(r / kUnitRows) * unit_bytes;
+    for (uint32_t off = 0; off < unit_bytes; off += img_chunk(p)) {
+      const uint32_t bytes = unit_bytes - off < img_chunk(p) ? unit_bytes - off : img_chunk(p);
+      wait_mbar(b, &s_empty[pr.stage], pr.phase ^ 1u, 200);
+      if (s_dead) return;
+      mbar_expect_tx(&s_full[pr.stage], bytes);
+      bulk_load(smem + (size_t)pr.stage * p.stage_bytes, src + off, bytes, &s_full[pr.stage]);
+      if (pr.issued < (uint32_t)p.n_stages) ++pr.issued;
+      if (++pr.stage == (uint32_t)p.n_stages) { pr.stage = 0; pr.phase ^= 1u; }
+    }
+  }
+}
+
+template <bool kSampler, int kImgs>
 __device__ void producer_main(Blk &b) {
+  constexpr bool kImg = kImgs > 0;
   const KParams &p = *b.p;
   Producer pr{0u, 0u, 0u};
-  for (int it = 0; it < p.n_iters && !*b.dead; ++it) {
-    for (int l = 0; l < p.L && !*b.dead; ++l) {
-      const LayerW lw = p.layers[l];
-      produce_matrix(b, pr, lw.wqkv, 3 * p.d, p.d, 2);
-      produce_matrix(b, pr, lw.wo, p.d, p.d, 1);
-      produce_matrix(b, pr, lw.wgate_up, 2 * p.f, p.d, 2);
+  // The layers' pointers sit in device memory that the weight stream has long pushed out of L2 when their turn
+  // comes: each layer's are fetched while the layer before is streamed.
+  LayerW lw = p.layers[0];
+  for (int it = 0; it < p.n_iters && !s_dead; ++it) {
+    for (int l = 0; l < p.L && !s_dead; ++l) {
+      const LayerW nxt = p.layers[l + 1 < p.L ? l + 1 : 0];
+      if constexpr (kImg) {
+        produce_image(b, pr, lw.wqkv_img, 3 * p.d, p.d);
+        produce_image(b, pr, lw.wo_img, p.d, p.d);
+        produce_image(b, pr, lw.wgate_up_img, 2 * p.f, p.d);
+      } else {
+        produce_matrix(b, pr, lw.wqkv, 3 * p.d, p.d, 2);
+        produce_matrix(b, pr, lw.wo, p.d, p.d, 1);
+        produce_matrix(b, pr, lw.wgate_up, 2 * p.f, p.d, 2);
+      }
       produce_matrix(b, pr, lw.wdown, p.d, p.f, 1);
+      lw = nxt;
     }
     const bool head = kSampler ? p.mode != kModePrefill : p.mode == kModeDecode;
-    if (head || it == p.n_iters - 1) produce_matrix(b, pr, p.lm_head, p.V, p.d, 1);
+    if (head || it == p.n_iters - 1) {
+      if constexpr (kImg) produce_image(b, pr, p.lm_head_img, p.V, p.d);
+      else produce_matrix(b, pr, p.lm_head, p.V, p.d, 1);
+    }
   }
-  if (*b.dead) {
+  if (s_dead) {
     // Giving up: nothing more is issued; wait (bounded) until every copy already issued has landed,
     // so that no copy writes into shared memory after the block has gone.
     uint32_t s = pr.stage, ph = pr.phase;
@@ -129,7 +179,7 @@ __device__ void producer_main(Blk &b) {
       if (s == 0) { s = (uint32_t)p.n_stages; ph ^= 1u; }
       --s;
       unsigned long long t0 = globaltimer();
-      while (!mbar_try_wait(&b.full[s], ph) && globaltimer() - t0 < kWaitNs) {}
+      while (!mbar_try_wait(&s_full[s], ph) && globaltimer() - t0 < kWaitNs) {}
     }
   }
 }
@@ -257,8 +307,9 @@ __device__ __forceinline__ void store_kv(const KParams &p, void *cache, size_t i
 }
 
 // Finishes rows [t0, t1) of the current matrix from the warps' partial sums.
+// rs: the factor of the phase's RMSNorm, 1 / rms(h), which the prologue left out of x (1 for a phase without one).
 __device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, const float *part, int t0, int t1, bool have_h,
-                                         float h_pre) {
+                                         float h_pre, float rs) {
   const KParams &p = *b.p;
   const int tid = threadIdx.x;
   const int rows = t1 - t0;
@@ -266,11 +317,11 @@ __device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, co
     // rows come in pairs (2i, 2i+1) of one head: rotate q and k, append k and v to the cache
     if (tid * 2 < rows) {
       const int r = t0 + tid * 2;
-      float a = part_sum(part + (size_t)(tid * 2) * kConsumerWarps);
-      float c = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps);
+      float a = part_sum(part + (size_t)(tid * 2) * kConsumerWarps) * rs;
+      float c = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps) * rs;
       const int sec = r / p.d, col = r - sec * p.d;
       if (sec < 2) {
-        const float2 cs = p.rope[(size_t)ea.pos * (p.hd / 2) + (col % p.hd) / 2];
+        const float2 cs = s_rope[(col % p.hd) / 2];  // the position's row of the rotary table
         const float ra = a * cs.x - c * cs.y, rc = a * cs.y + c * cs.x;
         a = ra;
         c = rc;
@@ -296,12 +347,12 @@ __device__ __forceinline__ void epilogue(Blk &b, int kind, const EpiArgs &ea, co
     }
   } else if (kind == kEpiSwiGLU) {
     if (tid * 2 < rows) {
-      const float g = part_sum(part + (size_t)(tid * 2) * kConsumerWarps);
-      const float up = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps);
+      const float g = part_sum(part + (size_t)(tid * 2) * kConsumerWarps) * rs;
+      const float up = part_sum(part + (size_t)(tid * 2 + 1) * kConsumerWarps) * rs;
       p.u[(t0 >> 1) + tid] = g / (1.f + __expf(-g)) * up;
     }
   } else {
-    if (tid < rows) p.logits[t0 + tid] = part_sum(part + (size_t)tid * kConsumerWarps);
+    if (tid < rows) p.logits[t0 + tid] = part_sum(part + (size_t)tid * kConsumerWarps) * rs;
   }
 }
 
@@ -317,42 +368,183 @@ __device__ __forceinline__ void consume_matrix(Blk &b, int R, int C, int gran, c
   // the residual rows this thread will update in the first tile are fetched now, off the critical path
   float h_pre = 0.f;
   if (kind == kEpiAddH && r0 + (int)threadIdx.x < min(r0 + kTile, r1)) h_pre = __ldcg(p.h + r0 + threadIdx.x);
+  float rs = 1.f;
   int buf = 0;
   for (int t0 = r0; t0 < r1; t0 += kTile) {
     const int t1 = min(t0 + kTile, r1);
-    float *part = b.part + (size_t)buf * kTile * kConsumerWarps;
+    float *part = scratch_base(p) + (size_t)buf * kTile * kConsumerWarps;
     for (int r = t0; r < t1; r += rpc) {
       const int n = min(rpc, t1 - r);
-      wait_mbar(b, &b.full[b.c_stage], b.c_phase, 300);
-      const uint8_t *stage = b.ring + (size_t)b.c_stage * p.stage_bytes;
+      wait_mbar(b, &s_full[b.c_stage], b.c_phase, 300);
+      const uint8_t *stage = smem + (size_t)b.c_stage * p.stage_bytes;
       float *prow = part + (size_t)(r - t0) * kConsumerWarps;
       if (n > 4) consume_chunk<8>(stage, n, rowbytes, nv, xr, prow, warp, lane);
       else if (n > 2) consume_chunk<4>(stage, n, rowbytes, nv, xr, prow, warp, lane);
       else if (n > 1) consume_chunk<2>(stage, n, rowbytes, nv, xr, prow, warp, lane);
       else consume_chunk<1>(stage, n, rowbytes, nv, xr, prow, warp, lane);
       __syncwarp();
-      if (lane == 0) mbar_arrive(&b.empty[b.c_stage]);
+      if (lane == 0) mbar_arrive(&s_empty[b.c_stage]);
       if (++b.c_stage == (uint32_t)p.n_stages) { b.c_stage = 0; b.c_phase ^= 1u; }
     }
     named_sync(1, kConsumerThreads);
-    epilogue(b, kind, ea, part, t0, t1, t0 == r0, h_pre);
+    if (kind != kEpiAddH && t0 == r0) {
+      // x came from prologue_norm without the factor 1 / rms(h): the warps' sums of squares are in red[] by now
+      const float4 *q = reinterpret_cast<const float4 *>(s_red);
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < kConsumerWarps / 4; ++i) {
+        const float4 a = q[i];
+        ss += a.x;
+        ss += a.y;
+        ss += a.z;
+        ss += a.w;
+      }
+      rs = rsqrtf(ss / (float)C + p.eps);
+    }
+    epilogue(b, kind, ea, part, t0, t1, t0 == r0, h_pre, rs);
+    buf ^= 1;
+  }
+}
+
+// ---------------------------------------------------------------- consumer: matrices in fragment order on the tensor cores
+// D (16 x 8) += A (16 x 16) * B (16 x 8): mma.sync m16n8k16, bf16 in, float32 accumulate.  A = a unit's weight rows x 16
+// columns in its first rows (the others are zero: a1 = a3 = 0), B = the three terms of 16 values of x in columns 0..2, so
+// that a lane's B registers are all in use and stay in registers for a whole phase.  d[0], d[1] of lane 4 g + t: weight
+// row g times terms 2t and 2t + 1; d[2], d[3] stay zero.
+__device__ __forceinline__ void mma_terms(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+
+// Term g (0, 1, 2) of v = hi + mid + lo, each the leading 8 significant bits of what is left (by truncation), so that
+// the three bf16 terms add up to v exactly and the tensor cores multiply exact operands.
+__device__ __forceinline__ uint32_t term_of(float v, int g) {
+  const uint32_t hi = __float_as_uint(v) & 0xffff0000u;
+  const float r1 = v - __uint_as_float(hi);
+  const uint32_t mid = __float_as_uint(r1) & 0xffff0000u;
+  const float r2 = r1 - __uint_as_float(mid);
+  const uint32_t pick = g == 0 ? hi : (g == 1 ? mid : __float_as_uint(r2));
+  return pick >> 16;
+}
+
+// The activation vector as B fragments in shared memory, behind the scratch area: per pair of 16-column blocks 12
+// vectors of 16 bytes, vector 4 g + t = term g of columns 2t, 2t+1 | 2t+8, 2t+9 of the first block and the same of
+// the second (what lane 4 g + t feeds to the two instructions of the pair; lanes 12..31 feed zeros).
+__device__ __forceinline__ uint32_t *xfrag_base(const KParams &p) {
+  return reinterpret_cast<uint32_t *>(smem + (size_t)p.n_stages * p.stage_bytes + kScratchBytes);
+}
+
+// Stores the thread's column vectors (8 consecutive columns each, as the prologues leave them in xr) as fragments.
+__device__ __forceinline__ void store_frags(const KParams &p, int C, const float (&xr)[kMaxVec][8]) {
+  uint32_t *xf = xfrag_base(p);
+  const int nv = C / 8;
+#pragma unroll
+  for (int i = 0; i < kMaxVec; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) {
+      // columns 8 v .. 8 v + 7: pair v / 4, word (v & 3) of each vector = block (v / 2) & 1, half v & 1
+      uint32_t *dst = xf + (size_t)(v >> 2) * 48 + (v & 3);
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const float x0 = xr[i][2 * t], x1 = xr[i][2 * t + 1];
+#pragma unroll
+        for (int g = 0; g < 3; ++g) dst[g * 16 + t * 4] = term_of(x0, g) | (term_of(x1, g) << 16);
+      }
+    }
+  }
+}
+
+// Streams this block's units of one matrix in fragment order through the ring: per unit and pair of column blocks one
+// 16-byte load of weights (lanes of the unit's rows; the others feed zero rows) and one of x (the fragments of two
+// instructions) and two instructions, the pairs of a stage dealt to the warps in turn; a row's sum is the sum of its
+// three terms' columns of the accumulator.
+__device__ __forceinline__ void consume_image(Blk &b, int R, int C, int kind, const EpiArgs &ea) {
+  const KParams &p = *b.p;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int r0, r1;
+  cta_rows(R, kUnitRows, r0, r1);
+  const int n_pairs = C / 32;
+  const uint4 *xf = reinterpret_cast<const uint4 *>(xfrag_base(p)) + lane;  // lanes < 12 only
+  float h_pre = 0.f;
+  if (kind == kEpiAddH && r0 + (int)threadIdx.x < min(r0 + kTile, r1)) h_pre = __ldcg(p.h + r0 + threadIdx.x);
+  float rs = 1.f;
+  int buf = 0;
+  for (int t0 = r0; t0 < r1; t0 += kTile) {
+    const int t1 = min(t0 + kTile, r1);
+    float *part = scratch_base(p) + (size_t)buf * kTile * kConsumerWarps;
+    for (int r = t0; r < t1; r += kUnitRows) {
+      float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+      const int per_stage = (int)(img_chunk(p) / kPairBytes);
+      for (int pr0 = 0; pr0 < n_pairs; pr0 += per_stage) {  // one stage
+        wait_mbar(b, &s_full[b.c_stage], b.c_phase, 300);
+        const uint8_t *stage = smem + (size_t)b.c_stage * p.stage_bytes;
+        const int n = min(per_stage, n_pairs - pr0);
+#pragma unroll 1  // unrolled, the loop costs more registers than the kernel has
+        for (int j = warp; j < n; j += kConsumerWarps) {
+          uint4 w = make_uint4(0u, 0u, 0u, 0u);
+          if (lane < 4 * kUnitRows) w = lds128(stage + ((size_t)j * (4 * kUnitRows) + lane) * 16);
+          uint4 x = make_uint4(0u, 0u, 0u, 0u);
+          if (lane < 12) x = xf[(size_t)(pr0 + j) * 12];
+          mma_terms(c0, w.x, w.y, x.x, x.y);
+          mma_terms(c1, w.z, w.w, x.z, x.w);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[b.c_stage]);
+        if (++b.c_stage == (uint32_t)p.n_stages) { b.c_stage = 0; b.c_phase ^= 1u; }
+      }
+      // row g: terms 0 and 1 in lane 4 g, term 2 in lane 4 g + 1 (whose d[1] is a sum of zeros)
+      const float s01 = (c0[0] + c1[0]) + (c0[1] + c1[1]);
+      const float s2 = __shfl_down_sync(0xffffffffu, s01, 1);
+      if ((lane & 3) == 0 && lane < 4 * kUnitRows) part[(size_t)(r - t0 + (lane >> 2)) * kConsumerWarps + warp] = s01 + s2;
+    }
+    named_sync(1, kConsumerThreads);
+    if (kind != kEpiAddH && t0 == r0) {
+      const float4 *q = reinterpret_cast<const float4 *>(s_red);
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < kConsumerWarps / 4; ++i) {
+        const float4 a = q[i];
+        ss += a.x;
+        ss += a.y;
+        ss += a.z;
+        ss += a.w;
+      }
+      rs = rsqrtf(ss / (float)C + p.eps);
+    }
+    epilogue(b, kind, ea, part, t0, t1, t0 == r0, h_pre, rs);
     buf ^= 1;
   }
 }
 
 // ---------------------------------------------------------------- consumer: activation prologues
-__device__ __forceinline__ float block_sum(Blk &b, float v) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  named_sync(1, kConsumerThreads);  // red[] free again
-  if (lane == 0) b.red[warp] = v;
-  named_sync(1, kConsumerThreads);
-  float s = 0.f;
-#pragma unroll
-  for (int w = 0; w < kConsumerWarps; ++w) s += b.red[w];
-  return s;
+// Gain vector of an RMSNorm to come.  Its turn comes once per timestep, by when the weight stream has pushed it out
+// of L2; a load issued after the grid barrier would add a trip to device memory to every phase boundary, so the
+// thread's first two 16-byte vectors are asked for a phase ahead and wait in registers (columns beyond
+// 2 * 512 * 8 are fetched late).
+struct Gain {
+  uint4 g[2];
+};
+
+// Pointer of the j-th RMSNorm gain of a timestep: attention norm of layer j / 2 (j even), FFN norm of layer j / 2
+// (j odd), final norm (j = 2 L).
+__device__ __forceinline__ const __nv_bfloat16 *gain_ptr(const Blk &b, int j) {
+  const KParams &p = *b.p;
+  if (2 * p.L + 1 <= kGainSlots) return s_gain_ptrs[j];
+  return j == 2 * p.L ? p.final_norm : ((j & 1) ? p.layers[j >> 1].ffn_norm : p.layers[j >> 1].attn_norm);
 }
+
+__device__ __forceinline__ void fetch_gain(const __nv_bfloat16 *gain, int C, Gain &gq) {
+  const int nv = C / 8;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int v = (int)threadIdx.x + i * kConsumerThreads;
+    if (v < nv) gq.g[i] = __ldg(reinterpret_cast<const uint4 *>(gain + (size_t)v * 8));
+  }
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); }
 
 __device__ __forceinline__ void load8(const float *src, float (&x)[8]) {
   const float4 a = __ldcg(reinterpret_cast<const float4 *>(src));
@@ -361,9 +553,11 @@ __device__ __forceinline__ void load8(const float *src, float (&x)[8]) {
   x[4] = c.x; x[5] = c.y; x[6] = c.z; x[7] = c.w;
 }
 
-// x = RMSNorm(h) * gain, each thread keeping its own column vectors
-__device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const __nv_bfloat16 *gain, int C,
-                                              float (&xr)[kMaxVec][8]) {
+// x = h * gain, each thread keeping its own column vectors; the factor 1 / rms(h) that completes RMSNorm(h) * gain
+// is common to all columns and is applied to the row sums (epilogue): the warps' sums of squares go to red[], which
+// the phase's first tile-end barrier makes visible, so no block-wide reduction stands between the grid barrier and
+// the first multiply.  red[] is next written a grid barrier later at the earliest.
+__device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const Gain &gq, int j, int C, float (&xr)[kMaxVec][8]) {
   const int nv = C / 8;
   float ss = 0.f;
 #pragma unroll
@@ -373,20 +567,24 @@ __device__ __forceinline__ void prologue_norm(Blk &b, const float *h, const __nv
       load8(h + (size_t)v * 8, xr[i]);
 #pragma unroll
       for (int e = 0; e < 8; ++e) ss = fmaf(xr[i][e], xr[i][e], ss);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xr[i][e] = 0.f;  // every vector is written: none outlives a phase
     }
   }
-  ss = block_sum(b, ss);
-  const float rs = rsqrtf(ss / (float)C + b.p->eps);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = ss;
 #pragma unroll
   for (int i = 0; i < kMaxVec; ++i) {
     const int v = (int)threadIdx.x + i * kConsumerThreads;
     if (v < nv) {
-      const uint4 g = *reinterpret_cast<const uint4 *>(gain + (size_t)v * 8);
+      const uint4 g = i < 2 ? gq.g[i] : __ldg(reinterpret_cast<const uint4 *>(gain_ptr(b, j) + (size_t)v * 8));
       const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        xr[i][2 * e] = xr[i][2 * e] * rs * __uint_as_float(gw[e] << 16);
-        xr[i][2 * e + 1] = xr[i][2 * e + 1] * rs * __uint_as_float(gw[e] & 0xffff0000u);
+        xr[i][2 * e] = xr[i][2 * e] * __uint_as_float(gw[e] << 16);
+        xr[i][2 * e + 1] = xr[i][2 * e + 1] * __uint_as_float(gw[e] & 0xffff0000u);
       }
     }
   }
@@ -397,7 +595,12 @@ __device__ __forceinline__ void prologue_plain(const float *src, int C, float (&
 #pragma unroll
   for (int i = 0; i < kMaxVec; ++i) {
     const int v = (int)threadIdx.x + i * kConsumerThreads;
-    if (v < nv) load8(src + (size_t)v * 8, xr[i]);
+    if (v < nv) {
+      load8(src + (size_t)v * 8, xr[i]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xr[i][e] = 0.f;  // every vector is written: none outlives a phase
+    }
   }
 }
 
@@ -416,23 +619,29 @@ __device__ __forceinline__ void prologue_attn(const KParams &p, int T, float (&x
     const int v = (int)threadIdx.x + i * kConsumerThreads;
     if (v < nv) {
       const int col = v * 8, head = col / p.hd, c = col - head * p.hd;
-      float M = -CUDART_INF_F;
-      for (int s = 0; s < ns; ++s) M = fmaxf(M, __ldcg(&p.oml[head * ns + s]).x);
-      float den = 0.f, acc[8];
+      // one pass with a running maximum, so that a split's (max, sum) and its partial output are asked for
+      // together: one trip to L2 after the grid barrier instead of two
+      float M = -CUDART_INF_F, den = 0.f, acc[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll 2
       for (int s = 0; s < ns; ++s) {
         const float2 ml = __ldcg(&p.oml[head * ns + s]);
-        const float w = __expf(ml.x - M);
-        den = fmaf(ml.y, w, den);
         float o[8];
         load8(p.opart + (size_t)(head * ns + s) * p.hd + c, o);
+        const float Mn = fmaxf(M, ml.x);
+        const float keep = M == -CUDART_INF_F ? 0.f : __expf(M - Mn), w = ml.x == -CUDART_INF_F ? 0.f : __expf(ml.x - Mn);
+        den = fmaf(den, keep, ml.y * w);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e] = fmaf(o[e], w, acc[e]);
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(acc[e], keep, o[e] * w);
+        M = Mn;
       }
       const float inv = 1.f / den;
 #pragma unroll
       for (int e = 0; e < 8; ++e) xr[i][e] = acc[e] * inv;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) xr[i][e] = 0.f;
     }
   }
 }
@@ -446,6 +655,27 @@ __device__ __forceinline__ float load_kv(const KParams &p, const void *cache, si
   return __ldcg(reinterpret_cast<const float *>(cache) + idx);
 }
 
+// Asks the cache rows that this block's attention items will read into L2 (all but the new position's, which this
+// phase writes).  They were last touched a timestep ago and the weight stream has pushed them out since: issued
+// at the start of the QKV phase, the requests travel with the weight stream, and the attention phase, which
+// stands between two grid barriers with the ring full, finds its rows in L2.
+__device__ __forceinline__ void prefetch_kv(const KParams &p, int layer, int pos) {
+  const int T = pos + 1, ns = attn_splits(p, T), items = p.H * ns;
+  const int esz = p.kv_bf16 ? 2 : 4;
+  const int lpr = (p.hd * esz + 127) >> 7;  // 128-byte lines per cache row of a head
+  for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    const int head = item / ns, sp = item - head * ns;
+    const int t0 = (int)((long long)T * sp / ns), t1 = min((int)((long long)T * (sp + 1) / ns), pos);
+    const int n = (t1 - t0) * lpr;
+    for (int i = threadIdx.x; i < n; i += kConsumerThreads) {
+      const int t = t0 + i / lpr, c = i - (i / lpr) * lpr;
+      const size_t off = (((size_t)layer * p.max_pos + t) * p.d + (size_t)head * p.hd) * esz + (size_t)c * 128;
+      prefetch_l2(reinterpret_cast<const uint8_t *>(p.kcache) + off);
+      prefetch_l2(reinterpret_cast<const uint8_t *>(p.vcache) + off);
+    }
+  }
+}
+
 // Fast path of the attention phase for a bf16 cache and head_dim 128 (a cache row of a head is 256 bytes):
 // half a warp takes one position with 16-byte loads, and each warp keeps eight positions in flight, so a
 // long context costs a few dependent memory round trips instead of one per position.  Each half-warp runs
@@ -455,8 +685,8 @@ __device__ void attention_phase_bf16_hd128(Blk &b, int layer, int pos) {
   const int T = pos + 1, ns = attn_splits(p, T), items = p.H * ns;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, l16 = lane & 15;
   const float scale = 1.f / sqrtf(128.f);
-  float *s_acc = b.part;                           // [warps][128]
-  float *s_m = b.part + kConsumerWarps * 256;      // [warps]
+  float *s_acc = scratch_base(p);                           // [warps][128]
+  float *s_m = scratch_base(p) + kConsumerWarps * 256;      // [warps]
   float *s_l = s_m + kConsumerWarps;               // [warps]
   const __nv_bfloat16 *kc = reinterpret_cast<const __nv_bfloat16 *>(p.kcache);
   const __nv_bfloat16 *vc = reinterpret_cast<const __nv_bfloat16 *>(p.vcache);
@@ -551,8 +781,8 @@ __device__ void attention_phase(Blk &b, int layer, int pos) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int epl = p.hd / 32;  // elements per lane, <= 8
   const float scale = 1.f / sqrtf((float)p.hd);
-  float *s_acc = b.part;                           // [warps][hd]
-  float *s_m = b.part + kConsumerWarps * 256;      // [warps]
+  float *s_acc = scratch_base(p);                           // [warps][hd]
+  float *s_m = scratch_base(p) + kConsumerWarps * 256;      // [warps]
   float *s_l = s_m + kConsumerWarps;               // [warps]
   for (int item = blockIdx.x; item < items; item += gridDim.x) {
     const int head = item / ns, sp = item - head * ns;
@@ -644,16 +874,28 @@ __device__ void sample_windows(const KParams &p, int it) {
 }
 
 // ---------------------------------------------------------------- consumer main loop
-template <bool kSampler>
+// kImgs > 0: QKV, attention output, gate / up and LM head also come in fragment order: a prologue leaves x
+// in shared memory as fragments (store_frags; the barrier after it orders the stores before the first instruction
+// that reads them) and consume_image multiplies.
+template <bool kSampler, int kImgs>
 __device__ void consumer_main(Blk &b) {
+  constexpr bool kImg = kImgs > 0;
   const KParams &p = *b.p;
   float xr[kMaxVec][8];
+  // Everything a phase needs besides the activations is asked for at least a phase ahead (the gains of the RMSNorms,
+  // the position's row of the rotary table, the cache rows of the attention items): after a grid barrier only the
+  // activation vector itself is fetched, one trip to L2.
+  Gain gq;
+  fetch_gain(gain_ptr(b, 0), p.d, gq);
   for (int it = 0; it < p.n_iters; ++it) {
     const int pos = p.pos0 + it;
+    const bool last = it == p.n_iters - 1;
+    const bool head = (kSampler ? p.mode != kModePrefill : p.mode == kModeDecode) || last;
+    if ((int)threadIdx.x < p.hd / 2) s_rope[threadIdx.x] = p.rope[(size_t)pos * (p.hd / 2) + threadIdx.x];
     if (blockIdx.x == 0) {
       if (kSampler && p.mode == kModeSample) {
         // the next token is drawn from the logits of the pass before (Section 4.5: a nucleus-sampled prefix)
-        const int tok = ns_sample(p.logits, p.V, p.ns_inv_temp, p.ns_p, p.ns_u[it], reinterpret_cast<uint8_t *>(b.part));
+        const int tok = ns_sample(p.logits, p.V, p.ns_inv_temp, p.ns_p, p.ns_u[it], reinterpret_cast<uint8_t *>(scratch_base(p)));
         if (threadIdx.x == 0) p.prefix[it] = tok;
         named_sync(1, kConsumerThreads);
       }
@@ -665,40 +907,65 @@ __device__ void consumer_main(Blk &b) {
       // barrier if the step before made the most probable draft end with it; every block then leaves, its producer
       // draining the copies in flight as when giving up, but without an error.
       if (threadIdx.x == 0) {
-        if (ld_relaxed(&p.st->stop)) *b.dead = 1;
-        *b.quit = *b.dead;
+        if (ld_relaxed(&p.st->stop)) s_dead = 1;
+        s_quit = s_dead;
       }
       named_sync(1, kConsumerThreads);
-      if (*b.quit) return;
+      if (s_quit) return;
     }
     for (int l = 0; l < p.L; ++l) {
-      const LayerW lw = p.layers[l];
       EpiArgs ea{l, pos, 0};
-      prologue_norm(b, p.h, lw.attn_norm, p.d, xr);
-      consume_matrix(b, 3 * p.d, p.d, 2, xr, kEpiQKV, ea);
+      prologue_norm(b, p.h, gq, 2 * l, p.d, xr);
+      prefetch_kv(p, l, pos);
+      if constexpr (kImg) {
+        store_frags(p, p.d, xr);
+        named_sync(1, kConsumerThreads);
+        consume_image(b, 3 * p.d, p.d, kEpiQKV, ea);
+      } else {
+        consume_matrix(b, 3 * p.d, p.d, 2, xr, kEpiQKV, ea);
+      }
       if (grid_barrier(b)) return;
       attention_phase(b, l, pos);
       if (grid_barrier(b)) return;
       prologue_attn(p, pos + 1, xr);
-      consume_matrix(b, p.d, p.d, 1, xr, kEpiAddH, ea);
+      fetch_gain(gain_ptr(b, 2 * l + 1), p.d, gq);
+      if constexpr (kImg) {
+        store_frags(p, p.d, xr);
+        named_sync(1, kConsumerThreads);
+        consume_image(b, p.d, p.d, kEpiAddH, ea);
+      } else {
+        consume_matrix(b, p.d, p.d, 1, xr, kEpiAddH, ea);
+      }
       if (grid_barrier(b)) return;
-      prologue_norm(b, p.h, lw.ffn_norm, p.d, xr);
-      consume_matrix(b, 2 * p.f, p.d, 2, xr, kEpiSwiGLU, ea);
+      prologue_norm(b, p.h, gq, 2 * l + 1, p.d, xr);
+      if constexpr (kImg) {
+        store_frags(p, p.d, xr);
+        named_sync(1, kConsumerThreads);
+        consume_image(b, 2 * p.f, p.d, kEpiSwiGLU, ea);
+      } else {
+        consume_matrix(b, 2 * p.f, p.d, 2, xr, kEpiSwiGLU, ea);
+      }
       if (grid_barrier(b)) return;
       prologue_plain(p.u, p.f, xr);
+      fetch_gain(gain_ptr(b, l + 1 < p.L || head ? 2 * l + 2 : 0), p.d, gq);
       ea.which = 1;
       consume_matrix(b, p.d, p.f, 1, xr, kEpiAddH, ea);
       if (grid_barrier(b)) return;
     }
-    const bool last = it == p.n_iters - 1;
-    const bool head = kSampler ? p.mode != kModePrefill : p.mode == kModeDecode;
-    if (head || last) {
+    if (head) {
       EpiArgs ea{0, pos, 0};
-      prologue_norm(b, p.h, p.final_norm, p.d, xr);
-      consume_matrix(b, p.V, p.d, 1, xr, kEpiLogits, ea);
+      prologue_norm(b, p.h, gq, 2 * p.L, p.d, xr);
+      if (!last) fetch_gain(gain_ptr(b, 0), p.d, gq);
+      if constexpr (kImg) {
+        store_frags(p, p.d, xr);
+        named_sync(1, kConsumerThreads);
+        consume_image(b, p.V, p.d, kEpiLogits, ea);
+      } else {
+        consume_matrix(b, p.V, p.d, 1, xr, kEpiLogits, ea);
+      }
       named_sync(1, kConsumerThreads);
       int r0, r1;
-      cta_rows(p.V, 1, r0, r1);
+      cta_rows(p.V, kImg ? kUnitRows : 1, r0, r1);
       if (threadIdx.x < 32) block_topk(p, r0, r1);
       if (grid_barrier(b)) return;
       if (blockIdx.x == 0 && (!kSampler || p.mode != kModeSample || last)) {
@@ -712,12 +979,8 @@ __device__ void consumer_main(Blk &b) {
   }
 }
 
-template <bool kSampler>
+template <bool kSampler, int kImgs>
 __device__ __forceinline__ void kernel_body(const KParams &p) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages];
-  __shared__ float s_red[64];
-  __shared__ int s_dead, s_quit;
   Blk b;
   b.p = &p;
   b.ring = smem;
@@ -725,6 +988,11 @@ __device__ __forceinline__ void kernel_body(const KParams &p) {
   b.full = s_full;
   b.empty = s_empty;
   b.red = s_red;
+  b.rope_s = s_rope;
+  b.gain_ptrs = s_gain_ptrs;
+  if (p.mode != kModeScoreOnly && p.mode != kModeNucleusOnly && 2 * p.L + 1 <= kGainSlots)
+    for (int j = threadIdx.x; j <= 2 * p.L; j += kThreads)
+      s_gain_ptrs[j] = j == 2 * p.L ? p.final_norm : ((j & 1) ? p.layers[j >> 1].ffn_norm : p.layers[j >> 1].attn_norm);
   b.dead = &s_dead;
   b.quit = &s_quit;
   b.bar_target = 0;
@@ -746,44 +1014,50 @@ __device__ __forceinline__ void kernel_body(const KParams &p) {
   }
   if (kSampler && p.mode == kModeNucleusOnly) {
     if (blockIdx.x == 0 && threadIdx.x < kConsumerThreads) {
-      const int tok = ns_sample(p.logits, p.V, p.ns_inv_temp, p.ns_p, p.ns_u[0], reinterpret_cast<uint8_t *>(b.part));
+      const int tok = ns_sample(p.logits, p.V, p.ns_inv_temp, p.ns_p, p.ns_u[0], reinterpret_cast<uint8_t *>(scratch_base(p)));
       if (threadIdx.x == 0) p.st->cand_tok[0] = tok;
     }
     return;
   }
   if (threadIdx.x >= kConsumerThreads) {
-    if (threadIdx.x == kConsumerThreads) producer_main<kSampler>(b);
+    if (threadIdx.x == kConsumerThreads) producer_main<kSampler, kImgs>(b);
   } else {
-    consumer_main<kSampler>(b);
+    consumer_main<kSampler, kImgs>(b);
   }
   __syncthreads();
 }
 
 // The decoding kernel, and its twin that also carries the nucleus sampler (kModeSample, kModeNucleusOnly): two
 // entry points so that the sampler's code does not weigh on the register allocation of the decode loop.
-__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) { kernel_body<false>(p); }
-__global__ void __launch_bounds__(kThreads, 1) spd_sample_kernel(const __grid_constant__ KParams p) { kernel_body<true>(p); }
+__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) { kernel_body<false, 0>(p); }
+__global__ void __launch_bounds__(kThreads, 1) spd_sample_kernel(const __grid_constant__ KParams p) { kernel_body<true, 0>(p); }
+// The decoding kernel for weights that also come in fragment order: QKV, attention output, gate / up and LM head
+// products on the tensor cores.  The down projection stays with the float32 multiply loop: its rows are long, so whole
+// units of them divide unevenly among the blocks and their fragments of x would take a third of the ring's memory
+// (measured: 2.96 ms per 7B timestep with it on the tensor cores too, against 2.64 ms).
+__global__ void __launch_bounds__(kThreads, 1) spd_decode_img_kernel(const __grid_constant__ KParams p) { kernel_body<false, 1>(p); }
 
 }  // namespace spd
 
 // Host-side launcher used by the API file.
-static const void *kernel_for(int mode) {
-  return mode == spd::kModeSample || mode == spd::kModeNucleusOnly ? reinterpret_cast<const void *>(&spd::spd_sample_kernel)
-                                                                  : reinterpret_cast<const void *>(&spd::spd_decode_kernel);
+static const void *kernel_for(int mode, int img) {
+  if (mode == spd::kModeSample || mode == spd::kModeNucleusOnly) return reinterpret_cast<const void *>(&spd::spd_sample_kernel);
+  return img ? reinterpret_cast<const void *>(&spd::spd_decode_img_kernel) : reinterpret_cast<const void *>(&spd::spd_decode_kernel);
 }
 
 extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size_t dyn_smem, cudaStream_t stream) {
   void *args[] = {const_cast<spd::KParams *>(p)};
-  return cudaLaunchCooperativeKernel(kernel_for(p->mode), dim3(grid), dim3(spd::kThreads), args, dyn_smem, stream);
+  return cudaLaunchCooperativeKernel(kernel_for(p->mode, p->lm_head_img != nullptr), dim3(grid), dim3(spd::kThreads), args, dyn_smem, stream);
 }
 
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm) {
   int least = 1 << 30;
-  for (int mode : {(int)spd::kModeDecode, (int)spd::kModeSample}) {
-    cudaError_t e = cudaFuncSetAttribute(kernel_for(mode), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
+  const void *kernels[3] = {kernel_for(spd::kModeDecode, 0), kernel_for(spd::kModeDecode, 1), kernel_for(spd::kModeSample, 0)};
+  for (const void *kernel : kernels) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
     if (e != cudaSuccess) return e;
     int n = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel_for(mode), spd::kThreads, dyn_smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, spd::kThreads, dyn_smem);
     if (e != cudaSuccess) return e;
     if (n < least) least = n;
   }
@@ -905,4 +1179,30 @@ extern "C" int spd_score_static(const spd_config *cfg, const spd_ngram_table *ta
   if (out_score)
     for (int q = 0; q < k * k; ++q) out_score[q] = back.score[q];
   return SPD_OK;
+}
+
+// ---------------------------------------------------------------- fragment order
+// spd_pack_image (see include/spd.h): every block of 8 rows x 32 columns of a row-major bf16 matrix becomes 32
+// vectors of 16 bytes, vector (g, t) = row g's column pairs 2t | 2t+8 | 2t+16 | 2t+24 of the block: the weight
+// fragments of two m16n8k16 instructions for lane 4 g + t.  Units of 8 rows follow one another, each with its column
+// blocks in order, so a unit is one contiguous run of cols * 16 bytes.
+namespace spd {
+__global__ void spd_pack_image_kernel(const uint32_t *w, uint4 *out, int rows, int cols) {
+  const size_t n = (size_t)rows * cols / 8;  // 16-byte vectors
+  const int pairs = cols / 32;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += (size_t)gridDim.x * blockDim.x) {
+    const int lane = (int)(idx % (4 * kUnitRows));
+    const size_t blk = idx / (4 * kUnitRows);
+    const int pr = (int)(blk % pairs);
+    const size_t unit = blk / pairs;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t *src = w + ((unit * kUnitRows + g) * (size_t)cols + (size_t)pr * 32) / 2 + t;
+    out[idx] = make_uint4(src[0], src[4], src[8], src[12]);
+  }
+}
+}  // namespace spd
+
+extern "C" cudaError_t spd_internal_pack_image(const void *w, void *out, int rows, int cols, cudaStream_t stream) {
+  spd::spd_pack_image_kernel<<<1184, 256, 0, stream>>>(static_cast<const uint32_t *>(w), static_cast<uint4 *>(out), rows, cols);
+  return cudaGetLastError();
 }

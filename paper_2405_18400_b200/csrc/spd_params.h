@@ -20,11 +20,16 @@ constexpr int kMaxVec = 4;          // 16-byte column vectors per thread: column
 constexpr int kMaxSplit = 8;        // attention splits per head
 constexpr int kTensorMapBytes = 128; // size of one tensor map object (CUtensorMap)
 constexpr int kPfTokens = 16;       // prefix tokens one prefill launch takes
+constexpr int kUnitRows = 8;        // rows of a unit of a matrix in fragment order (the granularity of the blocks' shares; 4 was
+                                    // measured too: the shares come out more even, but a 7B timestep took 4.16 ms against 2.65 ms)
+constexpr int kScratchBytes = 20480; // per-block scratch after the decode kernel's ring: row partials / attention merge / tail
 
 enum Mode { kModePrefill = 0, kModeDecode = 1, kModeScoreOnly = 2, kModeSample = 3, kModeNucleusOnly = 4 };
 
 struct LayerW {
   const __nv_bfloat16 *attn_norm, *wqkv, *wo, *ffn_norm, *wgate_up, *wdown;
+  // the same matrices in the decode kernel's fragment order (spd_pack_image), or null
+  const __nv_bfloat16 *wqkv_img, *wo_img, *wgate_up_img;
 };
 
 struct TableDev {
@@ -100,6 +105,7 @@ struct KParams {
   float *pf_ss;              // [grid][kPfTokens] per block: sums of squares of the residual values it produced
   int32_t pf_stall;          // prefill kernel, test hook: block 0 withholds its arrival at the grid barriers
   int32_t eos_id;            // stop token (-1: none): decoding ends with the step in which the most probable draft emits it
+  const __nv_bfloat16 *lm_head_img;  // the LM head in fragment order, or null
 };
 
 }  // namespace spd

@@ -26,6 +26,8 @@ struct Blk {
   unsigned int bar_target;
   // consumer ring cursor
   uint32_t c_stage, c_phase;
+  float2 *rope_s;    // decode kernel: the current position's row of the rotary table
+  const __nv_bfloat16 *const *gain_ptrs;  // decode kernel: the RMSNorm gains' pointers in the order a timestep uses them
 };
 
 __device__ __forceinline__ void give_up(Blk &b, int code, int info) {

@@ -11,10 +11,12 @@ LOGIT_TOL = 2e-2      # max-abs logit tolerance (bf16 weights, fp32 accumulation
 GAMMA_TOL = 1e-4
 
 
-def make_pair(shape, weights, tables, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype="bf16", device="cuda:0"):
+def make_pair(shape, weights, tables, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype="bf16", device="cuda:0",
+              images=True):
+    """images=False: no fragment-order weight images, so the decode timesteps run the float32 multiply loop."""
     import paper_2405_18400_b200 as P
 
-    packed = P.pack_weights(weights, device)
+    packed = P.pack_weights(weights, device, images=images)
     dtabs = P.build_ngram_tables(tables, device)
     ctx = P.SpdContext(shape, packed, dtabs, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype)
     cfg = so.make_config(shape, k, orders, lam, alpha, tau, delta, max_pos, kv_dtype)
@@ -22,11 +24,11 @@ def make_pair(shape, weights, tables, k, orders, lam, alpha, tau, delta, max_pos
     return ctx, orc
 
 
-def make_tiny_pair(tiny_inputs, k=None, kv_dtype="bf16", max_pos=None, tables=None, alpha=None, delta=None):
+def make_tiny_pair(tiny_inputs, k=None, kv_dtype="bf16", max_pos=None, tables=None, alpha=None, delta=None, images=True):
     wl, weights, tabs, prefix = tiny_inputs
     return make_pair(wl.shape, weights, tabs if tables is None else tables, wl.k if k is None else k, wl.orders,
                      wl.lambdas(), wl.alpha if alpha is None else alpha, wl.tau, wl.delta if delta is None else delta,
-                     wl.max_pos if max_pos is None else max_pos, kv_dtype)
+                     wl.max_pos if max_pos is None else max_pos, kv_dtype, images=images)
 
 
 def top_gap(values, k):

@@ -301,9 +301,10 @@ def test_call_order_and_range_errors(tiny_inputs):
     ctx.close()
 
 
-def test_ring_settings_do_not_change_results(tiny_inputs):
+@pytest.mark.parametrize("images", [False, True])
+def test_ring_settings_do_not_change_results(tiny_inputs, images):
     wl, weights, tables, prefix = tiny_inputs
-    ctx, _ = make_tiny_pair(tiny_inputs)
+    ctx, _ = make_tiny_pair(tiny_inputs, images=images)
     ctx.spd_prefill(prefix)
     base, lp0, _ = ctx.spd_generate(5, 6)
     z0 = ctx.spd_debug_read("LOGITS")
@@ -312,11 +313,51 @@ def test_ring_settings_do_not_change_results(tiny_inputs):
         ctx.spd_prefill(prefix)
         toks, lp, _ = ctx.spd_generate(5, 6)
         assert np.array_equal(toks, base)
-        assert np.abs(ctx.spd_debug_read("LOGITS") - z0).max() < 1e-4
+        # with fragment-order images the stage size decides which warp adds which products of a row: the sums differ
+        # in their last bits, and five timesteps carry that forward
+        assert np.abs(ctx.spd_debug_read("LOGITS") - z0).max() < (1e-3 if images else 1e-4)
     import paper_2405_18400_b200 as P
     with pytest.raises(P.SpdError):
         ctx.spd_set_ring(1024, 4)              # a 688-column row (1376 bytes) does not fit
     ctx.close()
+
+
+def test_fragment_order_image_layout():
+    """spd_pack_image against its definition: vector 4 g + t of a block of 8 rows x 32 columns holds row g's column
+    pairs 2t, 2t+8, 2t+16, 2t+24; blocks of a unit in column order, units in row order."""
+    import torch
+    import paper_2405_18400_b200 as P
+    from paper_2405_18400_b200.binding import _image
+
+    rows, cols = 24, 96
+    w = torch.arange(rows * cols, dtype=torch.int16, device="cuda:0").view(torch.bfloat16).reshape(rows, cols)
+    img = _image(w)
+    torch.cuda.synchronize()
+    got = img.view(torch.int16).cpu().numpy().reshape(-1)
+    src = np.arange(rows * cols, dtype=np.int16).reshape(rows, cols)
+    want = np.empty(rows * cols, np.int16)
+    at = 0
+    for unit in range(rows // 8):
+        for blk in range(cols // 32):
+            for lane in range(32):
+                g, t = lane // 4, lane % 4
+                for q in range(4):
+                    c = blk * 32 + 2 * t + 8 * q
+                    want[at: at + 2] = src[unit * 8 + g, c: c + 2]
+                    at += 2
+    assert np.array_equal(got, want)
+    assert P.load_library().spd_pack_image(w.data_ptr(), 20, 96, img.data_ptr(), None) == -1    # rows must be a multiple of 8
+    assert P.load_library().spd_pack_image(w.data_ptr(), 24, 80, img.data_ptr(), None) == -1    # columns a multiple of 32
+
+
+def test_steps_without_images_match_oracle(tiny_inputs):
+    """The float32 multiply loop (contexts whose weights come without fragment-order images) against the oracle."""
+    ctx, orc = make_tiny_pair(tiny_inputs, images=False)
+    wl, weights, tables, prefix = tiny_inputs
+    compare_first_step(ctx, orc, prefix)
+    for _ in range(4):
+        compare_step(ctx, orc)
+    ctx.close(); orc.close()
 
 
 def test_malformed_table_is_reported_not_hung(tiny_inputs):
