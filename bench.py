@@ -29,9 +29,27 @@ import torch
 
 import spd_inputs as si
 
-# dram bytes (read + write) / algorithmic bytes measured by ncu on a 4-layer case of the same kernel; traffic
-# grows in proportion to the layers streamed.  None whenever the kernel has changed since the counters were taken.
-TRAFFIC_RATIO = None
+# dram bytes (read + write) / algorithmic bytes measured by ncu on a 4-layer case of the decode kernel; traffic
+# grows in proportion to the layers streamed.  The ratio stands only for the kernel sources it was taken with:
+# `traffic` is null once any of them has changed.
+TRAFFIC = {"ratio": 1.002, "sources_sha256": "4c43125b4268b3df2f9cea2b4a4fac83e43e33559919a04e4475470bea42deb5"}
+KERNEL_SOURCES = ("spd_kernel.cu", "spd_params.h", "spd_ptx.cuh", "spd_score.cuh", "spd_tail.cuh", "spd_nucleus.cuh", "spd_hash.h")
+
+
+def kernel_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2405_18400_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def traffic_ratio():
+    try:
+        return TRAFFIC["ratio"] if TRAFFIC["ratio"] and kernel_sources_sha256() == TRAFFIC["sources_sha256"] else None
+    except OSError:
+        return None
 
 METRIC = "k-draft tokens/s"
 UNIT = "tokens/s"
@@ -392,7 +410,8 @@ def run_ours(args, wl):
         "data": "synthetic",
         "config": config_of(wl, k, world, reps),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC_RATIO * bytes_step * K if TRAFFIC_RATIO else None, "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_decode_kernel"},
+                     "traffic": traffic_ratio() * bytes_step * K if traffic_ratio() else None, "peak_kind": peak_kind,
+                     "bytes_per_step": bytes_step, "kernel": "spd_decode_img_kernel" if "lm_head_img" in packed else "spd_decode_kernel"},
         "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
     }
     if kpass:

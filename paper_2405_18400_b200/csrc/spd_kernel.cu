@@ -118,8 +118,14 @@ __device__ __forceinline__ void produce_matrix(Blk &b, Producer &pr, const __nv_
 }
 
 constexpr int kPairBytes = kUnitRows * 64;  // a unit's share of a pair of 16-column blocks: 4 lanes of 16 bytes per row
-// Bytes of a fragment-order unit that one ring stage takes: whole pairs of 16-column blocks.
-__device__ __forceinline__ uint32_t img_chunk(const KParams &p) { return (uint32_t)p.stage_bytes / kPairBytes * kPairBytes; }
+// Bytes of a fragment-order unit of C columns that one ring stage takes: the unit in the fewest equal parts that fit
+// a stage, in whole pairs of 16-column blocks (the last part may be shorter).
+__device__ __forceinline__ uint32_t img_chunk(const KParams &p, int C) {
+  const uint32_t unit = (uint32_t)C * 2u * kUnitRows, cap = (uint32_t)p.stage_bytes / kPairBytes * kPairBytes;
+  const uint32_t parts = (unit + cap - 1) / cap;
+  const uint32_t pairs = ((uint32_t)C / 32 + parts - 1) / parts;
+  return pairs * kPairBytes;
+}
 
 // A matrix in fragment order (spd_pack_image): the units of this block, each unit in stages of img_chunk bytes and a
 // shorter last one.
@@ -130,8 +136,9 @@ __device__ __forceinline__ void produce_image(Blk &b, Producer &pr, const __nv_b
   const uint32_t unit_bytes = (uint32_t)C * 2u * kUnitRows;
   for (int r = r0; r < r1; r += kUnitRows) {
     const uint8_t *src = reinterpret_cast<const uint8_t *>(img) + (size_t)(r / kUnitRows) * unit_bytes;
-    for (uint32_t off = 0; off < unit_bytes; off += img_chunk(p)) {
-      const uint32_t bytes = unit_bytes - off < img_chunk(p) ? unit_bytes - off : img_chunk(p);
+    const uint32_t chunk = img_chunk(p, C);
+    for (uint32_t off = 0; off < unit_bytes; off += chunk) {
+      const uint32_t bytes = unit_bytes - off < chunk ? unit_bytes - off : chunk;
       wait_mbar(b, &s_empty[pr.stage], pr.phase ^ 1u, 200);
       if (s_dead) return;
       mbar_expect_tx(&s_full[pr.stage], bytes);
@@ -476,7 +483,7 @@ __device__ __forceinline__ void consume_image(Blk &b, int R, int C, int kind, co
     float *part = scratch_base(p) + (size_t)buf * kTile * kConsumerWarps;
     for (int r = t0; r < t1; r += kUnitRows) {
       float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
-      const int per_stage = (int)(img_chunk(p) / kPairBytes);
+      const int per_stage = (int)(img_chunk(p, C) / kPairBytes);
       for (int pr0 = 0; pr0 < n_pairs; pr0 += per_stage) {  // one stage
         wait_mbar(b, &s_full[b.c_stage], b.c_phase, 300);
         const uint8_t *stage = smem + (size_t)b.c_stage * p.stage_bytes;
