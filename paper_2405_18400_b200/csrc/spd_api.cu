@@ -18,7 +18,8 @@ extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm);
 extern "C" cudaError_t spd_internal_prefill_launch(const spd::KParams *p, int grid, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_pack_image(const void *w, void *out, int rows, int cols, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd::KParams *kps, int n, int V, const __nv_bfloat16 *final_norm,
-                                               float *y_logits, cudaStream_t s, int *launches);
+                                               float *y_logits, size_t y_floats, size_t y_logits_floats, float *ss, int sm_count,
+                                               cudaStream_t s, int *launches);
 
 namespace {
 
@@ -43,7 +44,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
       trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, tc_tmaps, tc_h, tc_q, tc_y, tc_x, bt_kp, bt_y,
-      total;
+      bt_ss, total;
 };
 
 // Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 64 tokens send
@@ -116,7 +117,7 @@ Layout make_layout(const spd_config &c, int grid) {
   L.pf_xu = take(frag_bytes(c.d_ffn));
   const size_t tcr = (size_t)tc_rows(c);
   const size_t wide = (size_t)(3 * c.d_model > 2 * c.d_ffn ? 3 * c.d_model : 2 * c.d_ffn);
-  L.tc_tmaps = take(2 * sizeof(CUtensorMap));
+  L.tc_tmaps = take(8 * sizeof(CUtensorMap));  // term buffer as [..][d] and [..][f] in boxes of 128, 16, 32 and 64 rows
   L.tc_h = take(tcr * c.d_model * 4);
   L.tc_q = take(tcr * c.d_model * 4);
   L.tc_y = take(tcr * wide * 4);
@@ -124,6 +125,7 @@ Layout make_layout(const spd_config &c, int grid) {
   // batched timesteps led by this context: the requests' parameters and their rows of logits
   L.bt_kp = take(tcr ? (size_t)spd::kTcTile * sizeof(spd::KParams) : 0);
   L.bt_y = take(tcr ? (size_t)spd::kTcTile * c.vocab * 4 : 0);
+  L.bt_ss = take(tcr ? (size_t)spd::kTcTile * 32 * 4 : 0);  // per request and 512-column chunk: sums of squares of the residual row
   L.total = off;
   return L;
 }
@@ -145,11 +147,11 @@ bool weight_map(TensorMapEncode encode, const void *w, int rows, int cols, CUten
 }
 
 // Tensor map of the term buffer of the long-prefix path seen as a bf16 matrix [rows][cols]: boxes of 64 columns x
-// 128 rows, 128-byte swizzle, zeros outside.
-bool term_map(TensorMapEncode encode, const void *x, int rows, int cols, CUtensorMap *out) {
+// box_rows rows, 128-byte swizzle, zeros outside.
+bool term_map(TensorMapEncode encode, const void *x, int rows, int cols, int box_rows, CUtensorMap *out) {
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)spd::kTcTile};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t step[2] = {1, 1};
   return encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(x), dims, strides, box, step,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -490,7 +492,7 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
   }
   // tensor maps of the matrices in the order the prefill kernel walks them
   std::vector<CUtensorMap> tmaps((size_t)4 * cfg->n_layers + 1);
-  CUtensorMap xmaps[2];
+  CUtensorMap xmaps[8];
   std::memset(xmaps, 0, sizeof xmaps);
   ctx->layers_host = layers;
   {
@@ -508,7 +510,11 @@ int spd_create(const spd_config *cfg, const spd_weights *w, const spd_ngram_tabl
     }
     ok = ok && weight_map(encode, w->lm_head, cfg->vocab, d, &tmaps[(size_t)4 * cfg->n_layers]);
     if (ok && ctx->tc_rows > 0)
-      ok = term_map(encode, ws + lay.tc_x, 3 * ctx->tc_rows, d, &xmaps[0]) && term_map(encode, ws + lay.tc_x, 3 * ctx->tc_rows, f, &xmaps[1]);
+      for (int i = 0; i < 4 && ok; ++i) {
+        const int box_rows = i == 0 ? spd::kTcTile : 8 << i;  // 128, then 16, 32, 64 for the products of a small batch
+        ok = term_map(encode, ws + lay.tc_x, 3 * ctx->tc_rows, d, box_rows, &xmaps[2 * i]) &&
+             term_map(encode, ws + lay.tc_x, 3 * ctx->tc_rows, f, box_rows, &xmaps[2 * i + 1]);
+      }
     if (!ok) return fail(SPD_EINVAL);
   }
   cudaStream_t s = ctx->stream;
@@ -793,8 +799,11 @@ int batch_enqueue(spd_ctx *const *ctxs, int32_t n, int32_t n_steps) {
   const spd::TcJob job = tc_job(lead);
   for (int s = 0; s < n_steps; ++s) {
     int launched = 0;
+    const int wide = 3 * c0.d_model > 2 * c0.d_ffn ? 3 * c0.d_model : 2 * c0.d_ffn;
     const cudaError_t e = spd_internal_batch_step(&job, dkp, n, c0.vocab, lead->kp.final_norm,
-                                                  reinterpret_cast<float *>(lead->ws + lead->lay.bt_y), lead->stream, &launched);
+                                                  reinterpret_cast<float *>(lead->ws + lead->lay.bt_y), (size_t)lead->tc_rows * wide,
+                                                  (size_t)spd::kTcTile * c0.vocab, reinterpret_cast<float *>(lead->ws + lead->lay.bt_ss),
+                                                  lead->grid, lead->stream, &launched);
     lead->launches += launched;
     if (e != cudaSuccess) return cuda_fail(e, "batched timestep");
   }

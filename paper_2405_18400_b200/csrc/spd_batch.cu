@@ -32,6 +32,14 @@ __device__ __forceinline__ void bt_put3(uint16_t *X, size_t term_stride, size_t 
   X[at + 2 * term_stride] = (uint16_t)(__float_as_uint(r2) >> 16);
 }
 
+// A batch has few token rows, so the row-wise work between the products is spread over the columns: a block takes
+// kBtCols columns of one request's row.  RMSNorm's factor 1 / rms(h) is common to a row's columns and moves behind
+// the product (as in the single-request kernel): the kernels that write a residual row h store h * gain as the next
+// product's terms and the sum of squares of their columns (ss[request][chunk]); the kernels that read that product
+// multiply its rows by rsqrt(sum of the row's chunks / d + eps).
+constexpr int kBtCols = 512;      // columns per block: two per thread
+constexpr int kBtMaxChunks = 32;  // d_model <= 16384
+
 __device__ __forceinline__ float bt_block_sum(float v, float *scratch) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -40,55 +48,114 @@ __device__ __forceinline__ float bt_block_sum(float v, float *scratch) {
   float s = 0.f;
 #pragma unroll
   for (int w = 0; w < 8; ++w) s += scratch[w];
-  __syncthreads();
   return s;
+}
+
+__device__ __forceinline__ float bt_rs(const float *ss, int request, int d, float eps) {
+  const int nch = (d + kBtCols - 1) / kBtCols;
+  float s = 0.f;
+  for (int c = 0; c < nch; ++c) s += ss[request * kBtMaxChunks + c];
+  return rsqrtf(s / (float)d + eps);
 }
 
 // Position of the request's next input: the prefix's m positions, then one per superposed input so far.  The
 // device copy of a request's parameters keeps m - 1 in pos0; n_gen counts the tokens generated per draft.
 __device__ __forceinline__ int bt_pos(const KParams &p) { return p.pos0 + p.st->n_gen; }
 
-// One request per block: the superposed input of Eq. 3, h = sum_i gamma_i E[last token of draft i], stored as the
-// request's residual row, and its RMSNorm with the first layer's gain as three bf16 terms for the first product.
+// grid (requests, column chunks): the superposed input of Eq. 3, h = sum_i gamma_i E[last token of draft i], stored as
+// the request's residual row; h * gain of the first layer's norm as three bf16 terms; the chunk's sum of squares.
 __global__ void __launch_bounds__(256) spd_batch_input_kernel(const KParams *kps, float *h, const __nv_bfloat16 *gain, uint16_t *X,
-                                                              size_t term_stride, int d, float eps) {
+                                                              size_t term_stride, int d, float *ss) {
   __shared__ float scratch[8];
   const KParams &p = kps[blockIdx.x];
   const State *st = p.st;
-  float *hr = h + (size_t)blockIdx.x * d;
-  float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += 256) {
-    float acc = 0.f;
-    for (int i = 0; i < p.k; ++i) acc = fmaf(st->gamma[i], __bfloat162float(p.tok_emb[(size_t)st->win[i][kWin - 1] * d + c]), acc);
-    hr[c] = acc;
-    ss = fmaf(acc, acc, ss);
-  }
-  const float rs = rsqrtf(bt_block_sum(ss, scratch) / (float)d + eps);
-  for (int c = threadIdx.x; c < d; c += 256) bt_put3(X, term_stride, (size_t)blockIdx.x * d + c, hr[c] * rs * __bfloat162float(gain[c]));
-}
-
-// One request per block: rotary embedding of q and k (adjacent pairs) at the request's own position, q to Q, k and
-// v into the request's own cache.  Y row = [q | k | v].
-__global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *Y, float *Q, const KParams *kps, int d, int hd, int layer) {
-  const KParams &p = kps[blockIdx.x];
-  const int t = blockIdx.x, pos = bt_pos(p);
-  const float *yr = Y + (size_t)t * 3 * d;
-  const size_t crow = ((size_t)layer * p.max_pos + pos) * d;
-  for (int i = threadIdx.x; i < d / 2; i += 256) {
-    const float2 cs = p.rope[(size_t)pos * (hd / 2) + (i % (hd / 2))];
-    const float qe = yr[2 * i], qo = yr[2 * i + 1], ke = yr[d + 2 * i], ko = yr[d + 2 * i + 1];
-    Q[(size_t)t * d + 2 * i] = qe * cs.x - qo * cs.y;
-    Q[(size_t)t * d + 2 * i + 1] = qe * cs.y + qo * cs.x;
-    const float k0 = ke * cs.x - ko * cs.y, k1 = ke * cs.y + ko * cs.x;
-    const float v0 = yr[2 * d + 2 * i], v1 = yr[2 * d + 2 * i + 1];
-    if (p.kv_bf16) {
-      reinterpret_cast<__nv_bfloat162 *>(p.kcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(k0), __float2bfloat16_rn(k1));
-      reinterpret_cast<__nv_bfloat162 *>(p.vcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(v0), __float2bfloat16_rn(v1));
-    } else {
-      reinterpret_cast<float2 *>(p.kcache)[(crow >> 1) + i] = make_float2(k0, k1);
-      reinterpret_cast<float2 *>(p.vcache)[(crow >> 1) + i] = make_float2(v0, v1);
+  float sq = 0.f;
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int c = blockIdx.y * kBtCols + e * 256 + threadIdx.x;
+    if (c < d) {
+      float acc = 0.f;
+      for (int i = 0; i < p.k; ++i) acc = fmaf(st->gamma[i], __bfloat162float(p.tok_emb[(size_t)st->win[i][kWin - 1] * d + c]), acc);
+      h[(size_t)blockIdx.x * d + c] = acc;
+      sq = fmaf(acc, acc, sq);
+      bt_put3(X, term_stride, (size_t)blockIdx.x * d + c, acc * __bfloat162float(gain[c]));
     }
   }
+  sq = bt_block_sum(sq, scratch);
+  if (threadIdx.x == 0) ss[blockIdx.x * kBtMaxChunks + blockIdx.y] = sq;
+}
+
+// grid (requests, column chunks): residual add h += y (y = the sum of nz partial products zs floats apart), h * gain
+// of the next norm as terms, the chunk's sum of squares.
+__global__ void __launch_bounds__(256) spd_batch_resid_kernel(float *h, const float *y, int nz, size_t zs, const __nv_bfloat16 *gain, uint16_t *X,
+                                                              size_t term_stride, int d, float *ss) {
+  __shared__ float scratch[8];
+  float sq = 0.f;
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int c = blockIdx.y * kBtCols + e * 256 + threadIdx.x;
+    if (c < d) {
+      const size_t at = (size_t)blockIdx.x * d + c;
+      float v = h[at];
+      for (int z = 0; z < nz; ++z) v += y[z * zs + at];
+      h[at] = v;
+      sq = fmaf(v, v, sq);
+      bt_put3(X, term_stride, at, v * __bfloat162float(gain[c]));
+    }
+  }
+  sq = bt_block_sum(sq, scratch);
+  if (threadIdx.x == 0) ss[blockIdx.x * kBtMaxChunks + blockIdx.y] = sq;
+}
+
+// grid (requests, chunks of 256 column pairs): the QKV product's row times 1 / rms, rotary embedding of q and k
+// (adjacent pairs) at the request's own position, q to Q, k and v into the request's own cache.  Y row = [q | k | v].
+__global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, float *Q,
+                                                                   const KParams *kps, int d, int hd, int layer) {
+  const KParams &p = kps[blockIdx.x];
+  const int t = blockIdx.x, pos = bt_pos(p);
+  const int i = blockIdx.y * 256 + threadIdx.x;  // column pair
+  if (i >= d / 2) return;
+  const float rs = bt_rs(ss, t, d, eps);
+  const float *yr = Y + (size_t)t * 3 * d;
+  const size_t crow = ((size_t)layer * p.max_pos + pos) * d;
+  const float2 cs = p.rope[(size_t)pos * (hd / 2) + (i % (hd / 2))];
+  float2 qq = make_float2(0.f, 0.f), kk = qq, vv = qq;
+  for (int z = 0; z < nz; ++z) {  // the product's partial sums over column ranges, in order
+    const float *yz = yr + z * zs;
+    qq.x += yz[2 * i]; qq.y += yz[2 * i + 1];
+    kk.x += yz[d + 2 * i]; kk.y += yz[d + 2 * i + 1];
+    vv.x += yz[2 * d + 2 * i]; vv.y += yz[2 * d + 2 * i + 1];
+  }
+  const float qe = qq.x * rs, qo = qq.y * rs, ke = kk.x * rs, ko = kk.y * rs;
+  Q[(size_t)t * d + 2 * i] = qe * cs.x - qo * cs.y;
+  Q[(size_t)t * d + 2 * i + 1] = qe * cs.y + qo * cs.x;
+  const float k0 = ke * cs.x - ko * cs.y, k1 = ke * cs.y + ko * cs.x;
+  const float v0 = vv.x * rs, v1 = vv.y * rs;
+  if (p.kv_bf16) {
+    reinterpret_cast<__nv_bfloat162 *>(p.kcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(k0), __float2bfloat16_rn(k1));
+    reinterpret_cast<__nv_bfloat162 *>(p.vcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(v0), __float2bfloat16_rn(v1));
+  } else {
+    reinterpret_cast<float2 *>(p.kcache)[(crow >> 1) + i] = make_float2(k0, k1);
+    reinterpret_cast<float2 *>(p.vcache)[(crow >> 1) + i] = make_float2(v0, v1);
+  }
+}
+
+// grid (requests, chunks of 256 rows of the FFN): u = SiLU(gate) * up from the gate / up product's row times 1 / rms
+// (Y row = [gate_0, up_0, gate_1, up_1, ...]), as three bf16 terms.
+__global__ void __launch_bounds__(256) spd_batch_swiglu_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, int d, uint16_t *X,
+                                                               size_t term_stride, int f) {
+  const int t = blockIdx.x, j = blockIdx.y * 256 + threadIdx.x;
+  if (j >= f) return;
+  const float rs = bt_rs(ss, t, d, eps);
+  const float2 *yr = reinterpret_cast<const float2 *>(Y + (size_t)t * 2 * f);
+  float2 gu = make_float2(0.f, 0.f);
+  for (int z = 0; z < nz; ++z) {
+    const float2 more = yr[z * (zs / 2) + j];
+    gu.x += more.x;
+    gu.y += more.y;
+  }
+  const float g = gu.x * rs, up = gu.y * rs;
+  bt_put3(X, term_stride, (size_t)t * f + j, g / (1.f + __expf(-g)) * up);
 }
 
 // One (request, head) per block of four warps: softmax attention of the request's query over its own cache, a warp
@@ -160,31 +227,32 @@ __global__ void __launch_bounds__(128) spd_batch_attn_kernel(const float *Q, con
   }
 }
 
-// One request per block (512 threads): the request's row of logits goes to its own buffer; warp 0 ranks the whole
-// vocabulary (KeepTopK with log-probabilities under temperature tau, Algorithm 1); then Eq. 5-7, Eq. 2 and Eq. 4 on
-// the request's own draft state, as block 0 of the single-request kernel does.
-__global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const KParams *kps, const float *Y, int V) {
+// One request per block (512 threads): the request's row of logits (the LM head's partial products added, times
+// 1 / rms of the final norm) goes to its own buffer; every warp ranks a sixteenth of the vocabulary, warp 0 merges
+// the sixteen lists (KeepTopK with log-probabilities under temperature tau, Algorithm 1); then Eq. 5-7, Eq. 2 and
+// Eq. 4 on the request's own draft state, as block 0 of the single-request kernel does.
+__global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const KParams *kps, const float *Y, int nz, size_t zs, const float *ss,
+                                                                          float eps, int V) {
   extern __shared__ __align__(16) uint8_t bt_smem[];
   __shared__ int s_dead, s_quit;
   const KParams &p = kps[blockIdx.x];
+  const float rs = bt_rs(ss, blockIdx.x, p.d, eps);
   const float *row = Y + (size_t)blockIdx.x * V;
-  for (int c = threadIdx.x; c < V; c += kConsumerThreads) p.logits[c] = row[c];
+  for (int c = threadIdx.x; c < V; c += kConsumerThreads) {
+    float z = row[c];
+    for (int i = 1; i < nz; ++i) z += row[i * zs + c];
+    p.logits[c] = z * rs;
+  }
   if (threadIdx.x == 0) s_dead = s_quit = 0;
   __syncthreads();
-  State *st = p.st;
-  if (threadIdx.x < 32) {
-    block_topk(p, 0, V);  // the k best logits and (max, sum exp) of z / tau over the whole vocabulary, into this block's list
-    __syncwarp();
-    if (threadIdx.x == 0) {
-      const float2 ms = p.pk_ms[blockIdx.x];
-      const float lse = ms.x + __logf(ms.y);
-      for (int j = 0; j < p.k; ++j) {
-        const int id = p.pk_id[(size_t)blockIdx.x * p.k + j];
-        st->cand_tok[j] = id < 0 ? 0 : id;
-        st->cand_lp[j] = p.pk_val[(size_t)blockIdx.x * p.k + j] * p.inv_tau - lse;
-      }
-    }
+  {
+    const int warp = threadIdx.x >> 5;
+    const int r0 = (int)((long long)V * warp / kConsumerWarps), r1 = (int)((long long)V * (warp + 1) / kConsumerWarps);
+    block_topk(p, r0, r1, warp);  // this warp's list: slot `warp` of the request's own partial lists
   }
+  __threadfence_block();
+  __syncthreads();
+  if (threadIdx.x < 32) tail_keep_topk(p, kConsumerWarps);
   __syncthreads();
   Blk b;
   b.p = &p;
@@ -196,7 +264,9 @@ __global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const 
   b.quit = &s_quit;
   b.bar_target = 0;
   b.c_stage = b.c_phase = 0;
-  tail_score_select(b, false, st->n_gen);
+  b.rope_s = nullptr;
+  b.gain_ptrs = nullptr;
+  tail_score_select(b, false, p.st->n_gen);
 }
 
 }  // namespace spd
@@ -209,46 +279,62 @@ constexpr size_t kBatchTailSmem = 20480;
 // job: the buffers of the context that lends its long-prefix workspace (h, y, q, x, tensor maps); y_logits: [128][V]
 // floats; lm_tmap: the LM head's tensor map.  *launches receives the number of kernels enqueued.
 extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd::KParams *kps, int n, int V, const __nv_bfloat16 *final_norm,
-                                               float *y_logits, cudaStream_t s, int *launches) {
+                                               float *y_logits, size_t y_floats, size_t y_logits_floats, float *ss, int sm_count,
+                                               cudaStream_t s, int *launches) {
   const spd::TcJob &j = *job;
   const int d = j.d, f = j.f;
   const size_t ts_d = (size_t)j.x_term_rows * d, ts_f = (size_t)j.x_term_rows * f;
   const uint8_t *xmap_d = j.x_tmaps, *xmap_f = j.x_tmaps + spd::kTensorMapBytes;
   int count = 0;
   cudaError_t e = cudaSuccess;
-  auto gemm = [&](const uint8_t *xmap, int which, float *Y, int N, int C) {
+  // Up to 64 requests take the product built for few token rows (weights as the wide operand, columns split among
+  // blocks: its output is nz partial sums zs floats apart); more take the long-prefix path's 128-token tiles.
+  int nz = 1;
+  size_t zs = 0;
+  auto gemm = [&](const uint8_t *xmap, int which, float *Y, size_t room, int N, int C) {
     if (e != cudaSuccess) return;
-    e = spd_internal_tc_gemm(xmap, j.w_tmaps + (size_t)which * spd::kTensorMapBytes, Y, n, N, C, j.x_term_rows, j.st, s);
+    const uint8_t *wmap = j.w_tmaps + (size_t)which * spd::kTensorMapBytes;
+    if (n <= 64) {
+      e = spd_internal_batch_gemm(j.x_tmaps + 2 * spd::kTensorMapBytes, xmap != xmap_d, wmap, Y, room, n, N, C, j.x_term_rows, j.st, sm_count, s,
+                                  &nz, &zs);
+    } else {
+      nz = 1;
+      zs = 0;
+      e = spd_internal_tc_gemm(xmap, wmap, Y, n, N, C, j.x_term_rows, j.st, s);
+    }
     ++count;
   };
+  const int nch = (d + spd::kBtCols - 1) / spd::kBtCols;
   auto resid = [&](const __nv_bfloat16 *gain) {
     if (e != cudaSuccess) return;
-    e = spd_internal_tc_resid_norm(j.h, j.y, gain, j.x, ts_d, n, d, j.eps, s);
+    spd::spd_batch_resid_kernel<<<dim3(n, nch), 256, 0, s>>>(j.h, j.y, nz, zs, gain, j.x, ts_d, d, ss);
+    e = cudaGetLastError();
     ++count;
   };
-  spd::spd_batch_input_kernel<<<n, 256, 0, s>>>(kps, j.h, j.layers[0].attn_norm, j.x, ts_d, d, j.eps);
+  spd::spd_batch_input_kernel<<<dim3(n, nch), 256, 0, s>>>(kps, j.h, j.layers[0].attn_norm, j.x, ts_d, d, ss);
   e = cudaGetLastError();
   ++count;
   for (int l = 0; l < j.L && e == cudaSuccess; ++l) {
-    gemm(xmap_d, 4 * l, j.y, 3 * d, d);
+    gemm(xmap_d, 4 * l, j.y, y_floats, 3 * d, d);
     if (e != cudaSuccess) break;
-    spd::spd_batch_rope_cache_kernel<<<n, 256, 0, s>>>(j.y, j.q, kps, d, j.hd, l);
+    spd::spd_batch_rope_cache_kernel<<<dim3(n, (d / 2 + 255) / 256), 256, 0, s>>>(j.y, nz, zs, ss, j.eps, j.q, kps, d, j.hd, l);
     if ((e = cudaGetLastError()) != cudaSuccess) break;
     spd::spd_batch_attn_kernel<<<dim3(n, j.H), 128, 0, s>>>(j.q, kps, j.x, ts_d, d, j.hd, l);
     if ((e = cudaGetLastError()) != cudaSuccess) break;
     count += 2;
-    gemm(xmap_d, 4 * l + 1, j.y, d, d);
+    gemm(xmap_d, 4 * l + 1, j.y, y_floats, d, d);
     resid(j.layers[l].ffn_norm);
-    gemm(xmap_d, 4 * l + 2, j.y, 2 * f, d);
+    gemm(xmap_d, 4 * l + 2, j.y, y_floats, 2 * f, d);
     if (e != cudaSuccess) break;
-    e = spd_internal_tc_swiglu(j.y, j.x, ts_f, n, f, s);
+    spd::spd_batch_swiglu_kernel<<<dim3(n, (f + 255) / 256), 256, 0, s>>>(j.y, nz, zs, ss, j.eps, d, j.x, ts_f, f);
+    e = cudaGetLastError();
     ++count;
-    gemm(xmap_f, 4 * l + 3, j.y, d, f);
+    gemm(xmap_f, 4 * l + 3, j.y, y_floats, d, f);
     resid(l + 1 < j.L ? j.layers[l + 1].attn_norm : final_norm);
   }
-  gemm(xmap_d, 4 * j.L, y_logits, V, d);
+  gemm(xmap_d, 4 * j.L, y_logits, y_logits_floats, V, d);
   if (e == cudaSuccess) {
-    spd::spd_batch_tail_kernel<<<n, spd::kConsumerThreads, kBatchTailSmem, s>>>(kps, y_logits, V);
+    spd::spd_batch_tail_kernel<<<n, spd::kConsumerThreads, kBatchTailSmem, s>>>(kps, y_logits, nz, zs, ss, j.eps, V);
     e = cudaGetLastError();
     ++count;
   }

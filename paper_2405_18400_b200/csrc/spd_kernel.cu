@@ -973,10 +973,10 @@ __device__ void consumer_main(Blk &b) {
       named_sync(1, kConsumerThreads);
       int r0, r1;
       cta_rows(p.V, kImg ? kUnitRows : 1, r0, r1);
-      if (threadIdx.x < 32) block_topk(p, r0, r1);
+      if (threadIdx.x < 32) block_topk(p, r0, r1, blockIdx.x);
       if (grid_barrier(b)) return;
       if (blockIdx.x == 0 && (!kSampler || p.mode != kModeSample || last)) {
-        if (threadIdx.x < 32) tail_keep_topk(p);
+        if (threadIdx.x < 32) tail_keep_topk(p, gridDim.x);
         const bool first = p.mode != kModeDecode;
         if (kSampler && p.mode == kModeSample) sample_windows(p, it);
         tail_score_select(b, first, first ? 0 : p.step0 + it);

@@ -786,10 +786,10 @@ __device__ void pf_consumer(PfBlk &b) {
     named_sync(1, kPfThreads);
     int r0, r1;
     pf_rows(p.V, 1, r0, r1);
-    if (threadIdx.x < 32) block_topk(p, r0, r1);
+    if (threadIdx.x < 32) block_topk(p, r0, r1, blockIdx.x);
     if (pf_grid_barrier(b)) return;
     if (blockIdx.x == 0 && threadIdx.x < 32) {
-      tail_keep_topk(p);
+      tail_keep_topk(p, gridDim.x);
       tail_first(p, threadIdx.x, 0);
       __syncwarp();
       tail_gamma(p, threadIdx.x);

@@ -89,14 +89,34 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 consecutive float32 columns of this thread's lane of tensor memory.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 struct TcShared {
   uint64_t full[kTcStages], empty[kTcStages], acc_full[kTcAccs], acc_empty[kTcAccs];
   uint32_t tmem_base;
   int dead;
 };
 
+// The same for the small-batch product, whose ring has up to kBgMaxStages stages.
+constexpr int kBgMaxStages = 8;
+struct BgShared {
+  uint64_t full[kBgMaxStages], empty[kBgMaxStages], acc_full[kTcAccs], acc_empty[kTcAccs];
+  uint32_t tmem_base;
+  int dead;
+};
+
 // Bounded wait on an mbarrier phase; false when the block gave up (here or elsewhere).
-__device__ __forceinline__ bool tc_wait(TcShared &sh, State *st, uint64_t *bar, uint32_t parity, int info) {
+template <typename Shared>
+__device__ __forceinline__ bool tc_wait(Shared &sh, State *st, uint64_t *bar, uint32_t parity, int info) {
   if (mbar_try_wait(bar, parity)) return true;
   volatile int *dead = &sh.dead;
   unsigned long long t0 = globaltimer();
@@ -238,6 +258,146 @@ __global__ void __launch_bounds__(kTcThreads, 1)
   if (warp == 1) {
     tc_fence_after();
     tc_dealloc(tmem, kTcAccs * kTcN);
+  }
+}
+
+// ---------------------------------------------------------------- products of a small batch
+// Y[token][row] = sum_c X[token][c] W[row][c] for up to NP <= 64 token rows (the requests of a batched timestep).
+// With so few tokens the product is bound by the weight stream, so the tile is turned round: the 128 weight rows
+// are the wide operand of tcgen05.mma (M = 128) and the requests' terms the narrow one (N = NP), a stage holds
+// 16 KB of weights and only 3 x NP x 128 bytes of terms (spd_tc_gemm_kernel, built for 128 tokens per tile, brings
+// 48 KB of terms per 16 KB of weights), and the columns are split among blockIdx.y so that every product fills
+// the GPU: block (x, y) adds columns [64 kb_lo, 64 kb_hi) of rows 128 x .. 128 x + 127 into its own copy of Y
+// (Y + y * split_stride), which the kernels that read Y add up in a fixed order.  Accumulators as in
+// spd_tc_gemm_kernel: four sets of NP tensor-memory columns in rotation, each the sum of 8 stages, added in registers
+// with round-to-nearest.  Every wait is bounded.
+template <int NP>
+struct BgShape {
+  static constexpr int kTermBytes = NP * kTcKB * 2;                 // one term tile: NP token rows x 64 columns
+  static constexpr int kStageBytes = kTcWBytes + 3 * kTermBytes;    // 128 weight rows x 64 columns, then the three term tiles
+  static constexpr int kStages = NP <= 16 ? 4 : (NP <= 32 ? 3 : 5); // 91 KB and 87 KB: two blocks per SM; NP = 64: 205 KB, one
+  static constexpr int kTmemCols = 4 * NP < 32 ? 32 : 4 * NP;
+};
+
+template <int NP>
+__global__ void __launch_bounds__(kTcThreads)
+    spd_batch_gemm_kernel(const void *tmap_x, const void *tmap_w, float *Y, size_t split_stride, int n_tok, int N, int C, int x_term_rows,
+                          State *st) {
+  using S = BgShape<NP>;
+  static_assert(S::kStages <= kBgMaxStages, "the block's mbarrier arrays hold kBgMaxStages stages");
+  extern __shared__ __align__(16) uint8_t tc_smem_raw[];
+  uint8_t *smem = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
+  __shared__ BgShared sh;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nk_all = (C + kTcKB - 1) / kTcKB;
+  const int kb_lo = (int)((long long)nk_all * blockIdx.y / gridDim.y), kb_hi = (int)((long long)nk_all * (blockIdx.y + 1) / gridDim.y);
+  const int nk = kb_hi - kb_lo;
+  const int n0 = blockIdx.x * kTcN;
+  if (threadIdx.x == 0) {
+    sh.dead = 0;
+    for (int s = 0; s < S::kStages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], 1);
+    }
+    for (int a = 0; a < kTcAccs; ++a) {
+      mbar_init(&sh.acc_full[a], 1);
+      mbar_init(&sh.acc_empty[a], 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tc_alloc(&sh.tmem_base, S::kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  const uint32_t ring = smem_u32(smem);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, issued = 0;
+      bool ok = true;
+      for (int ks = 0; ks < nk; ++ks) {
+        if (!tc_wait(sh, st, &sh.empty[stage], phase ^ 1u, 500)) { ok = false; break; }
+        mbar_expect_tx(&sh.full[stage], (uint32_t)S::kStageBytes);
+        const uint32_t base = ring + stage * (uint32_t)S::kStageBytes;
+        const int col = (kb_lo + ks) * kTcKB;
+#pragma unroll
+        for (int j = 0; j < kTcN / kTcWBoxRows; ++j)
+          tc_box_load(base + j * (kTcWBoxRows * kTcKB * 2), tmap_w, col, n0 + j * kTcWBoxRows, &sh.full[stage]);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) tc_box_load(base + kTcWBytes + j * S::kTermBytes, tmap_x, col, j * x_term_rows, &sh.full[stage]);
+        if (issued < (uint32_t)S::kStages) ++issued;
+        if (++stage == (uint32_t)S::kStages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) {
+        uint32_t s = stage, ph = phase;
+        for (uint32_t i = 0; i < issued; ++i) {
+          if (s == 0) { s = (uint32_t)S::kStages; ph ^= 1u; }
+          --s;
+          unsigned long long t0 = globaltimer();
+          while (!mbar_try_wait(&sh.full[s], ph) && globaltimer() - t0 < kTcWaitNs) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = tc_idesc(kTcN, NP);  // M = 128 weight rows, N = NP token rows
+      uint32_t stage = 0, phase = 0;
+      for (int ks = 0; ks < nk; ++ks) {
+        const int seg = ks / kTcSegSteps, in_seg = ks - seg * kTcSegSteps, a = seg % kTcAccs;
+        if (in_seg == 0 && !tc_wait(sh, st, &sh.acc_empty[a], (uint32_t)((seg / kTcAccs) & 1) ^ 1u, 530)) break;
+        if (!tc_wait(sh, st, &sh.full[stage], phase, 510)) break;
+        tc_fence_after();
+        const uint32_t base = ring + stage * (uint32_t)S::kStageBytes;
+#pragma unroll
+        for (int j = 0; j < 3; ++j)
+#pragma unroll
+          for (int kk = 0; kk < kTcKB / 16; ++kk)
+            tc_mma(tmem + (uint32_t)(a * NP), tc_desc(base + kk * 32), tc_desc(base + kTcWBytes + j * S::kTermBytes + kk * 32), idesc,
+                   (uint32_t)((in_seg | j | kk) != 0));
+        tc_commit(&sh.empty[stage]);
+        if (in_seg == kTcSegSteps - 1 || ks == nk - 1) tc_commit(&sh.acc_full[a]);
+        if (++stage == (uint32_t)S::kStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+    __syncwarp();
+  } else {
+    // lane l of warp w reads tensor-memory lane 32 (w % 4) + l: weight row n0 + that, a token per column
+    const int quarter = warp & 3;
+    float sum[NP];
+#pragma unroll
+    for (int j = 0; j < NP; ++j) sum[j] = 0.f;
+    const int nseg = (nk + kTcSegSteps - 1) / kTcSegSteps;
+    bool ok = true;
+    for (int seg = 0; seg < nseg; ++seg) {
+      const int a = seg % kTcAccs;
+      if (!tc_wait(sh, st, &sh.acc_full[a], (uint32_t)((seg / kTcAccs) & 1), 520)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int c0 = 0; c0 < NP; c0 += 16) {
+        uint32_t r[16];
+        tc_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * NP + c0), r);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) sum[c0 + j] += __uint_as_float(r[j]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
+    }
+    const int row = n0 + quarter * 32 + lane;
+    if (ok && row < N) {
+      float *out = Y + (size_t)blockIdx.y * split_stride + row;
+#pragma unroll
+      for (int j = 0; j < NP; ++j)
+        if (j < n_tok) out[(size_t)j * N] = sum[j];  // the lanes of a warp write 32 consecutive floats of token j's row
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem, S::kTmemCols);
   }
 }
 
@@ -656,15 +816,41 @@ extern "C" cudaError_t spd_internal_tc_gemm(const void *xmap, const void *wmap, 
   return cudaGetLastError();
 }
 
-extern "C" cudaError_t spd_internal_tc_resid_norm(float *h, const float *y, const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int n_tok,
-                                                  int d, float eps, cudaStream_t s) {
-  spd::spd_tc_resid_norm_kernel<<<n_tok, 256, 0, s>>>(h, y, nullptr, nullptr, gain, X, term_stride, d, eps);
+namespace {
+template <int NP>
+cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size_t zs, int nz, int n_tok, int N, int C, int x_term_rows,
+                              spd::State *st, cudaStream_t s) {
+  using S = spd::BgShape<NP>;
+  const size_t smem = (size_t)S::kStages * S::kStageBytes + 1024;
+  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_batch_gemm_kernel<NP>),
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  spd::spd_batch_gemm_kernel<NP><<<dim3((N + spd::kTcN - 1) / spd::kTcN, nz), spd::kTcThreads, smem, s>>>(xmap, wmap, Y, zs, n_tok, N, C,
+                                                                                                            x_term_rows, st);
   return cudaGetLastError();
 }
+}  // namespace
 
-extern "C" cudaError_t spd_internal_tc_swiglu(const float *Y, uint16_t *X, size_t term_stride, int n_tok, int f, cudaStream_t s) {
-  spd::spd_tc_swiglu_kernel<<<n_tok, 256, 0, s>>>(Y, X, term_stride, f);
-  return cudaGetLastError();
+// Product of a small batch (n_tok <= 64 token rows): xmaps = the term buffer's tensor maps with boxes of 16, 32 and 64
+// rows (two each: d_model and d_ffn columns; `wide` picks the second).  The columns are split nz ways (chosen here
+// so that the product has about two blocks per SM, within y_floats of room for the partial sums); *out_nz and
+// *out_zs tell the reader of Y how many partial sums there are and how far apart.
+extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
+                                               int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int *out_nz, size_t *out_zs) {
+  const int np = n_tok <= 16 ? 16 : (n_tok <= 32 ? 32 : 64);
+  const int slot = (np == 16 ? 0 : (np == 32 ? 1 : 2)) * 2 + (wide ? 1 : 0);
+  const void *xmap = xmaps + (size_t)slot * spd::kTensorMapBytes;
+  const int tiles = (N + spd::kTcN - 1) / spd::kTcN, nk = (C + spd::kTcKB - 1) / spd::kTcKB;
+  const size_t zs = (size_t)n_tok * N;
+  int nz = (2 * sm_count + tiles / 2) / tiles;               // about two blocks per SM
+  if (nz > nk / 8) nz = nk / 8;                               // at least 8 stages of work per block
+  if ((size_t)nz * zs > y_floats) nz = (int)(y_floats / zs);  // room for the partial sums
+  if (nz < 1) nz = 1;
+  *out_nz = nz;
+  *out_zs = zs;
+  if (np == 16) return launch_batch_gemm<16>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
+  if (np == 32) return launch_batch_gemm<32>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
+  return launch_batch_gemm<64>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
 }
 
 // Test hook: one tile of the first layer's QKV product whose first stage never arrives (see the kernel's `stall`).

@@ -15,7 +15,8 @@ struct TcJob {
   const LayerW *layers;              // HOST copy of the layer table [L]
   const __nv_bfloat16 *tok_emb;
   const uint8_t *w_tmaps;            // device: tensor maps of the layers' matrices, four per layer
-  const uint8_t *x_tmaps;            // device: tensor maps of the term buffer seen as [3 * x_term_rows][d] and [..][f]
+  const uint8_t *x_tmaps;            // device: tensor maps of the term buffer seen as [3 * x_term_rows][d] and [..][f], boxes of 128 rows;
+                                     // then three more pairs with boxes of 16, 32 and 64 rows (products of a small batch)
   void *kcache, *vcache;
   const float2 *rope;
   float *h, *y, *q;                  // [x_term_rows][d], [x_term_rows][max(3d, 2f)], [x_term_rows][d]
@@ -31,9 +32,8 @@ struct TcJob {
 extern "C" cudaError_t spd_internal_tc_prepare(void);
 extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);
-// The long-prefix path's products and row-wise kernels for other callers (the batched timestep).
+// The long-prefix path's product for other callers (the batched timestep), and the product of a small batch.
 extern "C" cudaError_t spd_internal_tc_gemm(const void *xmap, const void *wmap, float *Y, int n_tok, int N, int C, int x_term_rows,
                                             spd::State *st, cudaStream_t s);
-extern "C" cudaError_t spd_internal_tc_resid_norm(float *h, const float *y, const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int n_tok,
-                                                  int d, float eps, cudaStream_t s);
-extern "C" cudaError_t spd_internal_tc_swiglu(const float *Y, uint16_t *X, size_t term_stride, int n_tok, int f, cudaStream_t s);
+extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
+                                               int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int *out_nz, size_t *out_zs);

@@ -22,8 +22,9 @@ __device__ __forceinline__ void warp_best(float &v, int &i) {
   }
 }
 
-// Warp 0 of each block: the k best logits among rows [r0, r1) and (max, sum exp) of z / tau over them.
-static __device__ void block_topk(const KParams &p, int r0, int r1) {
+// One warp: the k best logits among rows [r0, r1) and (max, sum exp) of z / tau over them, into list `slot` of the
+// partial lists (the decode and prefill kernels: warp 0 of each block, slot = the block).
+static __device__ void block_topk(const KParams &p, int r0, int r1, int slot) {
   const int lane = threadIdx.x & 31;
   float pv = 0.f;
   int pi = -1;
@@ -38,8 +39,8 @@ static __device__ void block_topk(const KParams &p, int r0, int r1) {
     }
     warp_best(bv, bi);
     if (lane == 0) {
-      p.pk_val[(size_t)blockIdx.x * p.k + j] = bi >= 0 ? bv : -CUDART_INF_F;
-      p.pk_id[(size_t)blockIdx.x * p.k + j] = bi;
+      p.pk_val[(size_t)slot * p.k + j] = bi >= 0 ? bv : -CUDART_INF_F;
+      p.pk_id[(size_t)slot * p.k + j] = bi;
     }
     pv = bv;
     pi = bi;
@@ -47,8 +48,8 @@ static __device__ void block_topk(const KParams &p, int r0, int r1) {
     if (bi < 0) {  // fewer rows than k: the rest stay empty
       for (int jj = j + 1; jj < p.k; ++jj)
         if (lane == 0) {
-          p.pk_val[(size_t)blockIdx.x * p.k + jj] = -CUDART_INF_F;
-          p.pk_id[(size_t)blockIdx.x * p.k + jj] = -1;
+          p.pk_val[(size_t)slot * p.k + jj] = -CUDART_INF_F;
+          p.pk_id[(size_t)slot * p.k + jj] = -1;
         }
       break;
     }
@@ -57,21 +58,21 @@ static __device__ void block_topk(const KParams &p, int r0, int r1) {
   for (int r = r0 + lane; r < r1; r += 32) s += __expf(p.logits[r] * p.inv_tau - mx);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if (lane == 0) p.pk_ms[blockIdx.x] = make_float2(mx, s);
+  if (lane == 0) p.pk_ms[slot] = make_float2(mx, s);
 }
 
-// KeepTopK over the whole vocabulary from the blocks' partial lists (Algorithm 1), with
+// KeepTopK over the whole vocabulary from the n_lists partial lists (Algorithm 1), with
 // log-probabilities under temperature tau.  Warp 0.
-static __device__ void tail_keep_topk(const KParams &p) {
+static __device__ void tail_keep_topk(const KParams &p, int n_lists) {
   const int lane = threadIdx.x & 31;
   State *st = p.st;
-  const int ncand = (int)gridDim.x * p.k;
+  const int ncand = n_lists * p.k;
   float M = -CUDART_INF_F;
-  for (int g = lane; g < (int)gridDim.x; g += 32) M = fmaxf(M, __ldcg(&p.pk_ms[g]).x);
+  for (int g = lane; g < n_lists; g += 32) M = fmaxf(M, __ldcg(&p.pk_ms[g]).x);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   float S = 0.f;
-  for (int g = lane; g < (int)gridDim.x; g += 32) {
+  for (int g = lane; g < n_lists; g += 32) {
     const float2 ms = __ldcg(&p.pk_ms[g]);
     if (ms.x > -CUDART_INF_F) S = fmaf(ms.y, __expf(ms.x - M), S);
   }

@@ -24,7 +24,9 @@ def _requests(P, shape, packed, dtabs, host, tables, n, k, orders, lam, alpha, t
     return out
 
 
-@pytest.mark.parametrize("n,kv_dtype", [(2, "bf16"), (8, "f32"), (32, "bf16")])
+# up to 16, 32 and 64 requests take the small-batch product with token boxes of that many rows; more take the
+# long-prefix path's 128-token tiles
+@pytest.mark.parametrize("n,kv_dtype", [(2, "bf16"), (8, "f32"), (32, "bf16"), (48, "bf16"), (70, "f32")])
 def test_batched_steps_tiny(tiny_inputs, n, kv_dtype):
     import paper_2405_18400_b200 as P
 
