@@ -706,15 +706,22 @@ __device__ void attention_phase_bf16_hd128(Blk &b, int layer, int pos) {
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
     float m = -CUDART_INF_F, l = 0.f;
     const size_t col = (size_t)head * 128 + l16 * 8;
-    for (int tb = t0 + warp * 8; tb < t1; tb += kConsumerWarps * 8) {
-      uint4 kq[4], vq[4];
+    // A round = four positions per half-warp; they enter the running softmax together (one rescale per round instead
+    // of four dependent ones).
+    constexpr int kStep = kConsumerWarps * 8;
+    uint4 kq[4], vq[4];
+    auto fetch = [&](int tb, const __nv_bfloat16 *cache, uint4 (&dst)[4]) {
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int t = min(tb + 2 * u + half, t1 - 1);  // clamped: the extra loads are discarded below
-        const size_t off = ((size_t)layer * p.max_pos + t) * p.d + col;
-        kq[u] = __ldcg(reinterpret_cast<const uint4 *>(kc + off));
-        vq[u] = __ldcg(reinterpret_cast<const uint4 *>(vc + off));
+        const int t = max(min(tb + 2 * u + half, t1 - 1), 0);  // clamped: the extra loads are discarded below
+        dst[u] = __ldcg(reinterpret_cast<const uint4 *>(cache + ((size_t)layer * p.max_pos + t) * p.d + col));
       }
+    };
+    for (int tb = t0 + warp * 8; tb < t1; tb += kStep) {
+      fetch(tb, kc, kq);
+      fetch(tb, vc, vq);
+      float sc[4];
+      float mn = m;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const uint32_t kw[4] = {kq[u].x, kq[u].y, kq[u].z, kq[u].w};
@@ -726,19 +733,26 @@ __device__ void attention_phase_bf16_hd128(Blk &b, int layer, int pos) {
         }
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        if (tb + 2 * u + half < t1) {  // uniform within the half-warp
-          const float s = dot * scale;
-          const float mn = fmaxf(m, s);
-          const float c = __expf(m - mn), pw = __expf(s - mn);
-          l = l * c + pw;
+        sc[u] = tb + 2 * u + half < t1 ? dot * scale : -CUDART_INF_F;  // uniform within the half-warp
+        mn = fmaxf(mn, sc[u]);
+      }
+      if (mn > -CUDART_INF_F) {  // else nothing of this round (nor of an earlier one) belongs to the half-warp
+        const float c = __expf(m - mn);
+        l *= c;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] *= c;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float pw = __expf(sc[u] - mn);  // 0 for a position past the range
+          l += pw;
           const uint32_t vw[4] = {vq[u].x, vq[u].y, vq[u].z, vq[u].w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            acc[2 * e] = acc[2 * e] * c + pw * __uint_as_float(vw[e] << 16);
-            acc[2 * e + 1] = acc[2 * e + 1] * c + pw * __uint_as_float(vw[e] & 0xffff0000u);
+            acc[2 * e] = fmaf(pw, __uint_as_float(vw[e] << 16), acc[2 * e]);
+            acc[2 * e + 1] = fmaf(pw, __uint_as_float(vw[e] & 0xffff0000u), acc[2 * e + 1]);
           }
-          m = mn;
         }
+        m = mn;
       }
     }
     // merge the two half-warps
