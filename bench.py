@@ -234,7 +234,7 @@ def run_batched(args, wl, P, dev, rank, world, packed, dtabs, k, K, W):
            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": cfg,
            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
-                        "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_batch_gemm_kernel" if B <= 64 else "spd_tc_gemm_kernel",
+                        "peak_kind": peak_kind, "bytes_per_step": bytes_step, "kernel": "spd_batch_gemm_kernel",
                         "note": "weights once per timestep + per request its KV cache, embedding rows and table probes; the products' "
                                 "share of the step is in the launch list under profiles/"},
            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "batch": B}

@@ -2,14 +2,15 @@
 // remark: batching is complementary to the method, since each request still needs one pass for its k drafts).
 //
 // A request is a context of its own (prefix, KV cache, draft state); the requests of a batch share the weights and
-// the n-gram tables.  Their superposed inputs (Eq. 3) are the token rows of one tile of the tensor-core products that
-// the long-prefix path already has (spd_tc_gemm_kernel: tcgen05.mma with TMEM accumulators, activations as three
-// exact bf16 terms), so the weights are streamed once per timestep whatever the number of requests.  Between the
-// products run row-wise kernels, one block per request (and head): the superposed embedding, the rotary embedding
-// and the append to the request's own cache at its own position, attention over that cache, residual + RMSNorm
-// and SwiGLU (the long-prefix path's kernels).  After the LM head (one more product, a row of logits per request)
-// a block per request runs the method's tail on the request's own draft state: KeepTopK, Eq. 5-7 with the n-gram
-// probes, Eq. 2, Eq. 4.
+// the n-gram tables.  Their superposed inputs (Eq. 3) are the token rows of a tensor-core product made for few rows
+// (spd_batch_gemm_kernel in spd_prefill_tc.cu: the 128 weight rows of a tile are the wide tcgen05.mma operand, the
+// requests' activations, as three exact bf16 terms, the narrow one, TMEM accumulators, columns split among blocks),
+// so the weights are streamed once per timestep whatever the number of requests.  Between the products run
+// element-wise kernels spread over requests and columns: the superposed embedding, the rotary embedding and the
+// append to the request's own cache at its own position, attention over that cache (a block per request and head),
+// residual add and SwiGLU; RMSNorm's 1 / rms is applied behind the product that follows it.  After the LM head (one
+// more product, a row of logits per request) a block per request runs the method's tail on the request's own draft
+// state: KeepTopK, Eq. 5-7 with the n-gram probes, Eq. 2, Eq. 4.
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
@@ -287,21 +288,14 @@ extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd:
   const uint8_t *xmap_d = j.x_tmaps, *xmap_f = j.x_tmaps + spd::kTensorMapBytes;
   int count = 0;
   cudaError_t e = cudaSuccess;
-  // Up to 64 requests take the product built for few token rows (weights as the wide operand, columns split among
-  // blocks: its output is nz partial sums zs floats apart); more take the long-prefix path's 128-token tiles.
+  // The product built for few token rows (weights as the wide operand, columns split among blocks): its output is nz
+  // partial sums zs floats apart.
   int nz = 1;
   size_t zs = 0;
   auto gemm = [&](const uint8_t *xmap, int which, float *Y, size_t room, int N, int C) {
     if (e != cudaSuccess) return;
     const uint8_t *wmap = j.w_tmaps + (size_t)which * spd::kTensorMapBytes;
-    if (n <= 64) {
-      e = spd_internal_batch_gemm(j.x_tmaps + 2 * spd::kTensorMapBytes, xmap != xmap_d, wmap, Y, room, n, N, C, j.x_term_rows, j.st, sm_count, s,
-                                  &nz, &zs);
-    } else {
-      nz = 1;
-      zs = 0;
-      e = spd_internal_tc_gemm(xmap, wmap, Y, n, N, C, j.x_term_rows, j.st, s);
-    }
+    e = spd_internal_batch_gemm(j.x_tmaps, xmap != xmap_d, wmap, Y, room, n, N, C, j.x_term_rows, j.st, sm_count, s, &nz, &zs);
     ++count;
   };
   const int nch = (d + spd::kBtCols - 1) / spd::kBtCols;

@@ -275,7 +275,8 @@ template <int NP>
 struct BgShape {
   static constexpr int kTermBytes = NP * kTcKB * 2;                 // one term tile: NP token rows x 64 columns
   static constexpr int kStageBytes = kTcWBytes + 3 * kTermBytes;    // 128 weight rows x 64 columns, then the three term tiles
-  static constexpr int kStages = NP <= 16 ? 4 : (NP <= 32 ? 3 : 5); // 91 KB and 87 KB: two blocks per SM; NP = 64: 205 KB, one
+  static constexpr int kStages = NP <= 16 ? 4 : (NP <= 32 ? 3 : (NP <= 64 ? 5 : 3));  // 91 KB and 87 KB: two blocks per SM; NP = 64:
+                                                                                     // 205 KB, NP = 128: 197 KB, one block
   static constexpr int kTmemCols = 4 * NP < 32 ? 32 : 4 * NP;
 };
 
@@ -807,15 +808,6 @@ extern "C" cudaError_t spd_internal_tc_prepare(void) {
   return e;
 }
 
-// Launchers for the batched timestep (spd_batch.cu), which runs the same products and row-wise kernels on a tile of
-// requests instead of prefix tokens.
-extern "C" cudaError_t spd_internal_tc_gemm(const void *xmap, const void *wmap, float *Y, int n_tok, int N, int C, int x_term_rows,
-                                            spd::State *st, cudaStream_t s) {
-  const dim3 grid((n_tok + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
-  spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, wmap, Y, N, C, x_term_rows, st, 0);
-  return cudaGetLastError();
-}
-
 namespace {
 template <int NP>
 cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size_t zs, int nz, int n_tok, int N, int C, int x_term_rows,
@@ -831,18 +823,20 @@ cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size
 }
 }  // namespace
 
-// Product of a small batch (n_tok <= 64 token rows): xmaps = the term buffer's tensor maps with boxes of 16, 32 and 64
+// Product of a batch (n_tok <= 128 token rows): xmaps = the term buffer's tensor maps with boxes of 128, 16, 32 and 64
 // rows (two each: d_model and d_ffn columns; `wide` picks the second).  The columns are split nz ways (chosen here
 // so that the product has about two blocks per SM, within y_floats of room for the partial sums); *out_nz and
 // *out_zs tell the reader of Y how many partial sums there are and how far apart.
 extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
                                                int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int *out_nz, size_t *out_zs) {
-  const int np = n_tok <= 16 ? 16 : (n_tok <= 32 ? 32 : 64);
-  const int slot = (np == 16 ? 0 : (np == 32 ? 1 : 2)) * 2 + (wide ? 1 : 0);
+  const int np = n_tok <= 16 ? 16 : (n_tok <= 32 ? 32 : (n_tok <= 64 ? 64 : 128));
+  // the term buffer's tensor maps: boxes of 128 rows first, then 16, 32 and 64 (two each: d_model and d_ffn columns)
+  const int slot = (np == 128 ? 0 : (np == 16 ? 1 : (np == 32 ? 2 : 3))) * 2 + (wide ? 1 : 0);
   const void *xmap = xmaps + (size_t)slot * spd::kTensorMapBytes;
   const int tiles = (N + spd::kTcN - 1) / spd::kTcN, nk = (C + spd::kTcKB - 1) / spd::kTcKB;
   const size_t zs = (size_t)n_tok * N;
-  int nz = (2 * sm_count + tiles / 2) / tiles;               // about two blocks per SM
+  int nz = (2 * sm_count + tiles / 2) / tiles;               // about two blocks per SM (64 token rows, one block per SM at a
+                                                              // time: 7.1 ms per 7B timestep against 8.6 ms with half as many)
   if (nz > nk / 8) nz = nk / 8;                               // at least 8 stages of work per block
   if ((size_t)nz * zs > y_floats) nz = (int)(y_floats / zs);  // room for the partial sums
   if (nz < 1) nz = 1;
@@ -850,7 +844,8 @@ extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, c
   *out_zs = zs;
   if (np == 16) return launch_batch_gemm<16>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
   if (np == 32) return launch_batch_gemm<32>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
-  return launch_batch_gemm<64>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
+  if (np == 64) return launch_batch_gemm<64>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
+  return launch_batch_gemm<128>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
 }
 
 // Test hook: one tile of the first layer's QKV product whose first stage never arrives (see the kernel's `stall`).

@@ -32,8 +32,6 @@ struct TcJob {
 extern "C" cudaError_t spd_internal_tc_prepare(void);
 extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);
-// The long-prefix path's product for other callers (the batched timestep), and the product of a small batch.
-extern "C" cudaError_t spd_internal_tc_gemm(const void *xmap, const void *wmap, float *Y, int n_tok, int N, int C, int x_term_rows,
-                                            spd::State *st, cudaStream_t s);
+// The product of a batched timestep's few token rows.
 extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
                                                int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int *out_nz, size_t *out_zs);

@@ -43,7 +43,8 @@ U32 = 2.0 ** -24      # unit roundoff of float32
 # U32 * (layers + 1) * rms(cache).  A cache value of layer l is a float32 dot product over d terms (error of a
 # few U32 relative to the rms of the values, the partial sums being added as a tree) of a residual stream
 # that carries the errors of the l layers before it, each of the same kind; the sum grows at most linearly in
-# l.  Decode steps accumulate in float32 with round-to-nearest (measured: need <= ~3 of these units); the
+# l.  Decode steps accumulate in float32 with round-to-nearest, or, with fragment-order weight images, in chains of
+# at most 16 tensor-core instructions whose sums are then added in float32 (measured: need <= ~3 of these units); the
 # prefill kernels accumulate inside the tensor cores, which truncate every addition of a 96-instruction chain
 # (measured: need <= ~40 units).  The constants leave a factor of about four over what was measured.
 SLACK_UNITS = {"decode": 12.0, "prefill": 160.0}
