@@ -342,7 +342,7 @@ def run_ours(args, wl):
     e2e = {"value": world * k * gen / e2e_s if e2e_s else None, "unit": UNIT, "h2d_bytes_per_step": 4.0 * wl.prefix_len / gen,
            "d2h_bytes_per_step": 12.0 * k, "what": "spd_prefill(host ids) + %d spd_step calls returning ids, parents and gamma "
            "to the host, per request of %d tokens per draft; prefill = one launch of the batched kernel per 16 prefix tokens, the last one ending with the LM head and the first timestep; "
-           "prefixes over 64 tokens send all but their last 1..16 tokens through the tcgen05 long-prefix path" % (gen - 1, gen),
+           "prefixes over 32 tokens send all but their last 1..16 tokens through the tcgen05 long-prefix path" % (gen - 1, gen),
            "ms_per_request": e2e_s * 1e3 if e2e_s else None,
            "ms_to_first_drafts": min(first_t) * 1e3 if first_t else None}
 

@@ -125,7 +125,7 @@ int spd_create(const spd_config *cfg, const spd_weights *weights, const spd_ngra
  * over the m prefix tokens (HOST int32 ids, 1 <= m < max_pos), draft i takes the i-th most probable
  * next token and its probability, no n-gram term.  out_ids / out_gamma: HOST arrays of k entries
  * (token of draft i; gamma_i of Eq. 4), either may be NULL.  Restarts the context from scratch.
- * Synchronises the stream before returning.  Prefixes of more than 64 tokens (head size 64 or 128,
+ * Synchronises the stream before returning.  Prefixes of more than 32 tokens (head size 64 or 128,
  * max_pos >= 130) run all but their last 1..16 tokens through the long-prefix path (tensor-core
  * products over up to 512 tokens at a time, many small launches); its buffers are part of the
  * workspace.  The result does not depend on which path a token took beyond float rounding.

@@ -264,6 +264,8 @@ spd::TcJob tc_job(spd_ctx *ctx) {
   job.x = reinterpret_cast<uint16_t *>(ctx->ws + ctx->lay.tc_x);
   job.x_term_rows = ctx->tc_rows;
   job.st = kp.st;
+  job.sm_count = ctx->grid;
+  job.y_floats = (size_t)ctx->tc_rows * (size_t)(3 * kp.d > 2 * kp.f ? 3 * kp.d : 2 * kp.f);
   job.ids = nullptr;
   job.pos0 = job.n_tok = 0;
   return job;

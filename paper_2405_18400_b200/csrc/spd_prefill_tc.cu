@@ -427,10 +427,12 @@ __device__ __forceinline__ float tc_block_sum(float v, float *scratch) {
   return s;
 }
 
-// One token per block: the residual row (the embedding of ids[t] when `ids`, else h + y when `y`), stored, and
+// One token per block: the residual row (the embedding of ids[t] when `ids`, else h + y when `y`; y, like every
+// product's output read below, is the sum of nz partial products zs floats apart), stored, and
 // when `gain`: its RMSNorm (x * rsqrt(mean x^2 + eps) * gain) as three bf16 terms for the next product.
 __global__ void __launch_bounds__(256) spd_tc_resid_norm_kernel(float *h, const float *y, const int32_t *ids, const __nv_bfloat16 *emb,
-                                                                const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int d, float eps) {
+                                                                const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int d, float eps,
+                                                                int nz, size_t zs) {
   __shared__ float scratch[8];
   const int t = blockIdx.x;
   float *hr = h + (size_t)t * d;
@@ -438,7 +440,10 @@ __global__ void __launch_bounds__(256) spd_tc_resid_norm_kernel(float *h, const 
   for (int c = threadIdx.x; c < d; c += 256) {
     float v;
     if (ids) v = __bfloat162float(emb[(size_t)ids[t] * d + c]);
-    else v = hr[c] + y[(size_t)t * d + c];
+    else {
+      v = hr[c];
+      for (int z = 0; z < nz; ++z) v += y[z * zs + (size_t)t * d + c];
+    }
     hr[c] = v;
     ss = fmaf(v, v, ss);
   }
@@ -450,17 +455,22 @@ __global__ void __launch_bounds__(256) spd_tc_resid_norm_kernel(float *h, const 
 // One token per block: rotary embedding of q and k (adjacent pairs), q to Q, k and v into the cache at the
 // token's position.  Y row = [q | k | v].
 __global__ void __launch_bounds__(256) spd_tc_rope_cache_kernel(const float *Y, float *Q, void *kcache, void *vcache, const float2 *rope,
-                                                                int d, int hd, int max_pos, int layer, int pos0, int kv_bf16) {
+                                                                int d, int hd, int max_pos, int layer, int pos0, int kv_bf16, int nz, size_t zs) {
   const int t = blockIdx.x, pos = pos0 + t;
   const float *yr = Y + (size_t)t * 3 * d;
   const size_t crow = ((size_t)layer * max_pos + pos) * d;
   for (int i = threadIdx.x; i < d / 2; i += 256) {
     const float2 cs = rope[(size_t)pos * (hd / 2) + (i % (hd / 2))];
-    const float qe = yr[2 * i], qo = yr[2 * i + 1], ke = yr[d + 2 * i], ko = yr[d + 2 * i + 1];
+    float qe = 0.f, qo = 0.f, ke = 0.f, ko = 0.f, v0 = 0.f, v1 = 0.f;
+    for (int z = 0; z < nz; ++z) {
+      const float *yz = yr + z * zs;
+      qe += yz[2 * i]; qo += yz[2 * i + 1];
+      ke += yz[d + 2 * i]; ko += yz[d + 2 * i + 1];
+      v0 += yz[2 * d + 2 * i]; v1 += yz[2 * d + 2 * i + 1];
+    }
     Q[(size_t)t * d + 2 * i] = qe * cs.x - qo * cs.y;
     Q[(size_t)t * d + 2 * i + 1] = qe * cs.y + qo * cs.x;
     const float k0 = ke * cs.x - ko * cs.y, k1 = ke * cs.y + ko * cs.x;
-    const float v0 = yr[2 * d + 2 * i], v1 = yr[2 * d + 2 * i + 1];
     if (kv_bf16) {
       reinterpret_cast<__nv_bfloat162 *>(kcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(k0), __float2bfloat16_rn(k1));
       reinterpret_cast<__nv_bfloat162 *>(vcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(v0), __float2bfloat16_rn(v1));
@@ -472,11 +482,16 @@ __global__ void __launch_bounds__(256) spd_tc_rope_cache_kernel(const float *Y, 
 }
 
 // One token per block: u = SiLU(gate) * up from Y row = [gate_0, up_0, gate_1, up_1, ...], as three bf16 terms.
-__global__ void __launch_bounds__(256) spd_tc_swiglu_kernel(const float *Y, uint16_t *X, size_t term_stride, int f) {
+__global__ void __launch_bounds__(256) spd_tc_swiglu_kernel(const float *Y, uint16_t *X, size_t term_stride, int f, int nz, size_t zs) {
   const int t = blockIdx.x;
   const float2 *yr = reinterpret_cast<const float2 *>(Y + (size_t)t * 2 * f);
   for (int j = threadIdx.x; j < f; j += 256) {
-    const float2 gu = yr[j];
+    float2 gu = yr[j];
+    for (int z = 1; z < nz; ++z) {
+      const float2 more = yr[z * (zs / 2) + j];
+      gu.x += more.x;
+      gu.y += more.y;
+    }
     tc_put3(X, term_stride, (size_t)t * f + j, gu.x / (1.f + __expf(-gu.x)) * gu.y);
   }
 }
@@ -866,17 +881,26 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
   const uint8_t *xmap_d = j.x_tmaps, *xmap_f = j.x_tmaps + spd::kTensorMapBytes;
   int count = 0;
   cudaError_t e = cudaSuccess;
+  // A job of up to 128 tokens is one token tile: its products are bound by the weight stream and take the product
+  // made for few token rows (weights as the wide operand, columns split among blocks; its output is nz partial sums
+  // zs floats apart, which the row-wise kernels add up).
+  int nz = 1;
+  size_t zs = 0;
   auto gemm = [&](const uint8_t *xmap, int which, int N, int C) {
     if (e != cudaSuccess) return;
-    const dim3 grid((n + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
-    spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, j.w_tmaps + (size_t)which * spd::kTensorMapBytes, j.y, N, C,
-                                                                         j.x_term_rows, j.st, 0);
-    e = cudaGetLastError();
+    const uint8_t *wmap = j.w_tmaps + (size_t)which * spd::kTensorMapBytes;
+    if (n <= spd::kTcM) {
+      e = spd_internal_batch_gemm(j.x_tmaps, xmap != xmap_d, wmap, j.y, j.y_floats, n, N, C, j.x_term_rows, j.st, j.sm_count, s, &nz, &zs);
+    } else {
+      const dim3 grid((n + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
+      spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, wmap, j.y, N, C, j.x_term_rows, j.st, 0);
+      e = cudaGetLastError();
+    }
     ++count;
   };
   auto resid = [&](const float *y, const int32_t *ids, const __nv_bfloat16 *gain) {
     if (e != cudaSuccess) return;
-    spd::spd_tc_resid_norm_kernel<<<n, 256, 0, s>>>(j.h, y, ids, j.tok_emb, gain, j.x, ts_d, d, j.eps);
+    spd::spd_tc_resid_norm_kernel<<<n, 256, 0, s>>>(j.h, y, ids, j.tok_emb, gain, j.x, ts_d, d, j.eps, nz, zs);
     e = cudaGetLastError();
     ++count;
   };
@@ -884,7 +908,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
   for (int l = 0; l < j.L && e == cudaSuccess; ++l) {
     gemm(xmap_d, 4 * l, 3 * d, d);
     if (e != cudaSuccess) break;
-    spd::spd_tc_rope_cache_kernel<<<n, 256, 0, s>>>(j.y, j.q, j.kcache, j.vcache, j.rope, d, j.hd, j.max_pos, l, j.pos0, j.kv_bf16);
+    spd::spd_tc_rope_cache_kernel<<<n, 256, 0, s>>>(j.y, j.q, j.kcache, j.vcache, j.rope, d, j.hd, j.max_pos, l, j.pos0, j.kv_bf16, nz, zs);
     if ((e = cudaGetLastError()) != cudaSuccess) break;
     e = j.hd == 128 ? launch_attn<128>(j, l, n, s) : launch_attn<64>(j, l, n, s);  // other head sizes never get here
     count += 2;
@@ -892,7 +916,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
     resid(j.y, nullptr, j.layers[l].ffn_norm);
     gemm(xmap_d, 4 * l + 2, 2 * f, d);
     if (e != cudaSuccess) break;
-    spd::spd_tc_swiglu_kernel<<<n, 256, 0, s>>>(j.y, j.x, ts_f, f);
+    spd::spd_tc_swiglu_kernel<<<n, 256, 0, s>>>(j.y, j.x, ts_f, f, nz, zs);
     e = cudaGetLastError();
     ++count;
     gemm(xmap_f, 4 * l + 3, d, f);

@@ -6,8 +6,8 @@ namespace spd {
 
 constexpr int kTcTile = 128;      // tokens per tile of the tensor-core products
 constexpr int kTcMaxTokens = 512; // tokens one job takes at most
-constexpr int kTcMinPrefix = 64;  // runs of more tokens than this take the path: a job of up to 128 tokens costs about 2.7 launches
-                                  // of the 16-token kernel (7B shape: 12.6 ms against 4.66 ms), so four launches before the last pay for it
+constexpr int kTcMinPrefix = 32;  // runs of more tokens than this take the path: a job of up to 128 tokens costs about 1.5 launches
+                                  // of the 16-token kernel, so two launches before the last pay for it
 
 struct TcJob {
   int32_t L, d, H, hd, f, max_pos, kv_bf16;
@@ -25,6 +25,8 @@ struct TcJob {
   const int32_t *ids;                // device: the job's token ids
   int32_t pos0, n_tok;               // first position; tokens (<= x_term_rows)
   State *st;
+  int32_t sm_count;                  // SMs of the device
+  size_t y_floats;                   // room of y in floats (partial sums of a column-split product)
 };
 
 }  // namespace spd

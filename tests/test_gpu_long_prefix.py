@@ -1,4 +1,4 @@
-"""Prefixes of more than 64 tokens: all but the last 1..16 tokens go through the tensor-core path (tcgen05
+"""Prefixes of more than 32 tokens: all but the last 1..16 tokens go through the tensor-core path (tcgen05
 products over tiles of 128 tokens, up to 512 tokens per job), the rest through the 16-token prefill kernel,
 which ends with the first timestep (Eq. 1).  Both fill the same cache; the first timestep and the steps after
 it are compared with the oracle as for short prefixes."""
@@ -12,17 +12,19 @@ pytestmark = pytest.mark.gpu
 
 
 def _expected_launches(m, layers, job_tokens):
-    tc = m - ((m - 1) % 16 + 1) if m > 64 else 0
+    tc = m - ((m - 1) % 16 + 1) if m > 32 else 0
     jobs = -(-tc // job_tokens) if tc else 0
     return jobs * 9 * layers + (m - tc + 15) // 16
 
 
 @pytest.mark.parametrize("kv_dtype", ["bf16", "f32"])
-@pytest.mark.parametrize("m", [65, 129, 293, 700])
+@pytest.mark.parametrize("m", [33, 64, 65, 129, 145, 293, 700])
 def test_long_prefix_tiny(tiny_inputs, m, kv_dtype):
     """Tiny shape: d_ffn = 688 leaves a ragged last 64-column stage and 2 d_ffn = 1376 a ragged last row tile;
-    65 = the shortest prefix that takes the path (a tile with 64 tokens in it), 129 = one tile and one token, 293 = one job of 288 tokens (a last tile of 32), 700 = a job of 512 tokens and
-    one of 176."""
+    33 = the shortest prefix that takes the path (a job of 17 tokens: jobs of up to 128 tokens take the product made
+    for few token rows, with token boxes of 16, 32, 64 or 128 rows), 64 and 65 = jobs of 48 and 64 tokens, 129 = 128
+    tokens, 145 = 129 tokens (the shortest job on the 128-token tiles), 293 = one job of 288 tokens (a last tile of
+    32), 700 = a job of 512 tokens and one of 176."""
     wl, _, _, _ = tiny_inputs
     prefix = si.make_prefix("zipf", m, wl.shape.vocab, 1.1, seed=500 + m)
     ctx, orc = make_tiny_pair(tiny_inputs, max_pos=1024, kv_dtype=kv_dtype)
@@ -186,8 +188,8 @@ def test_long_context_decode_7b_width():
 
 
 def test_prefix_of_64_tokens_13b_width():
-    """A 64-token prefix at the 13B shape's width: four launches of the 16-token kernel (the longest prefix that
-    does not take the long-prefix path), five drafts, then decode steps."""
+    """A 64-token prefix at the 13B shape's width (the fifth workload's prefix): a long-prefix job of 48 tokens on the
+    product made for few token rows, then one launch of the 16-token kernel; five drafts, then decode steps."""
     import torch
     import paper_2405_18400_b200 as P
     from oracle import spd_oracle as so
@@ -207,7 +209,7 @@ def test_prefix_of_64_tokens_13b_width():
     prefix = si.make_prefix("zipf", 64, shape.vocab, 1.05, seed=43)
     stats = []
     compare_first_step(ctx, orc, prefix, stats)
-    assert ctx.spd_launch_count() == 4
+    assert ctx.spd_launch_count() == 9 * shape.n_layers + 1
     for _ in range(3):
         compare_step(ctx, orc, stats)
     assert max(s["eps_z"] for s in stats if "eps_z" in s) < 2e-3

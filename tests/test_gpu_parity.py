@@ -80,10 +80,11 @@ def test_long_context_uses_split_attention(tiny_inputs):
 @pytest.mark.parametrize("m", [1, 2, 16, 17, 18, 33, 49])
 def test_prefill_chunk_boundaries(tiny_inputs, m):
     """The batched prefill takes 16 prefix tokens per launch, the last launch ending with the LM head and the
-    first timestep: prefix lengths around those boundaries (one token, a full launch, one token over, several)."""
+    first timestep: prefix lengths around those boundaries (one token, a full launch, one token over, several).  A
+    context of 128 positions has no long-prefix buffers, so every token goes through this kernel."""
     wl, _, _, _ = tiny_inputs
     prefix = si.make_prefix("zipf", m, wl.shape.vocab, 1.1, seed=30 + m)
-    ctx, orc = make_tiny_pair(tiny_inputs)
+    ctx, orc = make_tiny_pair(tiny_inputs, max_pos=128)
     compare_first_step(ctx, orc, prefix)
     assert ctx.spd_launch_count() == (m + 15) // 16
     compare_step(ctx, orc)
