@@ -257,16 +257,11 @@ __global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const 
   __syncthreads();
   Blk b;
   b.p = &p;
-  b.ring = nullptr;
   b.part = reinterpret_cast<float *>(bt_smem);
-  b.full = b.empty = nullptr;
-  b.red = nullptr;
   b.dead = &s_dead;
   b.quit = &s_quit;
   b.bar_target = 0;
   b.c_stage = b.c_phase = 0;
-  b.rope_s = nullptr;
-  b.gain_ptrs = nullptr;
   tail_score_select(b, false, p.st->n_gen);
 }
 

@@ -5,9 +5,12 @@
 // (contiguous row ranges of every matrix, in the order the decoder uses them) and streams them
 // into a shared-memory ring with bulk asynchronous copies that signal mbarriers; because weights do
 // not depend on activations it runs ahead across phase boundaries and across timesteps, so HBM
-// stays busy while the consumers exchange activation vectors through L2 at grid barriers.  The
-// consumers split the columns of each row among all threads (the activation slice of a thread stays
-// in registers for a whole phase), reduce with shuffles, and finish rows in per-phase epilogues
+// stays busy while the consumers exchange activation vectors through L2 at grid barriers.  Matrices
+// that also come in fragment order (spd_pack_image) are multiplied on the tensor cores: mma.sync over
+// 8-row units whose 16-byte vectors are the instruction's weight registers, x as three exact bf16 terms
+// kept as fragments in shared memory.  For the others the consumers split the columns of each row among
+// all threads (the activation slice of a thread stays in registers for a whole phase) and reduce with
+// shuffles.  Rows are finished in per-phase epilogues
 // (rotary embedding + cache append, residual add, SwiGLU, logits + block-level top-k).  Block 0 then
 // runs the method's tail: KeepTopK over the whole vocabulary, the k*k expansion with n-gram hash
 // probes (Eq. 5), the interpolation (Eq. 6/7), the selection of the k best options (Eq. 2) and the
@@ -149,9 +152,8 @@ __device__ __forceinline__ void produce_image(Blk &b, Producer &pr, const __nv_b
   }
 }
 
-template <bool kSampler, int kImgs>
+template <bool kSampler, bool kImg>
 __device__ void producer_main(Blk &b) {
-  constexpr bool kImg = kImgs > 0;
   const KParams &p = *b.p;
   Producer pr{0u, 0u, 0u};
   // The layers' pointers sit in device memory that the weight stream has long pushed out of L2 when their turn
@@ -895,12 +897,11 @@ __device__ void sample_windows(const KParams &p, int it) {
 }
 
 // ---------------------------------------------------------------- consumer main loop
-// kImgs > 0: QKV, attention output, gate / up and LM head also come in fragment order: a prologue leaves x
+// kImg: QKV, attention output, gate / up and LM head also come in fragment order: a prologue leaves x
 // in shared memory as fragments (store_frags; the barrier after it orders the stores before the first instruction
 // that reads them) and consume_image multiplies.
-template <bool kSampler, int kImgs>
+template <bool kSampler, bool kImg>
 __device__ void consumer_main(Blk &b) {
-  constexpr bool kImg = kImgs > 0;
   const KParams &p = *b.p;
   float xr[kMaxVec][8];
   // Everything a phase needs besides the activations is asked for at least a phase ahead (the gains of the RMSNorms,
@@ -1000,17 +1001,11 @@ __device__ void consumer_main(Blk &b) {
   }
 }
 
-template <bool kSampler, int kImgs>
+template <bool kSampler, bool kImg>
 __device__ __forceinline__ void kernel_body(const KParams &p) {
   Blk b;
   b.p = &p;
-  b.ring = smem;
   b.part = reinterpret_cast<float *>(smem + (size_t)p.n_stages * p.stage_bytes);
-  b.full = s_full;
-  b.empty = s_empty;
-  b.red = s_red;
-  b.rope_s = s_rope;
-  b.gain_ptrs = s_gain_ptrs;
   if (p.mode != kModeScoreOnly && p.mode != kModeNucleusOnly && 2 * p.L + 1 <= kGainSlots)
     for (int j = threadIdx.x; j <= 2 * p.L; j += kThreads)
       s_gain_ptrs[j] = j == 2 * p.L ? p.final_norm : ((j & 1) ? p.layers[j >> 1].ffn_norm : p.layers[j >> 1].attn_norm);
@@ -1041,27 +1036,27 @@ __device__ __forceinline__ void kernel_body(const KParams &p) {
     return;
   }
   if (threadIdx.x >= kConsumerThreads) {
-    if (threadIdx.x == kConsumerThreads) producer_main<kSampler, kImgs>(b);
+    if (threadIdx.x == kConsumerThreads) producer_main<kSampler, kImg>(b);
   } else {
-    consumer_main<kSampler, kImgs>(b);
+    consumer_main<kSampler, kImg>(b);
   }
   __syncthreads();
 }
 
 // The decoding kernel, and its twin that also carries the nucleus sampler (kModeSample, kModeNucleusOnly): two
 // entry points so that the sampler's code does not weigh on the register allocation of the decode loop.
-__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) { kernel_body<false, 0>(p); }
-__global__ void __launch_bounds__(kThreads, 1) spd_sample_kernel(const __grid_constant__ KParams p) { kernel_body<true, 0>(p); }
+__global__ void __launch_bounds__(kThreads, 1) spd_decode_kernel(const __grid_constant__ KParams p) { kernel_body<false, false>(p); }
+__global__ void __launch_bounds__(kThreads, 1) spd_sample_kernel(const __grid_constant__ KParams p) { kernel_body<true, false>(p); }
 // The decoding kernel for weights that also come in fragment order: QKV, attention output, gate / up and LM head
 // products on the tensor cores.  The down projection stays with the float32 multiply loop: its rows are long, so whole
 // units of them divide unevenly among the blocks and their fragments of x would take a third of the ring's memory
 // (measured: 2.96 ms per 7B timestep with it on the tensor cores too, against 2.64 ms).
-__global__ void __launch_bounds__(kThreads, 1) spd_decode_img_kernel(const __grid_constant__ KParams p) { kernel_body<false, 1>(p); }
+__global__ void __launch_bounds__(kThreads, 1) spd_decode_img_kernel(const __grid_constant__ KParams p) { kernel_body<false, true>(p); }
 
 }  // namespace spd
 
 // Host-side launcher used by the API file.
-static const void *kernel_for(int mode, int img) {
+static const void *kernel_for(int mode, bool img) {
   if (mode == spd::kModeSample || mode == spd::kModeNucleusOnly) return reinterpret_cast<const void *>(&spd::spd_sample_kernel);
   return img ? reinterpret_cast<const void *>(&spd::spd_decode_img_kernel) : reinterpret_cast<const void *>(&spd::spd_decode_kernel);
 }
@@ -1073,7 +1068,7 @@ extern "C" cudaError_t spd_internal_launch(const spd::KParams *p, int grid, size
 
 extern "C" cudaError_t spd_internal_prepare(size_t dyn_smem, int *blocks_per_sm) {
   int least = 1 << 30;
-  const void *kernels[3] = {kernel_for(spd::kModeDecode, 0), kernel_for(spd::kModeDecode, 1), kernel_for(spd::kModeSample, 0)};
+  const void *kernels[3] = {kernel_for(spd::kModeDecode, false), kernel_for(spd::kModeDecode, true), kernel_for(spd::kModeSample, false)};
   for (const void *kernel : kernels) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_smem);
     if (e != cudaSuccess) return e;

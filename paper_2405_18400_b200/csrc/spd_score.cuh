@@ -17,17 +17,12 @@ constexpr uint32_t kSkipped = 0xffffffffu;  // in the count / total arrays: this
 // ---------------------------------------------------------------- block context
 struct Blk {
   const KParams *p;
-  uint8_t *ring;
-  float *part;       // [2][kTile][kConsumerWarps]
-  uint64_t *full, *empty;
-  float *red;        // [64] reduction scratch
+  float *part;       // scratch of the scoring stage (the decode kernel's row partials live there between steps)
   volatile int *dead;
   volatile int *quit;  // block-uniform copy of *dead, refreshed inside every grid barrier
   unsigned int bar_target;
   // consumer ring cursor
   uint32_t c_stage, c_phase;
-  float2 *rope_s;    // decode kernel: the current position's row of the rotary table
-  const __nv_bfloat16 *const *gain_ptrs;  // decode kernel: the RMSNorm gains' pointers in the order a timestep uses them
 };
 
 __device__ __forceinline__ void give_up(Blk &b, int code, int info) {
