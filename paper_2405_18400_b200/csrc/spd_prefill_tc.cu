@@ -829,9 +829,17 @@ cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size
                               spd::State *st, cudaStream_t s) {
   using S = spd::BgShape<NP>;
   const size_t smem = (size_t)S::kStages * S::kStageBytes + 1024;
-  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_batch_gemm_kernel<NP>),
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  // the shared-memory attribute is per device: set on a device's first launch of this instance
+  static bool ready[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !ready[dev]) {
+    e = cudaFuncSetAttribute(reinterpret_cast<const void *>(&spd::spd_batch_gemm_kernel<NP>), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) ready[dev] = true;
+  }
   spd::spd_batch_gemm_kernel<NP><<<dim3((N + spd::kTcN - 1) / spd::kTcN, nz), spd::kTcThreads, smem, s>>>(xmap, wmap, Y, zs, n_tok, N, C,
                                                                                                             x_term_rows, st);
   return cudaGetLastError();

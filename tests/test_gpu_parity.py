@@ -489,3 +489,30 @@ def test_stop_token_ends_the_run(tiny_inputs):
     toks2, _, _ = ctx2.spd_generate(want_steps, 1 + want_steps)
     assert np.array_equal(toks2, want) and not ctx2.spd_finished()
     ctx.close(); ctx2.close()
+
+
+def test_image_and_row_major_paths_agree_at_7b_width():
+    """Two layers at the 7B shape's width (4096 / 11008 columns, head size 128): the decode steps of a context with
+    fragment-order weight images (tensor-core multiply, 8-row units, two stages per unit) and of one without (float32
+    loop for every matrix) give the same drafts and logits that differ by float rounding only."""
+    import paper_2405_18400_b200 as P
+
+    shape = si.ModelShape("w7b", 2, 4096, 32, 11008, 2000)
+    dev = torch.device("cuda:0")
+    weights = si.make_weights(shape, seed=61, device=dev)
+    tables = si.make_ngram_tables(shape.vocab, 1.1, 100_000, (2, 3, 4, 5, 6), 5000, seed=62)
+    lam = [0.01, 0.04, 0.15, 0.18, 0.12, 0.0, 0.0, 0.0]
+    dtabs = P.build_ngram_tables(tables, dev)
+    prefix = si.make_prefix("zipf", 15, shape.vocab, 1.1, seed=63)
+    out = []
+    for images in (True, False):
+        packed = P.pack_weights(weights, dev, images=images)
+        assert ("lm_head_img" in packed) == images
+        ctx = P.SpdContext(shape, packed, dtabs, 3, (2, 3, 4, 5, 6), lam, 0.54, 0.06, 0.01, 192, "bf16")
+        ctx.spd_prefill(prefix)
+        toks, lp, g = ctx.spd_generate(6, 7)
+        out.append((toks, lp, g, ctx.spd_debug_read("LOGITS")))
+        ctx.close()
+    assert np.array_equal(out[0][0], out[1][0])
+    assert np.abs(out[0][3] - out[1][3]).max() < 1e-4
+    assert np.abs(out[0][2] - out[1][2]).max() < 1e-4
