@@ -508,7 +508,9 @@ def test_image_and_row_major_paths_agree_at_7b_width():
     for images in (True, False):
         packed = P.pack_weights(weights, dev, images=images)
         assert ("lm_head_img" in packed) == images
-        ctx = P.SpdContext(shape, packed, dtabs, 3, (2, 3, 4, 5, 6), lam, 0.54, 0.06, 0.01, 192, "bf16")
+        # a float32 cache: with a bf16 cache the two paths' float differences flip cache roundings, which six
+        # free-running steps carry forward (9e-4 on the logits)
+        ctx = P.SpdContext(shape, packed, dtabs, 3, (2, 3, 4, 5, 6), lam, 0.54, 0.06, 0.01, 192, "f32")
         ctx.spd_prefill(prefix)
         toks, lp, g = ctx.spd_generate(6, 7)
         out.append((toks, lp, g, ctx.spd_debug_read("LOGITS")))
