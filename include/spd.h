@@ -342,6 +342,13 @@ int64_t spd_launch_count(const spd_ctx *ctx);
  * would overflow. */
 int spd_set_ring(spd_ctx *ctx, int32_t stage_bytes, int32_t n_stages);
 
+/* The ring spd_create chooses for a model (host only, no device needed): bytes per stage and stages of the decode
+ * kernel's weight ring, for a context whose weights come with fragment-order images (with_images != 0) or without.
+ * A stage takes two of the model's longest rows when four such stages fit beside the scratch area (and, with
+ * images, the fragments of x), else one row (rows over 16 KB) or 32 KB.  SPD_EINVAL for an invalid configuration or
+ * a row that fits no ring. */
+int spd_ring_plan(const spd_config *cfg, int32_t with_images, int32_t *stage_bytes, int32_t *n_stages);
+
 #ifdef __cplusplus
 }
 #endif

@@ -67,7 +67,7 @@ _lib: Optional[C.CDLL] = None
 EXPORTS = ["spd_workspace_bytes", "spd_create", "spd_prefill", "spd_step", "spd_generate", "spd_generate_async",
            "spd_sync", "spd_destroy", "spd_strerror", "spd_last_cuda_error", "spd_ngram_plan", "spd_ngram_build",
            "spd_debug_read", "spd_debug_score", "spd_launch_count", "spd_set_ring", "spd_score_static", "spd_reset",
-           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished", "spd_batch_generate", "spd_batch_step", "spd_pack_image"]
+           "spd_sample", "spd_debug_nucleus", "spd_debug_expire", "spd_debug_expire_products", "spd_debug_trace", "spd_finished", "spd_batch_generate", "spd_batch_step", "spd_pack_image", "spd_ring_plan"]
 
 
 def load_library() -> C.CDLL:
@@ -112,6 +112,7 @@ def load_library() -> C.CDLL:
     L.spd_batch_step.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.spd_debug_expire_products.argtypes = [C.c_void_p]
     L.spd_pack_image.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    L.spd_ring_plan.argtypes = [C.POINTER(SpdConfig), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.spd_launch_count.restype = C.c_int64
     L.spd_launch_count.argtypes = [C.c_void_p]
     L.spd_set_ring.argtypes = [C.c_void_p, C.c_int32, C.c_int32]

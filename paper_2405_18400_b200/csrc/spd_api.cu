@@ -541,6 +541,11 @@ int spd_destroy(spd_ctx *ctx) {
   return SPD_OK;
 }
 
+int spd_ring_plan(const spd_config *cfg, int32_t with_images, int32_t *stage_bytes, int32_t *n_stages) {
+  if (!valid_config(cfg) || !stage_bytes || !n_stages) return SPD_EINVAL;
+  return pick_ring(*cfg, 0, 0, with_images ? frag_bytes(*cfg) : 0, stage_bytes, n_stages);
+}
+
 int spd_set_ring(spd_ctx *ctx, int32_t stage_bytes, int32_t n_stages) {
   if (!ctx) return SPD_EINVAL;
   int32_t sb, ns;

@@ -109,3 +109,21 @@ def test_no_cpu_path():
     fake = {"tok_emb": torch.zeros(2, 2)}
     with pytest.raises(RuntimeError):
         P.SpdContext(wl.shape, fake, [], 3, wl.orders, wl.lambdas(), 0.5, 0.1, 0.01, 64)
+
+
+def test_ring_plan(lib):
+    """The decode kernel's default ring: two of the longest rows per stage when four such stages fit, else one row;
+    the fragments of x (192 bytes per 32 columns of d_model) come out of the ring's room when there are images."""
+    def plan(images, **kw):
+        sb, ns = C.c_int32(), C.c_int32()
+        assert lib.spd_ring_plan(C.byref(_cfg(**kw)), 1 if images else 0, C.byref(sb), C.byref(ns)) == 0
+        return sb.value, ns.value
+    big = dict(n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000, max_pos=4096)
+    assert plan(True, **big) == (44032, 4) and plan(False, **big) == (44032, 4)           # 2 x 22016 bytes (a multiple of 1 KB)
+    wide = dict(n_layers=40, d_model=5120, n_heads=40, d_ffn=13824, vocab=32000, max_pos=4096)
+    assert plan(True, **wide) == (27648, 6) and plan(False, **wide) == (27648, 7)         # four two-row stages do not fit
+    assert plan(True)[0] == 32768 and plan(False)[0] == 32768                             # short rows: 32 KB stages
+    for images in (False, True):
+        sb, ns = plan(images, **big)
+        assert sb * ns + 20480 + (4096 // 32 * 192 if images else 0) + 4096 <= 232448     # within the 227 KB of a block
+    assert lib.spd_ring_plan(C.byref(_cfg(k=0)), 0, C.byref(C.c_int32()), C.byref(C.c_int32())) == -1
