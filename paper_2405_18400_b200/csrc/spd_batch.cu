@@ -67,6 +67,8 @@ __device__ __forceinline__ int bt_pos(const KParams &p) { return p.pos0 + p.st->
 // the request's residual row; h * gain of the first layer's norm as three bf16 terms; the chunk's sum of squares.
 __global__ void __launch_bounds__(256) spd_batch_input_kernel(const KParams *kps, float *h, const __nv_bfloat16 *gain, uint16_t *X,
                                                               size_t term_stride, int d, float *ss) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   __shared__ float scratch[8];
   const KParams &p = kps[blockIdx.x];
   const State *st = p.st;
@@ -90,6 +92,8 @@ __global__ void __launch_bounds__(256) spd_batch_input_kernel(const KParams *kps
 // of the next norm as terms, the chunk's sum of squares.
 __global__ void __launch_bounds__(256) spd_batch_resid_kernel(float *h, const float *y, int nz, size_t zs, const __nv_bfloat16 *gain, uint16_t *X,
                                                               size_t term_stride, int d, float *ss) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   __shared__ float scratch[8];
   float sq = 0.f;
 #pragma unroll
@@ -112,6 +116,8 @@ __global__ void __launch_bounds__(256) spd_batch_resid_kernel(float *h, const fl
 // (adjacent pairs) at the request's own position, q to Q, k and v into the request's own cache.  Y row = [q | k | v].
 __global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, float *Q,
                                                                    const KParams *kps, int d, int hd, int layer) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   const KParams &p = kps[blockIdx.x];
   const int t = blockIdx.x, pos = bt_pos(p);
   const int i = blockIdx.y * 256 + threadIdx.x;  // column pair
@@ -145,6 +151,8 @@ __global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *
 // (Y row = [gate_0, up_0, gate_1, up_1, ...]), as three bf16 terms.
 __global__ void __launch_bounds__(256) spd_batch_swiglu_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, int d, uint16_t *X,
                                                                size_t term_stride, int f) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   const int t = blockIdx.x, j = blockIdx.y * 256 + threadIdx.x;
   if (j >= f) return;
   const float rs = bt_rs(ss, t, d, eps);
@@ -163,6 +171,8 @@ __global__ void __launch_bounds__(256) spd_batch_swiglu_kernel(const float *Y, i
 // per position with an online softmax, the warps' states merged in shared memory; output as three bf16 terms.
 __global__ void __launch_bounds__(128) spd_batch_attn_kernel(const float *Q, const KParams *kps, uint16_t *X, size_t term_stride, int d,
                                                              int hd, int layer) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   __shared__ float s_acc[4][256];
   __shared__ float s_m[4], s_l[4];
   const KParams &p = kps[blockIdx.x];
@@ -234,6 +244,8 @@ __global__ void __launch_bounds__(128) spd_batch_attn_kernel(const float *Q, con
 // Eq. 4 on the request's own draft state, as block 0 of the single-request kernel does.
 __global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const KParams *kps, const float *Y, int nz, size_t zs, const float *ss,
                                                                           float eps, int V) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   extern __shared__ __align__(16) uint8_t bt_smem[];
   __shared__ int s_dead, s_quit;
   const KParams &p = kps[blockIdx.x];
@@ -290,41 +302,37 @@ extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd:
   auto gemm = [&](const uint8_t *xmap, int which, float *Y, size_t room, int N, int C) {
     if (e != cudaSuccess) return;
     const uint8_t *wmap = j.w_tmaps + (size_t)which * spd::kTensorMapBytes;
-    e = spd_internal_batch_gemm(j.x_tmaps, xmap != xmap_d, wmap, Y, room, n, N, C, j.x_term_rows, j.st, sm_count, s, &nz, &zs);
+    e = spd_internal_batch_gemm(j.x_tmaps, xmap != xmap_d, wmap, Y, room, n, N, C, j.x_term_rows, j.st, sm_count, s, 1, &nz, &zs);
     ++count;
   };
   const int nch = (d + spd::kBtCols - 1) / spd::kBtCols;
   auto resid = [&](const __nv_bfloat16 *gain) {
     if (e != cudaSuccess) return;
-    spd::spd_batch_resid_kernel<<<dim3(n, nch), 256, 0, s>>>(j.h, j.y, nz, zs, gain, j.x, ts_d, d, ss);
-    e = cudaGetLastError();
+    e = spd::launch_dep(spd::spd_batch_resid_kernel, dim3(n, nch), dim3(256), 0, s, j.h, j.y, nz, zs, gain, j.x, ts_d, d, ss);
     ++count;
   };
-  spd::spd_batch_input_kernel<<<dim3(n, nch), 256, 0, s>>>(kps, j.h, j.layers[0].attn_norm, j.x, ts_d, d, ss);
-  e = cudaGetLastError();
+  e = spd::launch_dep(spd::spd_batch_input_kernel, dim3(n, nch), dim3(256), 0, s, kps, j.h, j.layers[0].attn_norm, j.x, ts_d, d, ss);
   ++count;
   for (int l = 0; l < j.L && e == cudaSuccess; ++l) {
     gemm(xmap_d, 4 * l, j.y, y_floats, 3 * d, d);
     if (e != cudaSuccess) break;
-    spd::spd_batch_rope_cache_kernel<<<dim3(n, (d / 2 + 255) / 256), 256, 0, s>>>(j.y, nz, zs, ss, j.eps, j.q, kps, d, j.hd, l);
-    if ((e = cudaGetLastError()) != cudaSuccess) break;
-    spd::spd_batch_attn_kernel<<<dim3(n, j.H), 128, 0, s>>>(j.q, kps, j.x, ts_d, d, j.hd, l);
-    if ((e = cudaGetLastError()) != cudaSuccess) break;
+    e = spd::launch_dep(spd::spd_batch_rope_cache_kernel, dim3(n, (d / 2 + 255) / 256), dim3(256), 0, s, j.y, nz, zs, ss, j.eps, j.q, kps, d, j.hd, l);
+    if (e != cudaSuccess) break;
+    e = spd::launch_dep(spd::spd_batch_attn_kernel, dim3(n, j.H), dim3(128), 0, s, j.q, kps, j.x, ts_d, d, j.hd, l);
+    if (e != cudaSuccess) break;
     count += 2;
     gemm(xmap_d, 4 * l + 1, j.y, y_floats, d, d);
     resid(j.layers[l].ffn_norm);
     gemm(xmap_d, 4 * l + 2, j.y, y_floats, 2 * f, d);
     if (e != cudaSuccess) break;
-    spd::spd_batch_swiglu_kernel<<<dim3(n, (f + 255) / 256), 256, 0, s>>>(j.y, nz, zs, ss, j.eps, d, j.x, ts_f, f);
-    e = cudaGetLastError();
+    e = spd::launch_dep(spd::spd_batch_swiglu_kernel, dim3(n, (f + 255) / 256), dim3(256), 0, s, j.y, nz, zs, ss, j.eps, d, j.x, ts_f, f);
     ++count;
     gemm(xmap_f, 4 * l + 3, j.y, y_floats, d, f);
     resid(l + 1 < j.L ? j.layers[l + 1].attn_norm : final_norm);
   }
   gemm(xmap_d, 4 * j.L, y_logits, y_logits_floats, V, d);
   if (e == cudaSuccess) {
-    spd::spd_batch_tail_kernel<<<n, spd::kConsumerThreads, kBatchTailSmem, s>>>(kps, y_logits, nz, zs, ss, j.eps, V);
-    e = cudaGetLastError();
+    e = spd::launch_dep(spd::spd_batch_tail_kernel, dim3(n), dim3(spd::kConsumerThreads), kBatchTailSmem, s, kps, y_logits, nz, zs, ss, j.eps, V);
     ++count;
   }
   if (launches) *launches = count;

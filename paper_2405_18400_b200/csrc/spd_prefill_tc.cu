@@ -271,6 +271,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 // (Y + y * split_stride), which the kernels that read Y add up in a fixed order.  Accumulators as in
 // spd_tc_gemm_kernel: four sets of NP tensor-memory columns in rotation, each the sum of 8 stages, added in registers
 // with round-to-nearest.  Every wait is bounded.
+// Launched as a programmatic dependent (a batched timestep), a block is set up and copies the weights of its first
+// stages while the kernel before it still runs; the terms, which that kernel writes, are asked for after dep_wait.
 template <int NP>
 struct BgShape {
   static constexpr int kTermBytes = NP * kTcKB * 2;                 // one term tile: NP token rows x 64 columns
@@ -294,6 +296,7 @@ __global__ void __launch_bounds__(kTcThreads)
   const int kb_lo = (int)((long long)nk_all * blockIdx.y / gridDim.y), kb_hi = (int)((long long)nk_all * (blockIdx.y + 1) / gridDim.y);
   const int nk = kb_hi - kb_lo;
   const int n0 = blockIdx.x * kTcN;
+  dep_launch();
   if (threadIdx.x == 0) {
     sh.dead = 0;
     for (int s = 0; s < S::kStages; ++s) {
@@ -317,7 +320,26 @@ __global__ void __launch_bounds__(kTcThreads)
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, issued = 0;
       bool ok = true;
-      for (int ks = 0; ks < nk; ++ks) {
+      // the first round of the ring: every stage is free; the weights go first, the terms once they are written
+      const int first = nk < S::kStages ? nk : S::kStages;
+      for (int ks = 0; ks < first; ++ks) {
+        mbar_expect_tx(&sh.full[ks], (uint32_t)S::kStageBytes);
+        const uint32_t base = ring + (uint32_t)ks * (uint32_t)S::kStageBytes;
+#pragma unroll
+        for (int j = 0; j < kTcN / kTcWBoxRows; ++j)
+          tc_box_load(base + j * (kTcWBoxRows * kTcKB * 2), tmap_w, (kb_lo + ks) * kTcKB, n0 + j * kTcWBoxRows, &sh.full[ks]);
+      }
+      dep_wait();
+      asm volatile("fence.proxy.async;" ::: "memory");  // the terms were written with ordinary stores
+      for (int ks = 0; ks < first; ++ks) {
+        const uint32_t base = ring + (uint32_t)ks * (uint32_t)S::kStageBytes;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) tc_box_load(base + kTcWBytes + j * S::kTermBytes, tmap_x, (kb_lo + ks) * kTcKB, j * x_term_rows, &sh.full[ks]);
+      }
+      issued = (uint32_t)first;
+      if (first == S::kStages) phase = 1u;
+      else stage = (uint32_t)first;
+      for (int ks = first; ks < nk; ++ks) {
         if (!tc_wait(sh, st, &sh.empty[stage], phase ^ 1u, 500)) { ok = false; break; }
         mbar_expect_tx(&sh.full[stage], (uint32_t)S::kStageBytes);
         const uint32_t base = ring + stage * (uint32_t)S::kStageBytes;
@@ -327,7 +349,6 @@ __global__ void __launch_bounds__(kTcThreads)
           tc_box_load(base + j * (kTcWBoxRows * kTcKB * 2), tmap_w, col, n0 + j * kTcWBoxRows, &sh.full[stage]);
 #pragma unroll
         for (int j = 0; j < 3; ++j) tc_box_load(base + kTcWBytes + j * S::kTermBytes, tmap_x, col, j * x_term_rows, &sh.full[stage]);
-        if (issued < (uint32_t)S::kStages) ++issued;
         if (++stage == (uint32_t)S::kStages) { stage = 0; phase ^= 1u; }
       }
       if (!ok) {
@@ -387,6 +408,7 @@ __global__ void __launch_bounds__(kTcThreads)
       if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
     }
     const int row = n0 + quarter * 32 + lane;
+    dep_wait();  // (long since true: the sums came from terms copied after the producer's dep_wait)
     if (ok && row < N) {
       float *out = Y + (size_t)blockIdx.y * split_stride + row;
 #pragma unroll
@@ -433,6 +455,8 @@ __device__ __forceinline__ float tc_block_sum(float v, float *scratch) {
 __global__ void __launch_bounds__(256) spd_tc_resid_norm_kernel(float *h, const float *y, const int32_t *ids, const __nv_bfloat16 *emb,
                                                                 const __nv_bfloat16 *gain, uint16_t *X, size_t term_stride, int d, float eps,
                                                                 int nz, size_t zs) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   __shared__ float scratch[8];
   const int t = blockIdx.x;
   float *hr = h + (size_t)t * d;
@@ -456,6 +480,8 @@ __global__ void __launch_bounds__(256) spd_tc_resid_norm_kernel(float *h, const 
 // token's position.  Y row = [q | k | v].
 __global__ void __launch_bounds__(256) spd_tc_rope_cache_kernel(const float *Y, float *Q, void *kcache, void *vcache, const float2 *rope,
                                                                 int d, int hd, int max_pos, int layer, int pos0, int kv_bf16, int nz, size_t zs) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   const int t = blockIdx.x, pos = pos0 + t;
   const float *yr = Y + (size_t)t * 3 * d;
   const size_t crow = ((size_t)layer * max_pos + pos) * d;
@@ -483,6 +509,8 @@ __global__ void __launch_bounds__(256) spd_tc_rope_cache_kernel(const float *Y, 
 
 // One token per block: u = SiLU(gate) * up from Y row = [gate_0, up_0, gate_1, up_1, ...], as three bf16 terms.
 __global__ void __launch_bounds__(256) spd_tc_swiglu_kernel(const float *Y, uint16_t *X, size_t term_stride, int f, int nz, size_t zs) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   const int t = blockIdx.x;
   const float2 *yr = reinterpret_cast<const float2 *>(Y + (size_t)t * 2 * f);
   for (int j = threadIdx.x; j < f; j += 256) {
@@ -505,6 +533,8 @@ __global__ void __launch_bounds__(256) spd_tc_swiglu_kernel(const float *Y, uint
 template <int HD>
 __global__ void __launch_bounds__(256) spd_tc_attn_kernel(const float *Q, const float *kcache, const float *vcache, uint16_t *X,
                                                           size_t term_stride, int d, int max_pos, int layer, int pos0, int n_tok) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   constexpr int kTok = 16, kPos = 32;
   constexpr int KS = HD + 4;    // key row stride in floats: 16-byte aligned, rows 4 banks apart
   constexpr int DPL = HD / 32;  // value dimensions per lane
@@ -648,6 +678,8 @@ __device__ __forceinline__ void tc_split3(float v, uint32_t &hi, uint32_t &mid, 
 template <int HD>
 __global__ void __launch_bounds__(128) spd_tc_attn_mma_kernel(const float *Q, const uint16_t *kcache, const uint16_t *vcache, uint16_t *X,
                                                               size_t term_stride, int d, int max_pos, int layer, int pos0, int n_tok) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
   constexpr int kTok = 64, kPos = 64;
   constexpr int RS = HD * 2 + 16;  // bytes per tile row
   constexpr int KS = HD / 16;      // k-steps over the head's dimensions
@@ -798,13 +830,11 @@ template <int HD>
 cudaError_t launch_attn(const spd::TcJob &j, int layer, int n_tok, cudaStream_t s) {
   const size_t ts = (size_t)j.x_term_rows * j.d;
   if (j.kv_bf16)
-    spd::spd_tc_attn_mma_kernel<HD><<<dim3((n_tok + 63) / 64, j.H), 128, attn_mma_smem<HD>(), s>>>(
-        j.q, static_cast<const uint16_t *>(j.kcache), static_cast<const uint16_t *>(j.vcache), j.x, ts, j.d, j.max_pos, layer, j.pos0, n_tok);
-  else
-    spd::spd_tc_attn_kernel<HD><<<dim3((n_tok + 15) / 16, j.H), 256, 0, s>>>(j.q, static_cast<const float *>(j.kcache),
-                                                                           static_cast<const float *>(j.vcache), j.x, ts, j.d, j.max_pos,
-                                                                           layer, j.pos0, n_tok);
-  return cudaGetLastError();
+    return spd::launch_dep(spd::spd_tc_attn_mma_kernel<HD>, dim3((n_tok + 63) / 64, j.H), dim3(128), attn_mma_smem<HD>(), s, j.q,
+                           static_cast<const uint16_t *>(j.kcache), static_cast<const uint16_t *>(j.vcache), j.x, ts, j.d, j.max_pos, layer, j.pos0,
+                           n_tok);
+  return spd::launch_dep(spd::spd_tc_attn_kernel<HD>, dim3((n_tok + 15) / 16, j.H), dim3(256), 0, s, j.q, static_cast<const float *>(j.kcache),
+                         static_cast<const float *>(j.vcache), j.x, ts, j.d, j.max_pos, layer, j.pos0, n_tok);
 }
 
 size_t tc_gemm_smem() { return (size_t)spd::kTcStages * spd::kTcStageBytes + 1024; }
@@ -826,7 +856,7 @@ extern "C" cudaError_t spd_internal_tc_prepare(void) {
 namespace {
 template <int NP>
 cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size_t zs, int nz, int n_tok, int N, int C, int x_term_rows,
-                              spd::State *st, cudaStream_t s) {
+                              spd::State *st, cudaStream_t s, int dep) {
   using S = spd::BgShape<NP>;
   const size_t smem = (size_t)S::kStages * S::kStageBytes + 1024;
   // the shared-memory attribute is per device: set on a device's first launch of this instance
@@ -840,8 +870,9 @@ cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) ready[dev] = true;
   }
-  spd::spd_batch_gemm_kernel<NP><<<dim3((N + spd::kTcN - 1) / spd::kTcN, nz), spd::kTcThreads, smem, s>>>(xmap, wmap, Y, zs, n_tok, N, C,
-                                                                                                            x_term_rows, st);
+  const dim3 grid((N + spd::kTcN - 1) / spd::kTcN, nz);
+  if (dep) return spd::launch_dep(spd::spd_batch_gemm_kernel<NP>, grid, dim3(spd::kTcThreads), smem, s, xmap, wmap, Y, zs, n_tok, N, C, x_term_rows, st);
+  spd::spd_batch_gemm_kernel<NP><<<grid, spd::kTcThreads, smem, s>>>(xmap, wmap, Y, zs, n_tok, N, C, x_term_rows, st);
   return cudaGetLastError();
 }
 }  // namespace
@@ -851,7 +882,7 @@ cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size
 // so that the product has about two blocks per SM, within y_floats of room for the partial sums); *out_nz and
 // *out_zs tell the reader of Y how many partial sums there are and how far apart.
 extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
-                                               int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int *out_nz, size_t *out_zs) {
+                                               int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int dep, int *out_nz, size_t *out_zs) {
   const int np = n_tok <= 16 ? 16 : (n_tok <= 32 ? 32 : (n_tok <= 64 ? 64 : 128));
   // the term buffer's tensor maps: boxes of 128 rows first, then 16, 32 and 64 (two each: d_model and d_ffn columns)
   const int slot = (np == 128 ? 0 : (np == 16 ? 1 : (np == 32 ? 2 : 3))) * 2 + (wide ? 1 : 0);
@@ -865,10 +896,10 @@ extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, c
   if (nz < 1) nz = 1;
   *out_nz = nz;
   *out_zs = zs;
-  if (np == 16) return launch_batch_gemm<16>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
-  if (np == 32) return launch_batch_gemm<32>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
-  if (np == 64) return launch_batch_gemm<64>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
-  return launch_batch_gemm<128>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s);
+  if (np == 16) return launch_batch_gemm<16>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s, dep);
+  if (np == 32) return launch_batch_gemm<32>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s, dep);
+  if (np == 64) return launch_batch_gemm<64>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s, dep);
+  return launch_batch_gemm<128>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s, dep);
 }
 
 // Test hook: one tile of the first layer's QKV product whose first stage never arrives (see the kernel's `stall`).
@@ -898,7 +929,7 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
     if (e != cudaSuccess) return;
     const uint8_t *wmap = j.w_tmaps + (size_t)which * spd::kTensorMapBytes;
     if (n <= spd::kTcM) {
-      e = spd_internal_batch_gemm(j.x_tmaps, xmap != xmap_d, wmap, j.y, j.y_floats, n, N, C, j.x_term_rows, j.st, j.sm_count, s, &nz, &zs);
+      e = spd_internal_batch_gemm(j.x_tmaps, xmap != xmap_d, wmap, j.y, j.y_floats, n, N, C, j.x_term_rows, j.st, j.sm_count, s, 1, &nz, &zs);
     } else {
       const dim3 grid((n + spd::kTcM - 1) / spd::kTcM, (N + spd::kTcN - 1) / spd::kTcN);
       spd::spd_tc_gemm_kernel<<<grid, spd::kTcThreads, tc_gemm_smem(), s>>>(xmap, wmap, j.y, N, C, j.x_term_rows, j.st, 0);
@@ -908,24 +939,23 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
   };
   auto resid = [&](const float *y, const int32_t *ids, const __nv_bfloat16 *gain) {
     if (e != cudaSuccess) return;
-    spd::spd_tc_resid_norm_kernel<<<n, 256, 0, s>>>(j.h, y, ids, j.tok_emb, gain, j.x, ts_d, d, j.eps, nz, zs);
-    e = cudaGetLastError();
+    e = spd::launch_dep(spd::spd_tc_resid_norm_kernel, dim3(n), dim3(256), 0, s, j.h, y, ids, j.tok_emb, gain, j.x, ts_d, d, j.eps, nz, zs);
     ++count;
   };
   resid(nullptr, j.ids, j.layers[0].attn_norm);
   for (int l = 0; l < j.L && e == cudaSuccess; ++l) {
     gemm(xmap_d, 4 * l, 3 * d, d);
     if (e != cudaSuccess) break;
-    spd::spd_tc_rope_cache_kernel<<<n, 256, 0, s>>>(j.y, j.q, j.kcache, j.vcache, j.rope, d, j.hd, j.max_pos, l, j.pos0, j.kv_bf16, nz, zs);
-    if ((e = cudaGetLastError()) != cudaSuccess) break;
+    e = spd::launch_dep(spd::spd_tc_rope_cache_kernel, dim3(n), dim3(256), 0, s, j.y, j.q, j.kcache, j.vcache, j.rope, d, j.hd, j.max_pos, l, j.pos0,
+                        j.kv_bf16, nz, zs);
+    if (e != cudaSuccess) break;
     e = j.hd == 128 ? launch_attn<128>(j, l, n, s) : launch_attn<64>(j, l, n, s);  // other head sizes never get here
     count += 2;
     gemm(xmap_d, 4 * l + 1, d, d);
     resid(j.y, nullptr, j.layers[l].ffn_norm);
     gemm(xmap_d, 4 * l + 2, 2 * f, d);
     if (e != cudaSuccess) break;
-    spd::spd_tc_swiglu_kernel<<<n, 256, 0, s>>>(j.y, j.x, ts_f, f, nz, zs);
-    e = cudaGetLastError();
+    e = spd::launch_dep(spd::spd_tc_swiglu_kernel, dim3(n), dim3(256), 0, s, j.y, j.x, ts_f, f, nz, zs);
     ++count;
     gemm(xmap_f, 4 * l + 3, d, f);
     if (l + 1 < j.L) resid(j.y, nullptr, j.layers[l + 1].attn_norm);  // the last layer's output feeds nothing here

@@ -29,11 +29,40 @@ struct TcJob {
   size_t y_floats;                   // room of y in floats (partial sums of a column-split product)
 };
 
+// Programmatic dependent launch.  dep_wait: returns once the kernel before this one in the stream has completed and
+// its writes are visible (at once when the launch did not ask for the overlap).  dep_launch: the kernel after this
+// one may be brought onto the SMs, where it runs up to its own dep_wait, as soon as every block of this kernel has
+// said so or has ended.
+#ifdef __CUDACC__
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
+// Launch with programmatic stream serialization: the kernel may be brought onto the SMs while the one before it in the
+// stream still runs, and waits there (dep_wait) until that one has completed.  The kernels launched this way start
+// with dep_wait (the small-batch product: before its first read of the terms), so that the launch latency, the
+// set-up of a block and the product's first weight copies overlap the tail of the kernel before.
+template <typename... P, typename... A>
+inline cudaError_t launch_dep(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
 }  // namespace spd
 
 extern "C" cudaError_t spd_internal_tc_prepare(void);
 extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);
-// The product of a batched timestep's few token rows.
+// The product of a batched timestep's few token rows.  dep: launch it so that it may start while the kernel before it
+// in the stream still runs (it then copies weights only, until that kernel has completed).
 extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
-                                               int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int *out_nz, size_t *out_zs);
+                                               int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int dep, int *out_nz, size_t *out_zs);
