@@ -277,8 +277,11 @@ template <int NP>
 struct BgShape {
   static constexpr int kTermBytes = NP * kTcKB * 2;                 // one term tile: NP token rows x 64 columns
   static constexpr int kStageBytes = kTcWBytes + 3 * kTermBytes;    // 128 weight rows x 64 columns, then the three term tiles
-  static constexpr int kStages = NP <= 16 ? 4 : (NP <= 32 ? 3 : (NP <= 64 ? 5 : 3));  // 91 KB and 87 KB: two blocks per SM; NP = 64:
-                                                                                     // 205 KB, NP = 128: 197 KB, one block
+  // Two blocks per SM wherever they fit (91, 87 and 83 KB for NP = 16, 32, 64; NP = 128: one block of 197 KB): one
+  // block's set-up and epilogue run beside the other's stages.  64 token rows with one block of five stages took
+  // 6.9 ms per 7B timestep, with two blocks of two stages 5.5 ms; three blocks of fewer stages for NP <= 32 were
+  // slower than two (4.4 against 4.0 ms for 8 requests).
+  static constexpr int kStages = NP <= 16 ? 4 : (NP <= 32 ? 3 : (NP <= 64 ? 2 : 3));
   static constexpr int kTmemCols = 4 * NP < 32 ? 32 : 4 * NP;
 };
 
