@@ -882,7 +882,7 @@ cudaError_t launch_batch_gemm(const void *xmap, const void *wmap, float *Y, size
 
 // Product of a batch (n_tok <= 128 token rows): xmaps = the term buffer's tensor maps with boxes of 128, 16, 32 and 64
 // rows (two each: d_model and d_ffn columns; `wide` picks the second).  The columns are split nz ways (chosen here
-// so that the product has about two blocks per SM, within y_floats of room for the partial sums); *out_nz and
+// for the fewest waves of blocks, within y_floats of room for the partial sums); *out_nz and
 // *out_zs tell the reader of Y how many partial sums there are and how far apart.
 extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
                                                int x_term_rows, spd::State *st, int sm_count, cudaStream_t s, int dep, int *out_nz, size_t *out_zs) {
@@ -892,11 +892,22 @@ extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, c
   const void *xmap = xmaps + (size_t)slot * spd::kTensorMapBytes;
   const int tiles = (N + spd::kTcN - 1) / spd::kTcN, nk = (C + spd::kTcKB - 1) / spd::kTcKB;
   const size_t zs = (size_t)n_tok * N;
-  int nz = (2 * sm_count + tiles / 2) / tiles;               // about two blocks per SM (64 token rows, one block per SM at a
-                                                              // time: 7.1 ms per 7B timestep against 8.6 ms with half as many)
-  if (nz > nk / 8) nz = nk / 8;                               // at least 8 stages of work per block
-  if ((size_t)nz * zs > y_floats) nz = (int)(y_floats / zs);  // room for the partial sums
-  if (nz < 1) nz = 1;
+  // The split that needs the fewest stage times: the blocks run in waves of as many as fit the GPU (two per SM, one
+  // with boxes of 128 rows), a block costs its stages plus about eight stages' worth of set-up, ring fill and epilogue,
+  // and a last wave that is nearly empty costs as much as a full one (the 7B gate / up product, 172 row tiles: two
+  // ways = 344 blocks = two waves of 32 stages, three ways = 516 blocks = two waves of 22).  At least 8 stages of
+  // work per block, and room for the partial sums.
+  const int slots = (np == 128 ? 1 : 2) * (sm_count > 0 ? sm_count : 1);
+  int nz_max = nk / 8;
+  if ((size_t)nz_max * zs > y_floats) nz_max = (int)(y_floats / zs);
+  if (nz_max < 1) nz_max = 1;
+  int nz = 1;
+  long best = -1;
+  for (int z = 1; z <= nz_max; ++z) {
+    const long waves = ((long)tiles * z + slots - 1) / slots;
+    const long cost = waves * ((nk + z - 1) / z + 8);
+    if (best < 0 || cost < best) { best = cost; nz = z; }
+  }
   *out_nz = nz;
   *out_zs = zs;
   if (np == 16) return launch_batch_gemm<16>(xmap, wmap, Y, zs, nz, n_tok, N, C, x_term_rows, st, s, dep);
