@@ -266,6 +266,7 @@ spd::TcJob tc_job(spd_ctx *ctx) {
   job.st = kp.st;
   job.sm_count = ctx->grid;
   job.y_floats = (size_t)ctx->tc_rows * (size_t)(3 * kp.d > 2 * kp.f ? 3 * kp.d : 2 * kp.f);
+  job.ss = reinterpret_cast<float *>(ctx->ws + ctx->lay.bt_ss);
   job.ids = nullptr;
   job.pos0 = job.n_tok = 0;
   return job;

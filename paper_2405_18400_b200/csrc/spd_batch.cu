@@ -112,20 +112,14 @@ __global__ void __launch_bounds__(256) spd_batch_resid_kernel(float *h, const fl
   if (threadIdx.x == 0) ss[blockIdx.x * kBtMaxChunks + blockIdx.y] = sq;
 }
 
-// grid (requests, chunks of 256 column pairs): the QKV product's row times 1 / rms, rotary embedding of q and k
-// (adjacent pairs) at the request's own position, q to Q, k and v into the request's own cache.  Y row = [q | k | v].
-__global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, float *Q,
-                                                                   const KParams *kps, int d, int hd, int layer) {
-  dep_wait();    // the kernel before this one in the stream wrote what this one reads
-  dep_launch();  // the next one may set itself up meanwhile
-  const KParams &p = kps[blockIdx.x];
-  const int t = blockIdx.x, pos = bt_pos(p);
-  const int i = blockIdx.y * 256 + threadIdx.x;  // column pair
-  if (i >= d / 2) return;
-  const float rs = bt_rs(ss, t, d, eps);
+// One column pair of one token row: the QKV product's row (the sum of its nz partial sums) times 1 / rms, rotary
+// embedding of q and k (adjacent pairs) at position pos, q to Q, k and v into the cache.  Y row = [q | k | v].
+__device__ __forceinline__ void bt_rope_cache_pair(const float *Y, int nz, size_t zs, float rs, float *Q, void *kcache, void *vcache,
+                                                   const float2 *rope, int max_pos, int kv_bf16, int d, int hd, int layer, int t, int pos,
+                                                   int i) {
   const float *yr = Y + (size_t)t * 3 * d;
-  const size_t crow = ((size_t)layer * p.max_pos + pos) * d;
-  const float2 cs = p.rope[(size_t)pos * (hd / 2) + (i % (hd / 2))];
+  const size_t crow = ((size_t)layer * max_pos + pos) * d;
+  const float2 cs = rope[(size_t)pos * (hd / 2) + (i % (hd / 2))];
   float2 qq = make_float2(0.f, 0.f), kk = qq, vv = qq;
   for (int z = 0; z < nz; ++z) {  // the product's partial sums over column ranges, in order
     const float *yz = yr + z * zs;
@@ -138,13 +132,60 @@ __global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *
   Q[(size_t)t * d + 2 * i + 1] = qe * cs.y + qo * cs.x;
   const float k0 = ke * cs.x - ko * cs.y, k1 = ke * cs.y + ko * cs.x;
   const float v0 = vv.x * rs, v1 = vv.y * rs;
-  if (p.kv_bf16) {
-    reinterpret_cast<__nv_bfloat162 *>(p.kcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(k0), __float2bfloat16_rn(k1));
-    reinterpret_cast<__nv_bfloat162 *>(p.vcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(v0), __float2bfloat16_rn(v1));
+  if (kv_bf16) {
+    reinterpret_cast<__nv_bfloat162 *>(kcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(k0), __float2bfloat16_rn(k1));
+    reinterpret_cast<__nv_bfloat162 *>(vcache)[(crow >> 1) + i] = __halves2bfloat162(__float2bfloat16_rn(v0), __float2bfloat16_rn(v1));
   } else {
-    reinterpret_cast<float2 *>(p.kcache)[(crow >> 1) + i] = make_float2(k0, k1);
-    reinterpret_cast<float2 *>(p.vcache)[(crow >> 1) + i] = make_float2(v0, v1);
+    reinterpret_cast<float2 *>(kcache)[(crow >> 1) + i] = make_float2(k0, k1);
+    reinterpret_cast<float2 *>(vcache)[(crow >> 1) + i] = make_float2(v0, v1);
   }
+}
+
+// grid (requests, chunks of 256 column pairs): each request at its own position, into its own cache.
+__global__ void __launch_bounds__(256) spd_batch_rope_cache_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, float *Q,
+                                                                   const KParams *kps, int d, int hd, int layer) {
+  dep_wait();    // the kernel before this one in the stream wrote what this one reads
+  dep_launch();  // the next one may set itself up meanwhile
+  const KParams &p = kps[blockIdx.x];
+  const int i = blockIdx.y * 256 + threadIdx.x;  // column pair
+  if (i >= d / 2) return;
+  bt_rope_cache_pair(Y, nz, zs, bt_rs(ss, blockIdx.x, d, eps), Q, p.kcache, p.vcache, p.rope, p.max_pos, p.kv_bf16, d, hd, layer, blockIdx.x,
+                     bt_pos(p), i);
+}
+
+// The same for a job of prefix tokens of one request (token t at position pos0 + t, one cache).
+__global__ void __launch_bounds__(256) spd_job_rope_cache_kernel(const float *Y, int nz, size_t zs, const float *ss, float eps, float *Q,
+                                                                 void *kcache, void *vcache, const float2 *rope, int max_pos, int kv_bf16, int d,
+                                                                 int hd, int layer, int pos0) {
+  dep_wait();
+  dep_launch();
+  const int i = blockIdx.y * 256 + threadIdx.x;
+  if (i >= d / 2) return;
+  bt_rope_cache_pair(Y, nz, zs, bt_rs(ss, blockIdx.x, d, eps), Q, kcache, vcache, rope, max_pos, kv_bf16, d, hd, layer, blockIdx.x,
+                     pos0 + blockIdx.x, i);
+}
+
+// grid (tokens, column chunks): a job's residual rows start as its tokens' embeddings; h * gain of the first layer's
+// norm as three bf16 terms; the chunk's sum of squares.
+__global__ void __launch_bounds__(256) spd_job_input_kernel(const int32_t *ids, const __nv_bfloat16 *tok_emb, float *h, const __nv_bfloat16 *gain,
+                                                            uint16_t *X, size_t term_stride, int d, float *ss) {
+  dep_wait();
+  dep_launch();
+  __shared__ float scratch[8];
+  const __nv_bfloat16 *row = tok_emb + (size_t)ids[blockIdx.x] * d;
+  float sq = 0.f;
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int c = blockIdx.y * kBtCols + e * 256 + threadIdx.x;
+    if (c < d) {
+      const float v = __bfloat162float(row[c]);
+      h[(size_t)blockIdx.x * d + c] = v;
+      sq = fmaf(v, v, sq);
+      bt_put3(X, term_stride, (size_t)blockIdx.x * d + c, v * __bfloat162float(gain[c]));
+    }
+  }
+  sq = bt_block_sum(sq, scratch);
+  if (threadIdx.x == 0) ss[blockIdx.x * kBtMaxChunks + blockIdx.y] = sq;
 }
 
 // grid (requests, chunks of 256 rows of the FFN): u = SiLU(gate) * up from the gate / up product's row times 1 / rms
@@ -337,4 +378,27 @@ extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd:
   }
   if (launches) *launches = count;
   return e;
+}
+
+// The row-wise kernels of a job of up to 128 prefix tokens of one request (the long-prefix path's small jobs): the same
+// column-parallel kernels as a batched timestep's, token t at position job.pos0 + t.  ss: [128][32] floats.
+extern "C" cudaError_t spd_internal_job_input(const spd::TcJob *job, float *ss, cudaStream_t s) {
+  const spd::TcJob &j = *job;
+  return spd::launch_dep(spd::spd_job_input_kernel, dim3(j.n_tok, (j.d + spd::kBtCols - 1) / spd::kBtCols), dim3(256), 0, s, j.ids, j.tok_emb, j.h,
+                         j.layers[0].attn_norm, j.x, (size_t)j.x_term_rows * j.d, j.d, ss);
+}
+extern "C" cudaError_t spd_internal_job_rope_cache(const spd::TcJob *job, float *ss, int nz, size_t zs, int layer, cudaStream_t s) {
+  const spd::TcJob &j = *job;
+  return spd::launch_dep(spd::spd_job_rope_cache_kernel, dim3(j.n_tok, (j.d / 2 + 255) / 256), dim3(256), 0, s, j.y, nz, zs, ss, j.eps, j.q, j.kcache,
+                         j.vcache, j.rope, j.max_pos, j.kv_bf16, j.d, j.hd, layer, j.pos0);
+}
+extern "C" cudaError_t spd_internal_job_resid(const spd::TcJob *job, float *ss, int nz, size_t zs, const __nv_bfloat16 *gain, cudaStream_t s) {
+  const spd::TcJob &j = *job;
+  return spd::launch_dep(spd::spd_batch_resid_kernel, dim3(j.n_tok, (j.d + spd::kBtCols - 1) / spd::kBtCols), dim3(256), 0, s, j.h, j.y, nz, zs, gain,
+                         j.x, (size_t)j.x_term_rows * j.d, j.d, ss);
+}
+extern "C" cudaError_t spd_internal_job_swiglu(const spd::TcJob *job, float *ss, int nz, size_t zs, cudaStream_t s) {
+  const spd::TcJob &j = *job;
+  return spd::launch_dep(spd::spd_batch_swiglu_kernel, dim3(j.n_tok, (j.f + 255) / 256), dim3(256), 0, s, j.y, nz, zs, ss, j.eps, j.d, j.x,
+                         (size_t)j.x_term_rows * j.f, j.f);
 }

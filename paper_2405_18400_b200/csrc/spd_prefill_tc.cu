@@ -951,6 +951,36 @@ extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream
     }
     ++count;
   };
+  if (n <= spd::kTcM) {
+    // ... and the column-parallel row-wise kernels of a batched timestep (a block per 512 columns of a token row
+    // instead of one per row; RMSNorm's 1 / rms applied behind the product from per-chunk sums of squares).
+    e = spd_internal_job_input(job, j.ss, s);
+    ++count;
+    for (int l = 0; l < j.L && e == cudaSuccess; ++l) {
+      gemm(xmap_d, 4 * l, 3 * d, d);
+      if (e != cudaSuccess) break;
+      e = spd_internal_job_rope_cache(job, j.ss, nz, zs, l, s);
+      if (e != cudaSuccess) break;
+      e = j.hd == 128 ? launch_attn<128>(j, l, n, s) : launch_attn<64>(j, l, n, s);
+      count += 2;
+      gemm(xmap_d, 4 * l + 1, d, d);
+      if (e != cudaSuccess) break;
+      e = spd_internal_job_resid(job, j.ss, nz, zs, j.layers[l].ffn_norm, s);
+      ++count;
+      gemm(xmap_d, 4 * l + 2, 2 * f, d);
+      if (e != cudaSuccess) break;
+      e = spd_internal_job_swiglu(job, j.ss, nz, zs, s);
+      ++count;
+      gemm(xmap_f, 4 * l + 3, d, f);
+      if (e != cudaSuccess) break;
+      if (l + 1 < j.L) {  // the last layer's output feeds nothing here
+        e = spd_internal_job_resid(job, j.ss, nz, zs, j.layers[l + 1].attn_norm, s);
+        ++count;
+      }
+    }
+    if (launches) *launches = count;
+    return e;
+  }
   auto resid = [&](const float *y, const int32_t *ids, const __nv_bfloat16 *gain) {
     if (e != cudaSuccess) return;
     e = spd::launch_dep(spd::spd_tc_resid_norm_kernel, dim3(n), dim3(256), 0, s, j.h, y, ids, j.tok_emb, gain, j.x, ts_d, d, j.eps, nz, zs);

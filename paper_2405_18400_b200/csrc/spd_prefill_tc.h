@@ -27,6 +27,7 @@ struct TcJob {
   State *st;
   int32_t sm_count;                  // SMs of the device
   size_t y_floats;                   // room of y in floats (partial sums of a column-split product)
+  float *ss;                         // [128][32]: sums of squares of the residual rows per 512-column chunk (jobs of up to 128 tokens)
 };
 
 // Programmatic dependent launch.  dep_wait: returns once the kernel before this one in the stream has completed and
@@ -62,6 +63,11 @@ inline cudaError_t launch_dep(void (*kernel)(P...), dim3 grid, dim3 block, size_
 extern "C" cudaError_t spd_internal_tc_prepare(void);
 extern "C" cudaError_t spd_internal_tc_stall(const spd::TcJob *job, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_tc_prefill(const spd::TcJob *job, cudaStream_t stream, int *launches);
+// Row-wise kernels of a job of up to 128 tokens (column-parallel, 1 / rms applied behind the product; spd_batch.cu).
+extern "C" cudaError_t spd_internal_job_input(const spd::TcJob *job, float *ss, cudaStream_t s);
+extern "C" cudaError_t spd_internal_job_rope_cache(const spd::TcJob *job, float *ss, int nz, size_t zs, int layer, cudaStream_t s);
+extern "C" cudaError_t spd_internal_job_resid(const spd::TcJob *job, float *ss, int nz, size_t zs, const __nv_bfloat16 *gain, cudaStream_t s);
+extern "C" cudaError_t spd_internal_job_swiglu(const spd::TcJob *job, float *ss, int nz, size_t zs, cudaStream_t s);
 // The product of a batched timestep's few token rows.  dep: launch it so that it may start while the kernel before it
 // in the stream still runs (it then copies weights only, until that kernel has completed).
 extern "C" cudaError_t spd_internal_batch_gemm(const uint8_t *xmaps, int wide, const void *wmap, float *Y, size_t y_floats, int n_tok, int N, int C,
