@@ -301,6 +301,9 @@ __global__ void __launch_bounds__(kTcThreads)
   const int n0 = blockIdx.x * kTcN;
   dep_launch();
   if (threadIdx.x == 0) {
+    // the two descriptors on their way before the first copies ask for them
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tmap_x) : "memory");
     sh.dead = 0;
     for (int s = 0; s < S::kStages; ++s) {
       mbar_init(&sh.full[s], 1);
