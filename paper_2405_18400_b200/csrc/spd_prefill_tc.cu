@@ -269,8 +269,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 // 48 KB of terms per 16 KB of weights), and the columns are split among blockIdx.y so that every product fills
 // the GPU: block (x, y) adds columns [64 kb_lo, 64 kb_hi) of rows 128 x .. 128 x + 127 into its own copy of Y
 // (Y + y * split_stride), which the kernels that read Y add up in a fixed order.  Accumulators as in
-// spd_tc_gemm_kernel: four sets of NP tensor-memory columns in rotation, each the sum of 8 stages, added in registers
-// with round-to-nearest.  Every wait is bounded.
+// spd_tc_gemm_kernel: sets of tensor-memory columns in rotation, each the sum of a segment of stages (96 additions),
+// fetched by the epilogue warps and added in registers with round-to-nearest (BgShape says how many sets and
+// stages for each box).  Every wait is bounded.
 // Launched as a programmatic dependent (a batched timestep), a block is set up and copies the weights of its first
 // stages while the kernel before it still runs; the terms, which that kernel writes, are asked for after dep_wait.
 template <int NP>
@@ -282,7 +283,20 @@ struct BgShape {
   // 6.9 ms per 7B timestep, with two blocks of two stages 5.5 ms; three blocks of fewer stages for NP <= 32 were
   // slower than two (4.4 against 4.0 ms for 8 requests).
   static constexpr int kStages = NP <= 16 ? 4 : (NP <= 32 ? 3 : (NP <= 64 ? 2 : 3));
-  static constexpr int kTmemCols = 4 * NP < 32 ? 32 : 4 * NP;
+  // Boxes of 16 and 32 rows: the three term tiles lie behind one another in a stage, 3 NP rows of one K-major operand,
+  // so one instruction of N = 3 NP per 16 columns multiplies all three (a third of the instructions; an instruction
+  // of N = 16 costs about as much as one of N = 48: 8 requests 3.63 -> 3.35 ms per 7B timestep).  Each term then has
+  // its own NP accumulator columns, added up in the epilogue's registers, and an accumulator may take three times
+  // as many stages for the same number of additions (96) before it is fetched.  Two blocks per SM share the 512
+  // columns of tensor memory, so a block has 256: four accumulator sets of 48 columns, two of 96, or one of 192
+  // (the product then waits while its sum is fetched, once or twice per block; the SM's other block does not).
+  // Boxes of 128 rows keep one instruction per term.
+  static constexpr bool kFused = NP <= 64;
+  static constexpr int kAccCols = kFused ? 3 * NP : NP;  // columns of one accumulator set
+  static constexpr int kAccs = NP == 32 ? 2 : (NP == 64 ? 1 : kTcAccs);  // accumulator sets in rotation
+  static constexpr int kSegSteps = kFused ? 3 * kTcSegSteps : kTcSegSteps;  // stages summed in one accumulator
+  static constexpr int kTmemCols = kFused ? 256 : 4 * NP;  // a power of two
+  static_assert(kAccs * kAccCols <= kTmemCols && kAccs <= kTcAccs, "the accumulator sets fit the allocation and the barrier arrays");
 };
 
 template <int NP>
@@ -370,22 +384,29 @@ __global__ void __launch_bounds__(kTcThreads)
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = tc_idesc(kTcN, NP);  // M = 128 weight rows, N = NP token rows
+      const uint32_t idesc = tc_idesc(kTcN, S::kAccCols);  // M = 128 weight rows, N = NP token rows (x 3 terms when fused)
       uint32_t stage = 0, phase = 0;
       for (int ks = 0; ks < nk; ++ks) {
-        const int seg = ks / kTcSegSteps, in_seg = ks - seg * kTcSegSteps, a = seg % kTcAccs;
-        if (in_seg == 0 && !tc_wait(sh, st, &sh.acc_empty[a], (uint32_t)((seg / kTcAccs) & 1) ^ 1u, 530)) break;
+        const int seg = ks / S::kSegSteps, in_seg = ks - seg * S::kSegSteps, a = seg % S::kAccs;
+        if (in_seg == 0 && !tc_wait(sh, st, &sh.acc_empty[a], (uint32_t)((seg / S::kAccs) & 1) ^ 1u, 530)) break;
         if (!tc_wait(sh, st, &sh.full[stage], phase, 510)) break;
         tc_fence_after();
         const uint32_t base = ring + stage * (uint32_t)S::kStageBytes;
-#pragma unroll
-        for (int j = 0; j < 3; ++j)
+        if constexpr (S::kFused) {
 #pragma unroll
           for (int kk = 0; kk < kTcKB / 16; ++kk)
-            tc_mma(tmem + (uint32_t)(a * NP), tc_desc(base + kk * 32), tc_desc(base + kTcWBytes + j * S::kTermBytes + kk * 32), idesc,
-                   (uint32_t)((in_seg | j | kk) != 0));
+            tc_mma(tmem + (uint32_t)(a * S::kAccCols), tc_desc(base + kk * 32), tc_desc(base + kTcWBytes + kk * 32), idesc,
+                   (uint32_t)((in_seg | kk) != 0));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 3; ++j)
+#pragma unroll
+            for (int kk = 0; kk < kTcKB / 16; ++kk)
+              tc_mma(tmem + (uint32_t)(a * S::kAccCols), tc_desc(base + kk * 32), tc_desc(base + kTcWBytes + j * S::kTermBytes + kk * 32), idesc,
+                     (uint32_t)((in_seg | j | kk) != 0));
+        }
         tc_commit(&sh.empty[stage]);
-        if (in_seg == kTcSegSteps - 1 || ks == nk - 1) tc_commit(&sh.acc_full[a]);
+        if (in_seg == S::kSegSteps - 1 || ks == nk - 1) tc_commit(&sh.acc_full[a]);
         if (++stage == (uint32_t)S::kStages) { stage = 0; phase ^= 1u; }
       }
     }
@@ -396,18 +417,18 @@ __global__ void __launch_bounds__(kTcThreads)
     float sum[NP];
 #pragma unroll
     for (int j = 0; j < NP; ++j) sum[j] = 0.f;
-    const int nseg = (nk + kTcSegSteps - 1) / kTcSegSteps;
+    const int nseg = (nk + S::kSegSteps - 1) / S::kSegSteps;
     bool ok = true;
     for (int seg = 0; seg < nseg; ++seg) {
-      const int a = seg % kTcAccs;
-      if (!tc_wait(sh, st, &sh.acc_full[a], (uint32_t)((seg / kTcAccs) & 1), 520)) { ok = false; break; }
+      const int a = seg % S::kAccs;
+      if (!tc_wait(sh, st, &sh.acc_full[a], (uint32_t)((seg / S::kAccs) & 1), 520)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll
-      for (int c0 = 0; c0 < NP; c0 += 16) {
+      for (int c0 = 0; c0 < S::kAccCols; c0 += 16) {  // (fused: the columns of term c0 / NP, added to the same tokens' sums)
         uint32_t r[16];
-        tc_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * NP + c0), r);
+        tc_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * S::kAccCols + c0), r);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) sum[c0 + j] += __uint_as_float(r[j]);
+        for (int j = 0; j < 16; ++j) sum[c0 % NP + j] += __uint_as_float(r[j]);
       }
       tc_fence_before();
       __syncwarp();
