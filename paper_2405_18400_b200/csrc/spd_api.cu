@@ -18,8 +18,8 @@ extern "C" cudaError_t spd_internal_prefill_prepare(int *blocks_per_sm);
 extern "C" cudaError_t spd_internal_prefill_launch(const spd::KParams *p, int grid, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_pack_image(const void *w, void *out, int rows, int cols, cudaStream_t stream);
 extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd::KParams *kps, int n, int V, const __nv_bfloat16 *final_norm,
-                                               float *y_logits, size_t y_floats, size_t y_logits_floats, float *ss, int sm_count,
-                                               cudaStream_t s, int *launches);
+                                               float *y_logits, size_t y_floats, size_t y_logits_floats, float *ss, int32_t *results,
+                                               int sm_count, cudaStream_t s, int *launches);
 
 namespace {
 
@@ -44,7 +44,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 struct Layout {
   size_t kcache, vcache, rope, layers, h, q, u, logits, opart, oml, pk_val, pk_id, pk_ms, state, hist_tok, hist_par, prefix,
       trace, ns_u, pf_tmaps, pf_h, pf_q, pf_ss, pf_part, pf_ml, pf_cnt, pf_xh, pf_xo, pf_xu, tc_tmaps, tc_h, tc_q, tc_y, tc_x, bt_kp, bt_y,
-      bt_ss, total;
+      bt_ss, bt_out, total;
 };
 
 // Tokens one long-prefix job takes at most (0: the context never runs one): prefixes of more than 64 tokens send
@@ -126,6 +126,7 @@ Layout make_layout(const spd_config &c, int grid) {
   L.bt_kp = take(tcr ? (size_t)spd::kTcTile * sizeof(spd::KParams) : 0);
   L.bt_y = take(tcr ? (size_t)spd::kTcTile * c.vocab * 4 : 0);
   L.bt_ss = take(tcr ? (size_t)spd::kTcTile * 32 * 4 : 0);  // per request and 512-column chunk: sums of squares of the residual row
+  L.bt_out = take(tcr ? (size_t)spd::kTcTile * spd::kBtResultWords * 4 : 0);  // per request: a timestep's results
   L.total = off;
   return L;
 }
@@ -813,7 +814,7 @@ int batch_enqueue(spd_ctx *const *ctxs, int32_t n, int32_t n_steps) {
     const cudaError_t e = spd_internal_batch_step(&job, dkp, n, c0.vocab, lead->kp.final_norm,
                                                   reinterpret_cast<float *>(lead->ws + lead->lay.bt_y), (size_t)lead->tc_rows * wide,
                                                   (size_t)spd::kTcTile * c0.vocab, reinterpret_cast<float *>(lead->ws + lead->lay.bt_ss),
-                                                  lead->grid, lead->stream, &launched);
+                                                  reinterpret_cast<int32_t *>(lead->ws + lead->lay.bt_out), lead->grid, lead->stream, &launched);
     lead->launches += launched;
     if (e != cudaSuccess) return cuda_fail(e, "batched timestep");
   }
@@ -847,21 +848,30 @@ int spd_batch_generate(spd_ctx *const *ctxs, int32_t n, int32_t n_steps) {
 int spd_batch_step(spd_ctx *const *ctxs, int32_t n, int32_t *out_ids, int32_t *out_parent, float *out_gamma) {
   int rc = batch_enqueue(ctxs, n, 1);
   if (rc) return rc;
-  if ((rc = batch_wait(ctxs, n))) return rc;
+  // One copy and one wait for the whole batch: the tail kernel left every request's state words and new tokens in
+  // its row of the leading context's results.  (The products record a wait that ran out in the leading context's
+  // state, which is row 0's.)
+  spd_ctx *lead = ctxs[0];
+  static_assert(SPD_MAX_K == spd::kMaxK, "the rows' lists are kMaxK apart");
+  std::vector<int32_t> rows((size_t)n * spd::kBtResultWords);
+  SPD_CUDA(cudaMemcpyAsync(rows.data(), lead->ws + lead->lay.bt_out, rows.size() * 4, cudaMemcpyDeviceToHost, lead->stream));
+  SPD_CUDA(cudaStreamSynchronize(lead->stream));
+  int first = SPD_OK;
   for (int r = 0; r < n; ++r) {
-    spd_ctx *x = ctxs[r];
-    const int k = x->cfg.k;
-    int32_t ids[SPD_MAX_K], par[SPD_MAX_K];
-    float gamma[SPD_MAX_K];
-    const size_t row = (size_t)(x->n_gen - 1) * k * 4;
-    SPD_CUDA(cudaMemcpyAsync(ids, x->ws + x->lay.hist_tok + row, (size_t)k * 4, cudaMemcpyDeviceToHost, x->stream));
-    SPD_CUDA(cudaMemcpyAsync(par, x->ws + x->lay.hist_par + row, (size_t)k * 4, cudaMemcpyDeviceToHost, x->stream));
-    if ((rc = read_state(x, offsetof(spd::State, gamma), gamma, sizeof gamma))) return rc;
-    SPD_CUDA(cudaStreamSynchronize(x->stream));
+    const int32_t *row = rows.data() + (size_t)r * spd::kBtResultWords;
+    if (row[2]) {
+      ctxs[r]->prefilled = false;
+      if (!first) first = row[2];
+    }
+  }
+  if (first) return first;
+  for (int r = 0; r < n; ++r) {
+    const int32_t *row = rows.data() + (size_t)r * spd::kBtResultWords;
+    const int k = ctxs[r]->cfg.k;
     for (int i = 0; i < k; ++i) {
-      if (out_ids) out_ids[r * SPD_MAX_K + i] = ids[i];
-      if (out_parent) out_parent[r * SPD_MAX_K + i] = par[i];
-      if (out_gamma) out_gamma[r * SPD_MAX_K + i] = gamma[i];
+      if (out_ids) out_ids[r * SPD_MAX_K + i] = row[8 + i];
+      if (out_parent) out_parent[r * SPD_MAX_K + i] = row[8 + spd::kMaxK + i];
+      if (out_gamma) std::memcpy(&out_gamma[r * SPD_MAX_K + i], &row[8 + 2 * spd::kMaxK + i], 4);
     }
   }
   return SPD_OK;

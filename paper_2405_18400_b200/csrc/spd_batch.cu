@@ -40,6 +40,7 @@ __device__ __forceinline__ void bt_put3(uint16_t *X, size_t term_stride, size_t 
 // multiply its rows by rsqrt(sum of the row's chunks / d + eps).
 constexpr int kBtCols = 512;      // columns per block: two per thread
 constexpr int kBtMaxChunks = 32;  // d_model <= 16384
+static_assert(8 + 3 * kMaxK <= kBtResultWords, "a request's row of results holds the head and three lists of k");
 
 __device__ __forceinline__ float bt_block_sum(float v, float *scratch) {
 #pragma unroll
@@ -284,7 +285,7 @@ __global__ void __launch_bounds__(128) spd_batch_attn_kernel(const float *Q, con
 // the sixteen lists (KeepTopK with log-probabilities under temperature tau, Algorithm 1); then Eq. 5-7, Eq. 2 and
 // Eq. 4 on the request's own draft state, as block 0 of the single-request kernel does.
 __global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const KParams *kps, const float *Y, int nz, size_t zs, const float *ss,
-                                                                          float eps, int V) {
+                                                                          float eps, int V, int32_t *results) {
   dep_wait();    // the kernel before this one in the stream wrote what this one reads
   dep_launch();  // the next one may set itself up meanwhile
   extern __shared__ __align__(16) uint8_t bt_smem[];
@@ -315,7 +316,27 @@ __global__ void __launch_bounds__(kConsumerThreads) spd_batch_tail_kernel(const 
   b.quit = &s_quit;
   b.bar_target = 0;
   b.c_stage = b.c_phase = 0;
-  tail_score_select(b, false, p.st->n_gen);
+  const int step = p.st->n_gen;
+  tail_score_select(b, false, step);
+  // The request's row of the batch's results, which the host fetches with one copy for all requests: the state's
+  // first words (stop, abort flag, error, error info, window length, tokens generated), then the k new tokens, their
+  // parents and gamma.
+  __syncthreads();
+  if (threadIdx.x < kBtResultWords) {
+    const State *st = p.st;
+    const int i = threadIdx.x;
+    int32_t v = 0;
+    if (i == 0) v = (int32_t)st->stop;
+    else if (i == 1) v = (int32_t)st->abort_flag;
+    else if (i == 2) v = st->err;
+    else if (i == 3) v = st->err_info;
+    else if (i == 4) v = st->win_len;
+    else if (i == 5) v = st->n_gen;
+    else if (i >= 8 && i < 8 + p.k) v = p.hist_tok[(size_t)step * p.k + (i - 8)];
+    else if (i >= 8 + kMaxK && i < 8 + kMaxK + p.k) v = p.hist_par[(size_t)step * p.k + (i - 8 - kMaxK)];
+    else if (i >= 8 + 2 * kMaxK && i < 8 + 2 * kMaxK + p.k) v = __float_as_int(st->gamma[i - 8 - 2 * kMaxK]);
+    results[(size_t)blockIdx.x * kBtResultWords + i] = v;
+  }
 }
 
 }  // namespace spd
@@ -328,8 +349,8 @@ constexpr size_t kBatchTailSmem = 20480;
 // job: the buffers of the context that lends its long-prefix workspace (h, y, q, x, tensor maps); y_logits: [128][V]
 // floats; lm_tmap: the LM head's tensor map.  *launches receives the number of kernels enqueued.
 extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd::KParams *kps, int n, int V, const __nv_bfloat16 *final_norm,
-                                               float *y_logits, size_t y_floats, size_t y_logits_floats, float *ss, int sm_count,
-                                               cudaStream_t s, int *launches) {
+                                               float *y_logits, size_t y_floats, size_t y_logits_floats, float *ss, int32_t *results,
+                                               int sm_count, cudaStream_t s, int *launches) {
   const spd::TcJob &j = *job;
   const int d = j.d, f = j.f;
   const size_t ts_d = (size_t)j.x_term_rows * d, ts_f = (size_t)j.x_term_rows * f;
@@ -373,7 +394,7 @@ extern "C" cudaError_t spd_internal_batch_step(const spd::TcJob *job, const spd:
   }
   gemm(xmap_d, 4 * j.L, y_logits, y_logits_floats, V, d);
   if (e == cudaSuccess) {
-    e = spd::launch_dep(spd::spd_batch_tail_kernel, dim3(n), dim3(spd::kConsumerThreads), kBatchTailSmem, s, kps, y_logits, nz, zs, ss, j.eps, V);
+    e = spd::launch_dep(spd::spd_batch_tail_kernel, dim3(n), dim3(spd::kConsumerThreads), kBatchTailSmem, s, kps, y_logits, nz, zs, ss, j.eps, V, results);
     ++count;
   }
   if (launches) *launches = count;

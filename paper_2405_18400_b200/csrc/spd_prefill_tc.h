@@ -30,6 +30,9 @@ struct TcJob {
   float *ss;                         // [128][32]: sums of squares of the residual rows per 512-column chunk (jobs of up to 128 tokens)
 };
 
+// Words of a request's row in a batched timestep's results (written by the tail kernel, fetched by the host in one copy).
+constexpr int kBtResultWords = 64;
+
 // Programmatic dependent launch.  dep_wait: returns once the kernel before this one in the stream has completed and
 // its writes are visible (at once when the launch did not ask for the overlap).  dep_launch: the kernel after this
 // one may be brought onto the SMs, where it runs up to its own dep_wait, as soon as every block of this kernel has
